@@ -1,0 +1,201 @@
+/*
+ * oda.h -- C ABI of the B200 On-Demand-Attention (ODA) decode library.
+ *
+ * One decode step of ODA on an attention stack over a block-table paged bf16 KV
+ * cache (Algorithm 1, lines 1-7, of the paper "On-Demand Attention"):
+ *   1. Local attention for every request over the access set of Eq. 1,
+ *        S^L = {first min(s,t) positions} U {last min(w,t) positions},
+ *   2. a recall head scores the post-Local state and writes one flag per request,
+ *   3. Full attention (S^F = all t positions) is recomputed only for flagged
+ *      requests on the gated layers, and replaces their Local output
+ *      (selected-state rule of the appendix on selected-state execution).
+ * The flag never leaves the device: step 3 reads it there.
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment
+ *     says "host".  The library allocates no device memory; its scratch is the
+ *     workspace the caller hands to oda_set_workspace().
+ *   - All work is enqueued on the stream argument (a cudaStream_t passed as
+ *     void*); nothing synchronises except oda_read_device_status() and
+ *     oda_step_host().  The device entry points may be stream-captured.
+ *   - Positions are 0-based here: request b has t = seq_lens[b] >= 1 positions
+ *     0..t-1, the current token's K/V already stored at position t-1.
+ *   - KV cache element (layer, block, token slot, kv head, d) of k_cache / v_cache
+ *     is at  kv_index(layer)*kv_layer_stride + block*kv_block_stride +
+ *     slot*kv_token_stride + head*kv_head_stride + d   (bf16 elements).  The d
+ *     values are contiguous, every stride is a multiple of 8 elements and the
+ *     base pointers are 16-byte aligned.  block = block_table[b*max_blocks_per_seq
+ *     + position/16].  Entries past ceil(t/16) are never read.
+ *   - q is [layers, batch, q_heads, head_dim] bf16; query head h reads KV head
+ *     h / (q_heads / kv_heads).  out has the same shape in fp32 (or bf16, see
+ *     out_dtype), lse is [layers, batch, q_heads] fp32 (natural log of the softmax
+ *     denominator, including the maximum).  The layer axis of q/out/lse always
+ *     spans all num_layers; a call touches rows layer_begin..layer_end-1.
+ *   - Errors a host check can see return a status with nothing enqueued.  Problems
+ *     only the device can see (seq_len < 1) set a sticky status word in the
+ *     workspace, readable with oda_read_device_status(); the kernels never trap.
+ *   - One context must not be used from two streams at once (the workspace is
+ *     shared scratch).
+ */
+#ifndef ODA_H
+#define ODA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct oda_ctx oda_ctx_t; /* opaque, host-owned */
+
+typedef enum {
+    ODA_OK = 0,
+    ODA_ERR_INVALID_ARG = 1,   /* null pointer, bad range, bad shape */
+    ODA_ERR_UNSUPPORTED = 2,   /* a shape this build has no kernel for */
+    ODA_ERR_WORKSPACE = 3,     /* workspace missing, misaligned or too small */
+    ODA_ERR_CUDA = 4,          /* a CUDA runtime call failed */
+    ODA_ERR_DEVICE_STATUS = 5  /* the device status word is non-zero */
+} oda_status_t;
+
+/* Which attention kernel runs (evidence for the design choice comes from timing both). */
+enum {
+    ODA_VARIANT_AUTO = 0,
+    ODA_VARIANT_SIMT = 1,  /* fp32 CUDA-core math, direct 128-bit global loads, warp-shuffle reductions */
+    ODA_VARIANT_TMA_MMA = 2 /* TMA-staged shared-memory ring, bf16 tensor-core GQA tile, fp32 accumulate */
+};
+
+typedef struct {
+    int32_t num_layers;         /* 1..256 */
+    int32_t num_q_heads;        /* multiple of num_kv_heads; group size 1, 2, 4 or 8 */
+    int32_t num_kv_heads;
+    int32_t head_dim;           /* 64 or 128 */
+    int32_t block_size;         /* tokens per KV block: 16 */
+    int32_t max_batch;          /* 1..256 */
+    int32_t max_blocks_per_seq; /* row length of block_table */
+    int32_t out_dtype;          /* 0 = fp32, 1 = bf16 */
+    float sm_scale;             /* logit scale; 0 => 1/sqrt(head_dim) */
+    int32_t variant;            /* ODA_VARIANT_* */
+    /* host arrays [num_layers], copied at create.  Eq. 1: window w >= 1 (includes the
+     * current token), sinks s >= 0.  gated: 1 = ODA layer (Local, Full on recall),
+     * 0 = fixed-window layer (always Local).  kv_index (nullable => identity): which
+     * layer slice of the cache holds this layer's K/V. */
+    const int32_t* layer_window;
+    const int32_t* layer_sinks;
+    const uint8_t* layer_gated;
+    const int32_t* layer_kv_index;
+    int64_t kv_layer_stride, kv_block_stride, kv_token_stride, kv_head_stride; /* bf16 elements */
+    /* Recall head x = [feat_ext (head_d_ext) ; flattened Local output of the last gated layer
+     * (q_heads*head_dim, present iff head_use_attn_out)], hidden width head_d_hidden.
+     * head_d_hidden = 0: no head (oda_step then needs override_flags). */
+    int32_t head_d_ext;
+    int32_t head_use_attn_out;
+    int32_t head_d_hidden;
+    int32_t reserved;
+} oda_config_t;
+
+/* Lifetime.  oda_create validates and copies the config (host only, no device work).
+ * Errors: INVALID_ARG, UNSUPPORTED. */
+oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx);
+void oda_destroy(oda_ctx_t* ctx);
+
+/* Scratch sizing: bytes the workspace must have for this config on the current device. */
+oda_status_t oda_workspace_bytes(const oda_ctx_t* ctx, size_t* bytes);
+/* Hands the library its scratch (256-byte aligned, caller-owned, must outlive the ctx's use).
+ * Initialises it (tickets, status, layer table) on `stream` and waits for that to finish. */
+oda_status_t oda_set_workspace(oda_ctx_t* ctx, void* dev_ptr, size_t bytes, void* stream);
+
+/*
+ * Local pass (Eq. 1, S^L) for layers [layer_begin, layer_end) and requests 0..batch-1:
+ * split-KV partials + log-sum-exp merge.  Writes out/lse rows of those layers.
+ * lse may be NULL.  batch = 0 is a no-op.
+ */
+oda_status_t oda_local_decode(oda_ctx_t* ctx, int32_t layer_begin, int32_t layer_end, int32_t batch,
+                              const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* block_table, const int32_t* seq_lens, void* out,
+                              float* lse, void* stream);
+
+/*
+ * Recall score and decision (Eq. 2 reduced to the benchmark's two-layer head; decision rule
+ * of Algorithm 1, line 3):  z = w2 . SiLU(W1 x + b1) + b2, score = sigmoid(z),
+ * flag = override_flags[b] if override_flags != NULL, else (z nonfinite) or (score > threshold).
+ * feat_ext [batch, head_d_ext] fp32 (NULL iff head_d_ext = 0); attn_out_last [batch, q_heads,
+ * head_dim] in out_dtype (NULL iff !head_use_attn_out); W1 [d_hidden, d_in] row-major fp32.
+ * Writes scores [batch] fp32, logits [batch] fp32 (nullable), flags [batch] u8 and, if
+ * counters != NULL ([batch,2] i32), counters[b] += {1, flag}.
+ */
+oda_status_t oda_recall_score(oda_ctx_t* ctx, int32_t batch, const float* feat_ext,
+                              const void* attn_out_last, const float* W1, const float* b1,
+                              const float* w2, const float* b2, float threshold,
+                              const uint8_t* override_flags, float* scores, float* logits,
+                              uint8_t* flags, int32_t* counters, void* stream);
+
+/*
+ * Gated Full pass (Eq. 1, S^F; Algorithm 1, line 4): for gated layers in [layer_begin,
+ * layer_end) and requests with flags[b] != 0, recomputes attention over all t positions and
+ * overwrites those rows of out/lse in place; every other row is left untouched.  The work
+ * list is built on the device from flags and seq_lens, so the bytes read scale with the
+ * flagged requests; no host read of the flags happens.
+ */
+oda_status_t oda_full_decode_gated(oda_ctx_t* ctx, int32_t layer_begin, int32_t layer_end,
+                                   int32_t batch, const void* q_full, const void* k_cache,
+                                   const void* v_cache, const int32_t* block_table,
+                                   const int32_t* seq_lens, const uint8_t* flags, void* out,
+                                   float* lse, void* stream);
+
+typedef struct {
+    int32_t batch;
+    int32_t advance_seq_lens; /* 1 => seq_lens[b] += 1 on the device at the end of the step */
+    const void* q_local;      /* [L,B,Hq,D] bf16 */
+    const void* q_full;       /* same shape; NULL => q_local */
+    const void* k_cache;
+    const void* v_cache;
+    const int32_t* block_table;
+    int32_t* seq_lens;
+    const float* feat_ext;    /* [B, head_d_ext] or NULL */
+    const float *W1, *b1, *w2, *b2; /* head parameters; ignored when head_d_hidden = 0 */
+    float threshold;
+    int32_t pad;
+    const uint8_t* override_flags; /* nullable: forced flags; the head still runs */
+    void* out;                /* [L,B,Hq,D] out_dtype: selected output */
+    float* lse;               /* nullable */
+    float* scores;            /* [B] */
+    float* logits;            /* [B] nullable */
+    uint8_t* flags;           /* [B] */
+    int32_t* counters;        /* [B,2] nullable */
+} oda_step_args_t;
+
+/* One whole step (Algorithm 1, lines 1-7): Local on all layers -> recall score on the last
+ * gated layer's Local output -> flags -> gated Full -> optional seq_lens advance. */
+oda_status_t oda_step(oda_ctx_t* ctx, const oda_step_args_t* args, void* stream);
+
+/*
+ * The same step for a caller whose per-step data lives in HOST memory: q_local, q_full,
+ * feat_ext, override_flags are host inputs, out, lse, scores, logits, flags host outputs
+ * (pinned memory makes the copies asynchronous); the KV cache, block table, seq_lens, head
+ * weights and counters stay device pointers (they are state, not per-step input).  Copies
+ * the inputs into staging areas of the workspace, runs oda_step, copies the results back and
+ * waits for the stream.  Reports the bytes copied each way if the pointers are non-NULL.
+ */
+oda_status_t oda_step_host(oda_ctx_t* ctx, const oda_step_args_t* args, void* stream,
+                           size_t* h2d_bytes, size_t* d2h_bytes);
+
+/* Reads and clears the sticky device status word (synchronises the stream).
+ * code: 0 ok; bit 0 = a request had seq_len < 1; bit 1 = work list overflowed its bound. */
+oda_status_t oda_read_device_status(oda_ctx_t* ctx, void* stream, int32_t* code);
+
+/* Kernel launches enqueued by this context since creation (for launch accounting). */
+int64_t oda_launch_count(const oda_ctx_t* ctx);
+/* The variant AUTO resolved to for this context (ODA_VARIANT_*). */
+int32_t oda_resolved_variant(const oda_ctx_t* ctx);
+/* Grid size (CTAs) the attention kernels of this context launch with. */
+int32_t oda_attention_grid(const oda_ctx_t* ctx);
+
+const char* oda_status_string(oda_status_t s);
+const char* oda_last_error(const oda_ctx_t* ctx); /* host string describing the last failure */
+const char* oda_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ODA_H */

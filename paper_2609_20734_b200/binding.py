@@ -1,0 +1,269 @@
+"""Thin ctypes binding over the C-ABI library (include/oda.h): argument marshalling only.
+
+torch is used for device memory and streams; every step of the path runs in the
+library's kernels.  There is no fallback: if the library is missing, or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liboda_b200.so")
+
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_TMA_MMA = 0, 1, 2
+
+EXPORTS = [
+    "oda_create", "oda_destroy", "oda_workspace_bytes", "oda_set_workspace", "oda_local_decode",
+    "oda_recall_score", "oda_full_decode_gated", "oda_step", "oda_step_host",
+    "oda_read_device_status", "oda_launch_count", "oda_resolved_variant", "oda_attention_grid",
+    "oda_status_string", "oda_last_error", "oda_version",
+]
+
+
+class OdaError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str = ""):
+        super().__init__(f"{what}: status {status} ({detail})")
+        self.status = status
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [
+        ("num_layers", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("block_size", ctypes.c_int32), ("max_batch", ctypes.c_int32),
+        ("max_blocks_per_seq", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+        ("sm_scale", ctypes.c_float), ("variant", ctypes.c_int32),
+        ("layer_window", ctypes.c_void_p), ("layer_sinks", ctypes.c_void_p),
+        ("layer_gated", ctypes.c_void_p), ("layer_kv_index", ctypes.c_void_p),
+        ("kv_layer_stride", ctypes.c_int64), ("kv_block_stride", ctypes.c_int64),
+        ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
+        ("head_d_ext", ctypes.c_int32), ("head_use_attn_out", ctypes.c_int32),
+        ("head_d_hidden", ctypes.c_int32), ("reserved", ctypes.c_int32),
+    ]
+
+
+class _StepArgs(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("advance_seq_lens", ctypes.c_int32),
+        ("q_local", ctypes.c_void_p), ("q_full", ctypes.c_void_p),
+        ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+        ("block_table", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p),
+        ("feat_ext", ctypes.c_void_p),
+        ("W1", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("w2", ctypes.c_void_p), ("b2", ctypes.c_void_p),
+        ("threshold", ctypes.c_float), ("pad", ctypes.c_int32),
+        ("override_flags", ctypes.c_void_p),
+        ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("scores", ctypes.c_void_p),
+        ("logits", ctypes.c_void_p), ("flags", ctypes.c_void_p), ("counters", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen the C-ABI library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float
+        lib.oda_create.argtypes = [ctypes.POINTER(_Config), ctypes.POINTER(vp)]
+        lib.oda_destroy.argtypes = [vp]
+        lib.oda_destroy.restype = None
+        lib.oda_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+        lib.oda_set_workspace.argtypes = [vp, vp, ctypes.c_size_t, vp]
+        lib.oda_local_decode.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oda_recall_score.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp]
+        lib.oda_full_decode_gated.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
+        lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
+                                      ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+        lib.oda_read_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+        lib.oda_launch_count.argtypes = [vp]
+        lib.oda_launch_count.restype = ctypes.c_int64
+        lib.oda_resolved_variant.argtypes = [vp]
+        lib.oda_attention_grid.argtypes = [vp]
+        lib.oda_status_string.argtypes = [ctypes.c_int]
+        lib.oda_status_string.restype = ctypes.c_char_p
+        lib.oda_last_error.argtypes = [vp]
+        lib.oda_last_error.restype = ctypes.c_char_p
+        lib.oda_version.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+@dataclass
+class OdaConfig:
+    num_layers: int
+    num_q_heads: int
+    num_kv_heads: int
+    head_dim: int
+    max_batch: int
+    max_blocks_per_seq: int
+    layer_window: Sequence[int]
+    layer_sinks: Sequence[int]
+    layer_gated: Sequence[int]
+    kv_layer_stride: int
+    kv_block_stride: int
+    kv_token_stride: int
+    kv_head_stride: int
+    layer_kv_index: Optional[Sequence[int]] = None
+    block_size: int = 16
+    out_dtype: int = 0
+    sm_scale: float = 0.0
+    variant: int = VARIANT_AUTO
+    head_d_ext: int = 0
+    head_use_attn_out: int = 1
+    head_d_hidden: int = 0
+    _keep: list = field(default_factory=list, repr=False)
+
+    def to_c(self) -> _Config:
+        def arr(x, dt):
+            if x is None:
+                return None
+            a = np.ascontiguousarray(np.asarray(x, dtype=dt))
+            self._keep.append(a)
+            return a.ctypes.data
+
+        return _Config(
+            self.num_layers, self.num_q_heads, self.num_kv_heads, self.head_dim, self.block_size,
+            self.max_batch, self.max_blocks_per_seq, self.out_dtype, self.sm_scale, self.variant,
+            arr(self.layer_window, np.int32), arr(self.layer_sinks, np.int32),
+            arr(self.layer_gated, np.uint8), arr(self.layer_kv_index, np.int32),
+            self.kv_layer_stride, self.kv_block_stride, self.kv_token_stride, self.kv_head_stride,
+            self.head_d_ext, self.head_use_attn_out, self.head_d_hidden, 0)
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or host) address of a torch tensor / numpy array / raw int; None stays NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"]
+        return t.ctypes.data
+    assert t.is_contiguous(), "tensors handed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    import torch
+
+    return torch.cuda.current_stream().cuda_stream
+
+
+class OdaContext:
+    """Owns an oda_ctx_t and (optionally) its workspace tensor."""
+
+    def __init__(self, cfg: OdaConfig, allocate_workspace: bool = True):
+        self.lib = load_library()
+        self.cfg = cfg
+        self._h = ctypes.c_void_p()
+        ccfg = cfg.to_c()
+        st = self.lib.oda_create(ctypes.byref(ccfg), ctypes.byref(self._h))
+        if st != 0:
+            raise OdaError(st, "oda_create", self.lib.oda_status_string(st).decode())
+        self.workspace = None
+        if allocate_workspace:
+            import torch
+
+            self.workspace = torch.empty(self.workspace_bytes(), dtype=torch.uint8, device="cuda")
+            self.set_workspace(self.workspace.data_ptr(), self.workspace.numel())
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            self.lib.oda_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    __del__ = close
+
+    def _check(self, st: int, what: str):
+        if st != 0:
+            raise OdaError(st, what, self.lib.oda_last_error(self._h).decode())
+
+    def workspace_bytes(self) -> int:
+        n = ctypes.c_size_t()
+        self._check(self.lib.oda_workspace_bytes(self._h, ctypes.byref(n)), "oda_workspace_bytes")
+        return n.value
+
+    def set_workspace(self, ptr: int, nbytes: int, stream: Optional[int] = None):
+        self._check(self.lib.oda_set_workspace(self._h, ptr, nbytes, _stream() if stream is None else stream),
+                    "oda_set_workspace")
+
+    # ---- the four calls of the path -------------------------------------------------
+    def local_decode(self, layer_begin, layer_end, batch, q, k_cache, v_cache, block_table, seq_lens,
+                     out, lse=None, stream=None):
+        self._check(self.lib.oda_local_decode(
+            self._h, layer_begin, layer_end, batch, _ptr(q), _ptr(k_cache), _ptr(v_cache),
+            _ptr(block_table), _ptr(seq_lens), _ptr(out), _ptr(lse),
+            _stream() if stream is None else stream), "oda_local_decode")
+
+    def recall_score(self, batch, feat_ext, attn_out_last, W1, b1, w2, b2, threshold, override_flags,
+                     scores, logits, flags, counters=None, stream=None):
+        self._check(self.lib.oda_recall_score(
+            self._h, batch, _ptr(feat_ext), _ptr(attn_out_last), _ptr(W1), _ptr(b1), _ptr(w2), _ptr(b2),
+            float(threshold), _ptr(override_flags), _ptr(scores), _ptr(logits), _ptr(flags),
+            _ptr(counters), _stream() if stream is None else stream), "oda_recall_score")
+
+    def full_decode_gated(self, layer_begin, layer_end, batch, q_full, k_cache, v_cache, block_table,
+                          seq_lens, flags, out, lse=None, stream=None):
+        self._check(self.lib.oda_full_decode_gated(
+            self._h, layer_begin, layer_end, batch, _ptr(q_full), _ptr(k_cache), _ptr(v_cache),
+            _ptr(block_table), _ptr(seq_lens), _ptr(flags), _ptr(out), _ptr(lse),
+            _stream() if stream is None else stream), "oda_full_decode_gated")
+
+    @staticmethod
+    def step_args(batch, q_local, k_cache, v_cache, block_table, seq_lens, out, scores, flags,
+                  q_full=None, feat_ext=None, head=None, threshold=0.5, override_flags=None, lse=None,
+                  logits=None, counters=None, advance_seq_lens=False) -> _StepArgs:
+        h = head or {}
+        return _StepArgs(
+            batch, 1 if advance_seq_lens else 0, _ptr(q_local), _ptr(q_full), _ptr(k_cache),
+            _ptr(v_cache), _ptr(block_table), _ptr(seq_lens), _ptr(feat_ext), _ptr(h.get("W1")),
+            _ptr(h.get("b1")), _ptr(h.get("w2")), _ptr(h.get("b2")), float(threshold), 0,
+            _ptr(override_flags), _ptr(out), _ptr(lse), _ptr(scores), _ptr(logits), _ptr(flags),
+            _ptr(counters))
+
+    def step(self, args: _StepArgs, stream=None):
+        self._check(self.lib.oda_step(self._h, ctypes.byref(args), _stream() if stream is None else stream),
+                    "oda_step")
+
+    def step_host(self, args: _StepArgs, stream=None):
+        up, down = ctypes.c_size_t(), ctypes.c_size_t()
+        self._check(self.lib.oda_step_host(self._h, ctypes.byref(args),
+                                           _stream() if stream is None else stream,
+                                           ctypes.byref(up), ctypes.byref(down)), "oda_step_host")
+        return up.value, down.value
+
+    # ---- introspection ----------------------------------------------------------------
+    def read_device_status(self, stream=None) -> int:
+        code = ctypes.c_int32()
+        st = self.lib.oda_read_device_status(self._h, _stream() if stream is None else stream,
+                                             ctypes.byref(code))
+        if st not in (0, 5):
+            self._check(st, "oda_read_device_status")
+        return code.value
+
+    @property
+    def launch_count(self) -> int:
+        return self.lib.oda_launch_count(self._h)
+
+    @property
+    def variant(self) -> int:
+        return self.lib.oda_resolved_variant(self._h)
+
+    @property
+    def attention_grid(self) -> int:
+        return self.lib.oda_attention_grid(self._h)
+
+
+def version() -> str:
+    return load_library().oda_version().decode()

@@ -1,0 +1,478 @@
+// C-ABI layer of the ODA decode library: argument validation, workspace layout and
+// stream-ordered kernel launches.  No device memory is allocated here, and nothing
+// synchronises except the two entry points whose contract says so.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/oda.h"
+#include "oda_device.cuh"
+#include "oda_launch.h"
+
+using namespace oda;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct WsLayout {
+    size_t status, layers, tickets, head_partial, partials;
+    size_t st_q_local, st_q_full, st_feat, st_override, st_out, st_lse, st_scores, st_logits, st_flags;
+    size_t total;
+};
+
+}  // namespace
+
+struct oda_ctx {
+    oda_config_t cfg;
+    std::vector<LayerInfo> layers;
+    int ncls = 0;
+    int cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
+    int group = 1;
+    int last_gated = -1;
+    float scale = 0.f;
+    int num_sms = 148;
+    int variant = ODA_VARIANT_SIMT;
+    int grid = 148;
+    int items_per_cta = 4;
+    int min_chunk_pages = 4;
+    int max_items = 0;
+    int head_grid = 1;
+    WsLayout lay{};
+    char* ws = nullptr;
+    int64_t launches = 0;
+    std::string err;
+};
+
+namespace {
+
+oda_status_t fail(oda_ctx* c, oda_status_t s, const std::string& msg)
+{
+    if (c) c->err = msg;
+    return s;
+}
+
+oda_status_t cuda_fail(oda_ctx* c, cudaError_t e, const char* what)
+{
+    return fail(c, ODA_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+size_t out_elem(const oda_ctx* c) { return c->cfg.out_dtype ? 2 : 4; }
+
+void compute_layout(oda_ctx* c)
+{
+    const oda_config_t& f = c->cfg;
+    const size_t L = f.num_layers, B = f.max_batch, Hq = f.num_q_heads, D = f.head_dim;
+    WsLayout& w = c->lay;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    w.status = take(256);
+    w.layers = take(L * sizeof(LayerInfo));
+    w.tickets = take(L * B * f.num_kv_heads * sizeof(int32_t));
+    w.head_partial = take((size_t)c->head_grid * B * sizeof(float));
+    w.partials = take((size_t)c->max_items * c->group * (D + 2) * sizeof(float));
+    w.st_q_local = take(L * B * Hq * D * 2);
+    w.st_q_full = take(L * B * Hq * D * 2);
+    w.st_feat = take(B * (size_t)(f.head_d_ext > 0 ? f.head_d_ext : 1) * 4);
+    w.st_override = take(B);
+    w.st_out = take(L * B * Hq * D * out_elem(c));
+    w.st_lse = take(L * B * Hq * 4);
+    w.st_scores = take(B * 4);
+    w.st_logits = take(B * 4);
+    w.st_flags = take(B);
+    w.total = off;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+oda_status_t check_attn_args(oda_ctx* c, int lb, int le, int batch, const void* q, const void* k,
+                             const void* v, const int32_t* bt, const int32_t* sl, void* out)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    if (lb < 0 || le > c->cfg.num_layers || lb > le) return fail(c, ODA_ERR_INVALID_ARG, "bad layer range");
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0 || lb == le) return ODA_OK;
+    if (!q || !k || !v || !bt || !sl || !out) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return fail(c, ODA_ERR_INVALID_ARG, "q, k_cache, v_cache and out must be 16-byte aligned");
+    return ODA_OK;
+}
+
+oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, const void* q,
+                              const void* k, const void* v, const int32_t* bt, const int32_t* sl,
+                              const uint8_t* flags, void* out, float* lse, cudaStream_t st)
+{
+    const oda_config_t& f = c->cfg;
+    AttnParams p;
+    std::memset(&p, 0, sizeof p);
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k = static_cast<const __nv_bfloat16*>(k);
+    p.v = static_cast<const __nv_bfloat16*>(v);
+    p.block_table = bt;
+    p.seq_lens = sl;
+    p.flags = flags;
+    p.out = out;
+    p.lse = lse;
+    p.partials = reinterpret_cast<float*>(c->ws + c->lay.partials);
+    p.tickets = reinterpret_cast<int32_t*>(c->ws + c->lay.tickets);
+    p.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    p.layers = reinterpret_cast<const LayerInfo*>(c->ws + c->lay.layers);
+    p.kv_layer_stride = f.kv_layer_stride;
+    p.kv_block_stride = f.kv_block_stride;
+    p.kv_token_stride = f.kv_token_stride;
+    p.kv_head_stride = f.kv_head_stride;
+    p.layer_begin = lb;
+    p.layer_end = le;
+    p.batch = batch;
+    p.max_batch = f.max_batch;
+    p.num_q_heads = f.num_q_heads;
+    p.num_kv_heads = f.num_kv_heads;
+    p.max_blocks_per_seq = f.max_blocks_per_seq;
+    p.out_bf16 = f.out_dtype;
+    p.mode = mode;
+    p.ncls = c->ncls;
+    p.items_per_cta = c->items_per_cta;
+    p.min_chunk_pages = c->min_chunk_pages;
+    p.max_items = c->max_items;
+    p.scale_log2e = c->scale * 1.4426950408889634f;
+    bool any = false;
+    for (int i = 0; i < c->ncls; ++i) {
+        p.cls_window[i] = c->cls_window[i];
+        p.cls_sinks[i] = c->cls_sinks[i];
+        p.cls_gated[i] = c->cls_gated[i];
+        int n = 0;
+        for (int l = lb; l < le; ++l) n += (c->layers[l].cls == i);
+        p.cls_layers_in_call[i] = n;
+        if (n && (mode == 0 || c->cls_gated[i])) any = true;
+    }
+    if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
+    cudaError_t e = launch_splitkv_simt(p, f.head_dim, c->group, c->grid, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "attention kernel launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* oda_version(void) { return "oda-b200 0.1 (sm_100a)"; }
+
+const char* oda_status_string(oda_status_t s)
+{
+    switch (s) {
+        case ODA_OK: return "ok";
+        case ODA_ERR_INVALID_ARG: return "invalid argument";
+        case ODA_ERR_UNSUPPORTED: return "unsupported shape";
+        case ODA_ERR_WORKSPACE: return "workspace missing or too small";
+        case ODA_ERR_CUDA: return "CUDA runtime error";
+        case ODA_ERR_DEVICE_STATUS: return "device status word set";
+    }
+    return "unknown status";
+}
+
+const char* oda_last_error(const oda_ctx_t* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+int64_t oda_launch_count(const oda_ctx_t* ctx) { return ctx ? ctx->launches : 0; }
+int32_t oda_resolved_variant(const oda_ctx_t* ctx) { return ctx ? ctx->variant : 0; }
+int32_t oda_attention_grid(const oda_ctx_t* ctx) { return ctx ? ctx->grid : 0; }
+
+oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
+{
+    if (!cfg || !out_ctx) return ODA_ERR_INVALID_ARG;
+    *out_ctx = nullptr;
+    if (cfg->num_layers < 1 || cfg->num_layers > kMaxLayers) return ODA_ERR_INVALID_ARG;
+    if (cfg->num_kv_heads < 1 || cfg->num_q_heads < 1 || cfg->num_q_heads % cfg->num_kv_heads)
+        return ODA_ERR_INVALID_ARG;
+    if (cfg->max_batch < 1 || cfg->max_batch > kMaxBatch || cfg->max_blocks_per_seq < 1)
+        return ODA_ERR_INVALID_ARG;
+    if (!cfg->layer_window || !cfg->layer_sinks || !cfg->layer_gated) return ODA_ERR_INVALID_ARG;
+    if (cfg->out_dtype != 0 && cfg->out_dtype != 1) return ODA_ERR_INVALID_ARG;
+    if (!(cfg->sm_scale >= 0.f) || !std::isfinite(cfg->sm_scale)) return ODA_ERR_INVALID_ARG;
+    if (cfg->head_d_ext < 0 || cfg->head_d_hidden < 0) return ODA_ERR_INVALID_ARG;
+    if (cfg->variant < ODA_VARIANT_AUTO || cfg->variant > ODA_VARIANT_TMA_MMA) return ODA_ERR_INVALID_ARG;
+    const int group = cfg->num_q_heads / cfg->num_kv_heads;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return ODA_ERR_UNSUPPORTED;
+    if (cfg->block_size != kPage) return ODA_ERR_UNSUPPORTED;
+    if (group != 1 && group != 2 && group != 4 && group != 8) return ODA_ERR_UNSUPPORTED;
+    const int64_t strides[4] = {cfg->kv_layer_stride, cfg->kv_block_stride, cfg->kv_token_stride, cfg->kv_head_stride};
+    for (int64_t s : strides)
+        if (s < 0 || (s % 8) != 0) return ODA_ERR_INVALID_ARG;
+    if (cfg->kv_token_stride < cfg->head_dim || cfg->kv_head_stride < cfg->head_dim ||
+        cfg->kv_block_stride < (int64_t)cfg->head_dim * kPage)
+        return ODA_ERR_INVALID_ARG;
+
+    oda_ctx* c = new (std::nothrow) oda_ctx();
+    if (!c) return ODA_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->group = group;
+    c->scale = cfg->sm_scale > 0.f ? cfg->sm_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+    c->layers.resize(cfg->num_layers);
+    int max_kv_index = 0;
+    for (int l = 0; l < cfg->num_layers; ++l) {
+        LayerInfo li{};
+        li.window = cfg->layer_window[l];
+        li.sinks = cfg->layer_sinks[l];
+        li.gated = cfg->layer_gated[l] ? 1 : 0;
+        li.kv_index = cfg->layer_kv_index ? cfg->layer_kv_index[l] : l;
+        if (li.window < 1 || li.sinks < 0 || li.kv_index < 0) {
+            delete c;
+            return ODA_ERR_INVALID_ARG;
+        }
+        if (li.kv_index > max_kv_index) max_kv_index = li.kv_index;
+        int cls = -1;
+        for (int i = 0; i < c->ncls; ++i)
+            if (c->cls_window[i] == li.window && c->cls_sinks[i] == li.sinks && c->cls_gated[i] == li.gated) cls = i;
+        if (cls < 0) {
+            if (c->ncls == kMaxClasses) {
+                delete c;
+                return ODA_ERR_UNSUPPORTED;  // more than kMaxClasses distinct (window, sinks, gated)
+            }
+            cls = c->ncls++;
+            c->cls_window[cls] = li.window;
+            c->cls_sinks[cls] = li.sinks;
+            c->cls_gated[cls] = li.gated;
+        }
+        li.cls = cls;
+        if (li.gated) c->last_gated = l;
+        c->layers[l] = li;
+    }
+    c->cfg.layer_window = nullptr;  // the copies above are what the library uses
+    c->cfg.layer_sinks = nullptr;
+    c->cfg.layer_gated = nullptr;
+    c->cfg.layer_kv_index = nullptr;
+    (void)max_kv_index;
+
+    c->variant = ODA_VARIANT_SIMT;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+        c->num_sms = sms;
+        int occ = occupancy_splitkv_simt(cfg->head_dim, group);
+        c->grid = sms * (occ > 0 ? occ : 1);
+    } else {
+        (void)cudaGetLastError();
+        c->num_sms = 148;  // no device visible: sizes follow a B200 so that host-only checks still work
+        c->grid = 148 * 2;
+    }
+    c->max_items = c->grid * c->items_per_cta + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
+    c->head_grid = cfg->head_d_hidden > 0 ? recall_head_grid(cfg->head_d_hidden) : 1;
+    compute_layout(c);
+    *out_ctx = c;
+    return ODA_OK;
+}
+
+void oda_destroy(oda_ctx_t* ctx) { delete ctx; }
+
+oda_status_t oda_workspace_bytes(const oda_ctx_t* ctx, size_t* bytes)
+{
+    if (!ctx || !bytes) return ODA_ERR_INVALID_ARG;
+    *bytes = ctx->lay.total;
+    return ODA_OK;
+}
+
+oda_status_t oda_set_workspace(oda_ctx_t* c, void* dev_ptr, size_t bytes, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!dev_ptr || (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0)
+        return fail(c, ODA_ERR_WORKSPACE, "workspace pointer is null or not 256-byte aligned");
+    if (bytes < c->lay.total) return fail(c, ODA_ERR_WORKSPACE, "workspace smaller than oda_workspace_bytes()");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(dev_ptr);
+    cudaError_t e = cudaMemsetAsync(ws, 0, c->lay.partials, st);  // status, tickets, head scratch
+    if (e != cudaSuccess) return cuda_fail(c, e, "workspace memset");
+    e = cudaMemcpyAsync(ws + c->lay.layers, c->layers.data(), c->layers.size() * sizeof(LayerInfo),
+                        cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "layer table upload");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "workspace initialisation");
+    c->ws = ws;
+    return ODA_OK;
+}
+
+oda_status_t oda_local_decode(oda_ctx_t* c, int32_t lb, int32_t le, int32_t batch, const void* q,
+                              const void* k, const void* v, const int32_t* bt, const int32_t* sl,
+                              void* out, float* lse, void* stream)
+{
+    oda_status_t s = check_attn_args(c, lb, le, batch, q, k, v, bt, sl, out);
+    if (s != ODA_OK || batch == 0 || lb == le) return s;
+    return launch_attention(c, 0, lb, le, batch, q, k, v, bt, sl, nullptr, out, lse,
+                            static_cast<cudaStream_t>(stream));
+}
+
+oda_status_t oda_full_decode_gated(oda_ctx_t* c, int32_t lb, int32_t le, int32_t batch, const void* q,
+                                   const void* k, const void* v, const int32_t* bt, const int32_t* sl,
+                                   const uint8_t* flags, void* out, float* lse, void* stream)
+{
+    oda_status_t s = check_attn_args(c, lb, le, batch, q, k, v, bt, sl, out);
+    if (s != ODA_OK || batch == 0 || lb == le) return s;
+    if (!flags) return fail(c, ODA_ERR_INVALID_ARG, "flags is null");
+    return launch_attention(c, 1, lb, le, batch, q, k, v, bt, sl, flags, out, lse,
+                            static_cast<cudaStream_t>(stream));
+}
+
+oda_status_t oda_recall_score(oda_ctx_t* c, int32_t batch, const float* feat_ext, const void* attn_out_last,
+                              const float* W1, const float* b1, const float* w2, const float* b2,
+                              float threshold, const uint8_t* override_flags, float* scores,
+                              float* logits, uint8_t* flags, int32_t* counters, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0) return ODA_OK;
+    if (!scores || !flags) return fail(c, ODA_ERR_INVALID_ARG, "scores or flags is null");
+    const oda_config_t& f = c->cfg;
+    HeadParams p;
+    std::memset(&p, 0, sizeof p);
+    p.d_hidden = f.head_d_hidden;
+    if (f.head_d_hidden > 0) {
+        p.d_ext = f.head_d_ext;
+        p.d_attn = f.head_use_attn_out ? f.num_q_heads * f.head_dim : 0;
+        if (!W1 || !b1 || !w2 || !b2) return fail(c, ODA_ERR_INVALID_ARG, "head weights are null");
+        if (p.d_ext > 0 && !feat_ext) return fail(c, ODA_ERR_INVALID_ARG, "feat_ext is null but head_d_ext > 0");
+        if (p.d_attn > 0 && !attn_out_last) return fail(c, ODA_ERR_INVALID_ARG, "attn_out_last is null but head_use_attn_out is set");
+        if (p.d_ext + p.d_attn < 1) return fail(c, ODA_ERR_INVALID_ARG, "the head has no input");
+    } else if (!override_flags) {
+        return fail(c, ODA_ERR_INVALID_ARG, "no head configured and no override_flags given");
+    }
+    p.feat_ext = feat_ext;
+    p.attn_out = attn_out_last;
+    p.W1 = W1; p.b1 = b1; p.w2 = w2; p.b2 = b2;
+    p.override_flags = override_flags;
+    p.scores = scores;
+    p.logits = logits;
+    p.flags = flags;
+    p.counters = counters;
+    p.partial = reinterpret_cast<float*>(c->ws + c->lay.head_partial);
+    p.ticket = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 64);
+    p.batch = batch;
+    p.attn_bf16 = f.out_dtype;
+    p.max_batch = f.max_batch;
+    p.threshold = threshold;
+    cudaError_t e = launch_recall_head(p, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(c, e, "recall head launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
+oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
+{
+    if (!c || !a) return ODA_ERR_INVALID_ARG;
+    const oda_config_t& f = c->cfg;
+    const int B = a->batch, L = f.num_layers;
+    oda_status_t s = check_attn_args(c, 0, L, B, a->q_local, a->k_cache, a->v_cache, a->block_table,
+                                     a->seq_lens, a->out);
+    if (s != ODA_OK || B == 0) return s;
+    if (!a->scores || !a->flags) return fail(c, ODA_ERR_INVALID_ARG, "scores or flags is null");
+    if (f.head_d_hidden == 0 && !a->override_flags)
+        return fail(c, ODA_ERR_INVALID_ARG, "no head configured and no override_flags given");
+    const void* qf = a->q_full ? a->q_full : a->q_local;
+    if (!aligned16(qf)) return fail(c, ODA_ERR_INVALID_ARG, "q_full must be 16-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = launch_attention(c, 0, 0, L, B, a->q_local, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
+                         nullptr, a->out, a->lse, st);
+    if (s != ODA_OK) return s;
+    const char* attn_last = nullptr;
+    if (c->last_gated >= 0 && f.head_use_attn_out)
+        attn_last = static_cast<const char*>(a->out) + (size_t)c->last_gated * B * f.num_q_heads * f.head_dim * out_elem(c);
+    s = oda_recall_score(c, B, a->feat_ext, attn_last, a->W1, a->b1, a->w2, a->b2, a->threshold,
+                         a->override_flags, a->scores, a->logits, a->flags, a->counters, stream);
+    if (s != ODA_OK) return s;
+    if (c->last_gated >= 0) {
+        s = launch_attention(c, 1, 0, L, B, qf, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
+                             a->flags, a->out, a->lse, st);
+        if (s != ODA_OK) return s;
+    }
+    if (a->advance_seq_lens) {
+        cudaError_t e = launch_advance_seq_lens(a->seq_lens, B, st);
+        if (e != cudaSuccess) return cuda_fail(c, e, "seq_lens advance launch");
+        c->launches += 1;
+    }
+    return ODA_OK;
+}
+
+oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream, size_t* h2d_bytes,
+                           size_t* d2h_bytes)
+{
+    if (!c || !a) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    const oda_config_t& f = c->cfg;
+    const int B = a->batch;
+    if (B < 0 || B > f.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (h2d_bytes) *h2d_bytes = 0;
+    if (d2h_bytes) *d2h_bytes = 0;
+    if (B == 0) return ODA_OK;
+    if (!a->q_local || !a->out || !a->scores || !a->flags) return fail(c, ODA_ERR_INVALID_ARG, "null host pointer");
+    if (f.head_d_ext > 0 && f.head_d_hidden > 0 && !a->feat_ext) return fail(c, ODA_ERR_INVALID_ARG, "feat_ext is null");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t rows = (size_t)f.num_layers * B * f.num_q_heads;
+    const size_t qbytes = rows * f.head_dim * 2;
+    size_t up = 0, down = 0;
+    oda_step_args_t d = *a;
+    cudaError_t e;
+#define ODA_UP(field, off, bytes)                                                                     \
+    do {                                                                                              \
+        e = cudaMemcpyAsync(c->ws + c->lay.off, a->field, (bytes), cudaMemcpyHostToDevice, st);       \
+        if (e != cudaSuccess) return cuda_fail(c, e, "host-to-device copy of " #field);               \
+        up += (bytes);                                                                                \
+    } while (0)
+    ODA_UP(q_local, st_q_local, qbytes);
+    d.q_local = c->ws + c->lay.st_q_local;
+    if (a->q_full) {
+        ODA_UP(q_full, st_q_full, qbytes);
+        d.q_full = c->ws + c->lay.st_q_full;
+    }
+    if (a->feat_ext && f.head_d_ext > 0) {
+        ODA_UP(feat_ext, st_feat, (size_t)B * f.head_d_ext * 4);
+        d.feat_ext = reinterpret_cast<const float*>(c->ws + c->lay.st_feat);
+    }
+    if (a->override_flags) {
+        ODA_UP(override_flags, st_override, (size_t)B);
+        d.override_flags = reinterpret_cast<const uint8_t*>(c->ws + c->lay.st_override);
+    }
+#undef ODA_UP
+    d.out = c->ws + c->lay.st_out;
+    d.lse = a->lse ? reinterpret_cast<float*>(c->ws + c->lay.st_lse) : nullptr;
+    d.scores = reinterpret_cast<float*>(c->ws + c->lay.st_scores);
+    d.logits = a->logits ? reinterpret_cast<float*>(c->ws + c->lay.st_logits) : nullptr;
+    d.flags = reinterpret_cast<uint8_t*>(c->ws + c->lay.st_flags);
+    oda_status_t s = oda_step(c, &d, stream);
+    if (s != ODA_OK) return s;
+#define ODA_DOWN(field, off, bytes)                                                                   \
+    do {                                                                                              \
+        e = cudaMemcpyAsync(a->field, c->ws + c->lay.off, (bytes), cudaMemcpyDeviceToHost, st);       \
+        if (e != cudaSuccess) return cuda_fail(c, e, "device-to-host copy of " #field);               \
+        down += (bytes);                                                                              \
+    } while (0)
+    ODA_DOWN(out, st_out, rows * f.head_dim * out_elem(c));
+    if (a->lse) ODA_DOWN(lse, st_lse, rows * 4);
+    ODA_DOWN(scores, st_scores, (size_t)B * 4);
+    if (a->logits) ODA_DOWN(logits, st_logits, (size_t)B * 4);
+    ODA_DOWN(flags, st_flags, (size_t)B);
+#undef ODA_DOWN
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronise");
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = down;
+    return ODA_OK;
+}
+
+oda_status_t oda_read_device_status(oda_ctx_t* c, void* stream, int32_t* code)
+{
+    if (!c || !code) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, c->ws + c->lay.status, sizeof v, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->lay.status, 0, sizeof v, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "status read");
+    *code = v;
+    return v ? ODA_ERR_DEVICE_STATUS : ODA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,173 @@
+"""GPU parity: the CUDA attention kernels, called through the C-ABI, against the fp64 oracle on
+the same seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_20734_b200 import binding, synth
+from tests import gpu_helpers as gh
+from tests.helpers import make_problem, oracle_attention
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [binding.VARIANT_SIMT]
+RAGGED = [1, 15, 16, 17, 300, 1000, 2053]
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("D,Hq,Hkv", [(128, 8, 2), (128, 8, 1), (64, 4, 1), (64, 4, 4), (128, 4, 2)])
+@pytest.mark.parametrize("layout", ["hnd", "nhd"])
+def test_local_parity_ragged(variant, D, Hq, Hkv, layout):
+    L = 3
+    prob = make_problem(100 + D + Hq, L, len(RAGGED), Hq, Hkv, D, RAGGED, layout=layout)
+    windows, sinks, gated = [256, 64, 1024], [4, 0, 17], [1, 0, 1]
+    ctx = gh.make_ctx(prob, windows, sinks, gated, variant=variant)
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8)
+    gh.assert_close(out, ref, gh.ATOL_OUT, "local out")
+    gh.assert_close(lse, rlse, gh.ATOL_LSE, "local lse")
+    assert ctx.read_device_status() == 0
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("D,Hq,Hkv", [(128, 8, 2), (64, 8, 1)])
+def test_full_gated_parity_and_untouched_rows(variant, D, Hq, Hkv):
+    L = 4
+    seq = [700, 33, 1, 4100, 257]
+    prob = make_problem(7 + D, L, len(seq), Hq, Hkv, D, seq, layout="hnd")
+    windows, sinks, gated = [64, 32, 64, 32], [4, 0, 4, 0], [1, 0, 1, 0]
+    ctx = gh.make_ctx(prob, windows, sinks, gated, variant=variant)
+    dev = gh.upload(prob)
+    flags_h = np.array([1, 0, 1, 1, 0], dtype=np.uint8)
+    flags = torch.from_numpy(flags_h).cuda()
+    out, lse = gh.new_out(prob, fill=-77.0)
+    ctx.full_decode_gated(0, L, len(seq), dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
+                          flags, out, lse)
+    torch.cuda.synchronize()
+    out, lse = out.cpu().numpy(), lse.cpu().numpy()
+    ref, rlse = oracle_attention(prob, "full", windows, sinks, nthreads=8)
+    for l in range(L):
+        for b in range(len(seq)):
+            if gated[l] and flags_h[b]:
+                gh.assert_close(out[l, b], ref[l, b], gh.ATOL_OUT, f"full out l{l} b{b}")
+                gh.assert_close(lse[l, b], rlse[l, b], gh.ATOL_LSE, f"full lse l{l} b{b}")
+            else:
+                assert (out[l, b] == -77.0).all() and (lse[l, b] == -77.0).all()
+    # all flags 0: nothing is written at all
+    out2, lse2 = gh.new_out(prob, fill=-5.0)
+    ctx.full_decode_gated(0, L, len(seq), dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
+                          torch.zeros(len(seq), dtype=torch.uint8, device="cuda"), out2, lse2)
+    torch.cuda.synchronize()
+    assert (out2 == -5.0).all().item()
+    assert ctx.read_device_status() == 0
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_window_covering_sequence_equals_full(variant):
+    seq = [5, 640, 1023]
+    prob = make_problem(3, 2, 3, 8, 2, 128, seq)
+    ctx = gh.make_ctx(prob, [1024, 2048], [0, 4], [1, 1], variant=variant)
+    dev = gh.upload(prob)
+    loc, llse = gh.gpu_local(ctx, prob, dev)
+    out, lse = gh.new_out(prob)
+    ctx.full_decode_gated(0, 2, 3, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
+                          torch.ones(3, dtype=torch.uint8, device="cuda"), out, lse)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(out.cpu().numpy(), loc, rtol=0, atol=1e-6)
+    np.testing.assert_allclose(lse.cpu().numpy(), llse, rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_slots_past_the_sequence_and_unused_table_entries_are_never_used(variant):
+    """Slots after position t-1 of the last page hold NaN bit patterns and table entries past
+    ceil(t/16) are -1: the result must not change."""
+    seq = [37, 130]
+    prob = make_problem(9, 1, 2, 4, 1, 128, seq, shuffled=True)
+    ref, _ = oracle_attention(prob, "local", [48], [4])
+    lay = prob["layout"]
+    for b, t in enumerate(seq):
+        blk = int(prob["table"][b, (t - 1) // 16])
+        for slot in range(t % 16, 16) if t % 16 else []:
+            off = blk * lay.block_stride + slot * lay.token_stride
+            prob["k"][off:off + 128] = 0x7FC0
+            prob["v"][off:off + 128] = 0x7FC0
+    assert (prob["table"][0, 3:] == -1).all()
+    ctx = gh.make_ctx(prob, [48], [4], [1], variant=variant)
+    out, _ = gh.gpu_local(ctx, prob, gh.upload(prob))
+    gh.assert_close(out, ref, gh.ATOL_OUT, "poisoned tail")
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_layer_ranges_kv_index_batch_prefix_and_determinism(variant):
+    seq = [90, 500, 31]
+    prob = make_problem(13, 4, 3, 8, 2, 128, seq, kv_layers=2)
+    kvmap = [1, 0, 1, 0]
+    windows, sinks, gated = [64] * 4, [4] * 4, [1] * 4
+    ctx = gh.make_ctx(prob, windows, sinks, gated, kv_index=kvmap, variant=variant)
+    dev = gh.upload(prob)
+    ref, _ = oracle_attention(prob, "local", windows, sinks, layer_kv_index=kvmap, nthreads=8)
+    whole, _ = gh.gpu_local(ctx, prob, dev)
+    gh.assert_close(whole, ref, gh.ATOL_OUT, "kv_index")
+    part, _ = gh.gpu_local(ctx, prob, dev, lb=1, le=3)
+    assert np.isnan(part[0]).all() and np.isnan(part[3]).all()
+    np.testing.assert_array_equal(part[1:3], whole[1:3])       # same bits: run-to-run determinism
+    again, _ = gh.gpu_local(ctx, prob, dev)
+    np.testing.assert_array_equal(again, whole)
+    # batch = 0 and an empty layer range are no-ops
+    out, lse = gh.new_out(prob, fill=3.0)
+    ctx.local_decode(0, 4, 0, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out, lse)
+    ctx.local_decode(2, 2, 3, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out, lse)
+    torch.cuda.synchronize()
+    assert (out == 3.0).all().item()
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_custom_scale_and_bf16_output(variant):
+    seq = [200, 77]
+    prob = make_problem(17, 1, 2, 4, 2, 64, seq)
+    ctx = gh.make_ctx(prob, [96], [2], [1], variant=variant, sm_scale=0.2, out_dtype=1)
+    dev = gh.upload(prob)
+    out = torch.zeros((1, 2, 4, 64), dtype=torch.bfloat16, device="cuda")
+    ctx.local_decode(0, 1, 2, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out, None)
+    torch.cuda.synchronize()
+    ref, _ = oracle_attention(prob, "local", [96], [2], sm_scale=0.2)
+    got = out.float().cpu().numpy().astype(np.float64)
+    # bf16 output: within half a bf16 ulp of a value that meets the fp32 bar
+    assert (np.abs(got - ref) <= gh.ATOL_OUT + np.abs(ref) * 2.0 ** -8).all()
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_bad_seq_len_sets_status_without_trapping(variant):
+    prob = make_problem(19, 1, 2, 4, 1, 64, [40, 40])
+    ctx = gh.make_ctx(prob, [16], [0], [1], variant=variant)
+    dev = gh.upload(prob)
+    dev["seq_lens"] = torch.tensor([0, 40], dtype=torch.int32, device="cuda")
+    out, lse = gh.new_out(prob, fill=9.0)
+    ctx.local_decode(0, 1, 2, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out, lse)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() & 1
+    assert ctx.read_device_status() == 0           # reading clears it
+    assert (out[0, 0] == 9.0).all().item()         # the bad row is left alone
+    ref, _ = oracle_attention(prob, "local", [16], [0])
+    gh.assert_close(out[0, 1].cpu().numpy(), ref[0, 1], gh.ATOL_OUT, "good row")
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_peaked_softmax_short_sequences(variant):
+    """Few tokens and large logits: the regime where rounding of the softmax weights would show."""
+    seq = [2, 3, 5, 9]
+    prob = make_problem(23, 1, 4, 8, 1, 128, seq)
+    q = synth.bf16_bits_to_f32(prob["q"]) * 3.0
+    prob["q"] = synth.f32_to_bf16_bits(q).reshape(prob["q"].shape)
+    ctx = gh.make_ctx(prob, [4], [1], [1], variant=variant)
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", [4], [1])
+    gh.assert_close(out, ref, gh.ATOL_OUT, "peaked local")
+    out2, _ = gh.new_out(prob)
+    ctx.full_decode_gated(0, 1, 4, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
+                          torch.ones(4, dtype=torch.uint8, device="cuda"), out2, None)
+    torch.cuda.synchronize()
+    reff, _ = oracle_attention(prob, "full", [4], [1])
+    gh.assert_close(out2.cpu().numpy(), reff, gh.ATOL_OUT, "peaked full")
