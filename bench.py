@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the ODA decode-attention step (one JSON line on stdout).
+
+A step is one pass of the whole hot path -- Local attention on every layer, recall score,
+device-side flags, gated Full attention, seq_lens advance -- for one batch of synthetic
+requests of the Llama-3-8B-shaped configuration (32 layers, 32q/8kv heads, D=128, batch 1,
+context 32768, window 1024 + 4 sinks, block size 16, bf16 KV ~ N(0,1), flags forced by a
+seeded Bernoulli draw).  The step is replayed from one CUDA graph; its time is taken with
+CUDA events around each replay, with an untimed L2 flush between steps.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attention_tokens_per_s"
+UNIT = "tokens/s"
+SWEEP_RATES = [0.0, 0.1, 0.25, 0.5, 1.0]
+FLUSH_BYTES = 256 << 20
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llama8b")
+    ap.add_argument("--recall-rate", type=float, default=0.25)
+    ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 SIMT, 2 TMA+MMA")
+    ap.add_argument("--sinks", type=int, default=None)
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--kernel-reps", type=int, default=10)
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def reference_arm(args, wl):
+    """The oracle, as it stands, timed on the host cores.  A step is a bounded sample of the
+    workload: Local on `nl` layers and Full on `nf` layers of the stack, extrapolated to all
+    layers and combined at the realised recall rate of the same forced-flag schedule."""
+    from oracle import oda_oracle as orc
+    from paper_2609_20734_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = orc.host_threads()
+    nl, nf = 1, 1
+    table, nb = wl.tables()
+    lay = orc.hnd_layout(nb, wl.Hkv, 16, wl.D)
+    kk, vk = synth.stream_key(wl.seed, synth.STREAM_K), synth.stream_key(wl.seed, synth.STREAM_V)
+    idx = np.arange(0, nl * lay.layer_stride, dtype=np.uint64)
+    k, v = synth.gauss_bf16(kk, idx), synth.gauss_bf16(vk, idx)
+    flags = [wl.override_flags(s) for s in range(args.warmup + args.steps)]
+    realised = float(np.mean([f.mean() for f in flags[args.warmup:]]))
+
+    def one(step, mode, n):
+        q = wl.q_host(step)[:n]
+        t0 = time.perf_counter()
+        orc.attention(mode, q, k, v, table, np.asarray(wl.seq_lens0) + step, num_kv_heads=wl.Hkv,
+                      block_size=16, layout=lay, layer_window=wl.windows[:n], layer_sinks=wl.sinks[:n],
+                      nthreads=cores)
+        return time.perf_counter() - t0
+
+    for s in range(args.warmup):
+        one(s, "local", nl)
+    tl, tf = [], []
+    for s in range(args.steps):
+        tl.append(one(args.warmup + s, "local", nl) * wl.L / nl)
+        if s < max(1, min(args.steps, 3)):
+            tf.append(one(args.warmup + s, "full", nf) * sum(wl.gated) / nf)
+    step_s = float(np.mean(tl) + realised * np.mean(tf))
+    val = wl.B / step_s
+    sample = (f"per step: Local on {nl} of {wl.L} layers (every step) and Full on {nf} of {wl.L} layers "
+              f"({len(tf)} steps), scaled to all layers and combined at the realised recall rate {realised:.3f}")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": config_dict(wl, args, realised),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_dict(wl, args, realised):
+    return {"workload": f"{wl.name}: L={wl.L} B={wl.B} Hq={wl.Hq} Hkv={wl.Hkv} D={wl.D} "
+                        f"context={int(np.max(wl.seq_lens0))} window={wl.windows[0]} sinks={wl.sinks[0]} block=16 "
+                        f"bf16 KV ~N(0,1), {wl.schedule} flags",
+            "recall_rate_target": wl.recall_rate, "recall_rate_realised": realised,
+            "global_batch": wl.B * args.gpus, "parallelism": f"dp{args.gpus} (requests sharded, no collective)",
+            "l2": "flushed between timed steps (256 MiB write, untimed)",
+            "launch": "one CUDA graph replay per step"}
+
+
+def main():
+    args = parse()
+    from paper_2609_20734_b200 import workloads
+
+    ov = {"recall_rate": args.recall_rate}
+    wl = workloads.make(args.config, **ov)
+    if args.sinks is not None:
+        wl.sinks = [args.sinks if g else s for g, s in zip(wl.gated, wl.sinks)]
+    wl.steps = args.steps + args.warmup + 1
+    if args.impl == "reference":
+        reference_arm(args, wl)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and world == 1:
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", "29531", os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_20734_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    # requests are independent: every rank serves its own batch of the same shape (weak scaling)
+    wl.seed = wl.seed + rank
+
+    st = workloads.materialize(wl)
+    ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks, variant=args.variant))
+    B, L = wl.B, wl.L
+    shape = (L, B, wl.Hq, wl.D)
+    nsteps = args.warmup + args.steps
+    qs = [workloads.q_device(wl, s) for s in range(nsteps)]
+    flags_h = [wl.override_flags(s) for s in range(nsteps)]
+    ovs = [torch.from_numpy(f).cuda() for f in flags_h]
+    feats = [None if wl.feat_host(s) is None else torch.from_numpy(wl.feat_host(s)).cuda() for s in range(nsteps)]
+    q_s = torch.empty_like(qs[0])
+    ov_s = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    fe_s = None if feats[0] is None else torch.empty_like(feats[0])
+    out = torch.zeros(shape, device="cuda")
+    lse = torch.zeros(shape[:3], device="cuda")
+    scores = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    counters = torch.zeros((B, 2), dtype=torch.int32, device="cuda")
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    seq0 = torch.from_numpy(np.asarray(wl.seq_lens0, dtype=np.int32)).cuda()
+
+    step_args = ctx.step_args(B, q_s, st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, scores,
+                              flags, feat_ext=fe_s, head=st.head, threshold=wl.threshold,
+                              override_flags=ov_s, lse=lse, counters=counters, advance_seq_lens=True)
+    # capture one step; every replay reads lengths and flags on the device
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    before = ctx.launch_count
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            ctx.step(step_args, stream=side.cuda_stream)
+    launches_per_step = ctx.launch_count - before
+    torch.cuda.synchronize()
+
+    def set_inputs(s):
+        q_s.copy_(qs[s])
+        ov_s.copy_(ovs[s])
+        if fe_s is not None:
+            fe_s.copy_(feats[s])
+
+    def run_steps(first, count, timed):
+        evs = []
+        for s in range(first, first + count):
+            set_inputs(s)
+            flush.fill_(s & 0xFF)  # evict the previous step's KV from L2 (untimed)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs] if timed else None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    st.seq_lens.copy_(seq0)
+    run_steps(0, args.warmup, False)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    t_wall = time.perf_counter()
+    ms = run_steps(args.warmup, args.steps, True)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    total_ms = float(np.sum(ms))
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    realised = float(np.mean([f.mean() for f in flags_h[args.warmup:]]))
+    assert ctx.read_device_status() == 0, "device status word set during the timed region"
+    assert int(counters[0, 0].item()) == nsteps, "the recall kernel did not run once per step"
+    value = world * B * args.steps / (total_ms * 1e-3)
+
+    # per-step algorithmic bytes (exact tokens of Eq. 1, not rounded to pages)
+    seq_steps = [np.asarray(wl.seq_lens0) + s for s in range(args.warmup, nsteps)]
+    ab = [wl.algorithmic_bytes(sl, f) for sl, f in zip(seq_steps, flags_h[args.warmup:])]
+    step_bytes = float(np.mean([a + b for a, b in ab]))
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
+            "data": "synthetic", "config": config_dict(wl, args, realised),
+            "gpu_launches": launches_per_step * args.steps,
+            "step_gbs": step_bytes / (total_ms / args.steps * 1e-3) / 1e9,
+            "variant": {1: "simt", 2: "tma_mma"}.get(ctx.variant, str(ctx.variant)),
+            "attention_grid": ctx.attention_grid,
+            "wall_s_timed_region_incl_flush": t_wall}
+
+    if rank == 0:
+        peak, peak_src = peaks()
+        # ---- the two attention kernels alone, events around each launch, L2 flushed ----
+        reps = args.kernel_reps
+        ones = torch.ones(B, dtype=torch.uint8, device="cuda")
+        st.seq_lens.copy_(seq0)
+        kt = {"local": [], "full": []}
+        for r in range(reps + 2):
+            for name in ("local", "full"):
+                flush.fill_(r)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                if name == "local":
+                    ctx.local_decode(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, lse)
+                else:
+                    ctx.full_decode_gated(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table,
+                                          st.seq_lens, ones, out, lse)
+                e1.record()
+                torch.cuda.synchronize()
+                if r >= 2:
+                    kt[name].append(e0.elapsed_time(e1))
+        lb, fb = wl.algorithmic_bytes(np.asarray(wl.seq_lens0), np.ones(B))
+        kernels = {}
+        for name, nbytes in (("local", lb), ("full", fb)):
+            t = float(np.mean(kt[name])) * 1e-3
+            kernels[name] = {"bound": "hbm", "achieved": nbytes / t / 1e9, "peak": peak, "unit": "GB/s",
+                             "frac": nbytes / t / 1e9 / peak, "traffic": None,
+                             "algorithmic_bytes": nbytes, "us": t * 1e6, "frac_of_8000_nominal": nbytes / t / 8e12}
+        dominant = "full" if realised * kernels["full"]["us"] > kernels["local"]["us"] else "local"
+        line["roofline"] = dict(kernels[dominant], kernel=f"splitkv ({dominant} pass)", peak_source=peak_src)
+        line["roofline_other"] = dict(kernels["local" if dominant == "full" else "full"],
+                                      kernel=f"splitkv ({'local' if dominant == 'full' else 'full'} pass)")
+        traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(traffic_path):  # DRAM bytes per launch from the committed ncu summary
+            tr = json.load(open(traffic_path))
+            line["roofline"]["traffic"] = tr.get(dominant)
+            line["roofline_other"]["traffic"] = tr.get("local" if dominant == "full" else "full")
+
+        # ---- recall-rate sweep: step time must be affine in the realised rate ----
+        if not args.no_sweep:
+            sweep = []
+            n_sw = min(args.steps, 32)
+            for rate in SWEEP_RATES:
+                wl_r = workloads.make(args.config, recall_rate=rate)
+                fl = [wl_r.override_flags(s) for s in range(n_sw)]
+                st.seq_lens.copy_(seq0)
+                tms = []
+                for s in range(n_sw):
+                    q_s.copy_(qs[s % nsteps])
+                    ov_s.copy_(torch.from_numpy(fl[s]).cuda())
+                    flush.fill_(s & 0xFF)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    graph.replay()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    tms.append(e0.elapsed_time(e1))
+                rr = float(np.mean([f.mean() for f in fl]))
+                bts = np.mean([sum(wl.algorithmic_bytes(np.asarray(wl.seq_lens0) + s, fl[s])) for s in range(n_sw)])
+                sweep.append({"rate": rate, "realised": rr, "ms_per_step": float(np.mean(tms)),
+                              "tokens_per_s": B / (float(np.mean(tms)) * 1e-3),
+                              "gbs": float(bts) / (float(np.mean(tms)) * 1e-3) / 1e9})
+            x = np.array([s["realised"] for s in sweep])
+            y = np.array([s["ms_per_step"] for s in sweep])
+            A = np.vstack([x, np.ones_like(x)]).T
+            coef, res, *_ = np.linalg.lstsq(A, y, rcond=None)
+            ss_tot = float(((y - y.mean()) ** 2).sum())
+            r2 = 1.0 - float(((A @ coef - y) ** 2).sum()) / ss_tot if ss_tot > 0 else 1.0
+            line["sweep"] = sweep
+            line["affine_fit"] = {"slope_ms": float(coef[0]), "intercept_ms": float(coef[1]), "r2": r2}
+
+        # ---- end to end: host buffers through oda_step_host, copies inside the timed region ----
+        if not args.no_e2e:
+            q_hs = [q.cpu().pin_memory() for q in qs]
+            ov_hs = [torch.from_numpy(f).pin_memory() for f in flags_h]
+            fe_hs = [None if f is None else f.cpu().pin_memory() for f in feats]
+            out_h = torch.zeros(shape).pin_memory()
+            sc_h = torch.zeros(B).pin_memory()
+            fl_h = torch.zeros(B, dtype=torch.uint8).pin_memory()
+            st.seq_lens.copy_(seq0)
+            torch.cuda.synchronize()
+            tot, up, down = 0.0, 0, 0
+            for s in range(nsteps):
+                a = ctx.step_args(B, q_hs[s], st.k_cache, st.v_cache, st.block_table, st.seq_lens, out_h,
+                                  sc_h, fl_h, feat_ext=fe_hs[s], head=st.head, threshold=wl.threshold,
+                                  override_flags=ov_hs[s], counters=counters, advance_seq_lens=True)
+                flush.fill_(s & 0xFF)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                up, down = ctx.step_host(a)
+                dt = time.perf_counter() - t0
+                if s >= args.warmup:
+                    tot += dt
+            line["e2e"] = {"value": world * B * args.steps / tot, "unit": UNIT, "h2d_bytes_per_step": up,
+                           "d2h_bytes_per_step": down, "ms_per_step": tot / args.steps * 1e3,
+                           "note": "oda_step_host: pinned host q/flags in, out/scores/flags back, stream "
+                                   "sync inside; KV cache, block table and head weights are device-resident state"}
+        line["clocks"] = sampler.stop()
+
+        # ---- the oracle on the host cores, bounded sample ----
+        if not args.no_cpu_baseline and world == 1:
+            import contextlib
+            import io
+
+            buf = io.StringIO()
+            ref_args = argparse.Namespace(**vars(args))
+            ref_args.steps, ref_args.warmup = 3, 1
+            with contextlib.redirect_stdout(buf):
+                reference_arm(ref_args, workloads.make(args.config, recall_rate=args.recall_rate))
+            line["cpu_baseline"] = json.loads(buf.getvalue())["cpu_baseline"]
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
