@@ -44,6 +44,14 @@ struct oda_ctx {
     int head_grid = 1;
     WsLayout lay{};
     char* ws = nullptr;
+    // TMA variant: tensor maps of the two caches, re-encoded when a base pointer changes
+    alignas(64) unsigned char kmap[128];
+    alignas(64) unsigned char vmap[128];
+    const void* kmap_base = nullptr;
+    const void* vmap_base = nullptr;
+    int phys_layers = 1;
+    int blocks_per_layer = 0;
+    int64_t blocks_bound = 1;
     int64_t launches = 0;
     std::string err;
 };
@@ -151,7 +159,24 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
         if (n && (mode == 0 || c->cls_gated[i])) any = true;
     }
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
-    cudaError_t e = launch_splitkv_simt(p, f.head_dim, c->group, c->grid, st);
+    cudaError_t e;
+    if (c->variant == ODA_VARIANT_TMA_MMA) {
+        if (c->kmap_base != k) {
+            if (!encode_kv_map(c->kmap, k, f.head_dim, f.num_kv_heads, f.kv_token_stride, f.kv_head_stride,
+                               f.kv_block_stride, c->blocks_bound))
+                return fail(c, ODA_ERR_CUDA, "cuTensorMapEncodeTiled failed for k_cache");
+            c->kmap_base = k;
+        }
+        if (c->vmap_base != v) {
+            if (!encode_kv_map(c->vmap, v, f.head_dim, f.num_kv_heads, f.kv_token_stride, f.kv_head_stride,
+                               f.kv_block_stride, c->blocks_bound))
+                return fail(c, ODA_ERR_CUDA, "cuTensorMapEncodeTiled failed for v_cache");
+            c->vmap_base = v;
+        }
+        e = launch_splitkv_tma(p, c->kmap, c->vmap, c->blocks_per_layer, f.head_dim, c->group, c->grid, st);
+    } else {
+        e = launch_splitkv_simt(p, f.head_dim, c->group, c->grid, st);
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "attention kernel launch");
     c->launches += 1;
     return ODA_OK;
@@ -245,14 +270,26 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
     c->cfg.layer_sinks = nullptr;
     c->cfg.layer_gated = nullptr;
     c->cfg.layer_kv_index = nullptr;
-    (void)max_kv_index;
-
-    c->variant = ODA_VARIANT_SIMT;
+    c->phys_layers = max_kv_index + 1;
+    const bool tma_ok = tma_variant_supported(cfg->head_dim, cfg->kv_layer_stride, cfg->kv_block_stride, c->phys_layers);
+    if (c->phys_layers > 1) {
+        c->blocks_per_layer = tma_ok ? (int)(cfg->kv_layer_stride / cfg->kv_block_stride) : 0;
+        c->blocks_bound = (int64_t)c->phys_layers * c->blocks_per_layer;
+    } else {
+        c->blocks_per_layer = 0;
+        c->blocks_bound = (int64_t)1 << 30;
+    }
+    if (cfg->variant == ODA_VARIANT_TMA_MMA && !tma_ok) {
+        delete c;
+        return ODA_ERR_UNSUPPORTED;  // layer stride is not a whole number of blocks
+    }
+    c->variant = cfg->variant == ODA_VARIANT_AUTO ? (tma_ok ? ODA_VARIANT_TMA_MMA : ODA_VARIANT_SIMT) : cfg->variant;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
         c->num_sms = sms;
-        int occ = occupancy_splitkv_simt(cfg->head_dim, group);
+        int occ = c->variant == ODA_VARIANT_TMA_MMA ? occupancy_splitkv_tma(cfg->head_dim, group)
+                                                    : occupancy_splitkv_simt(cfg->head_dim, group);
         c->grid = sms * (occ > 0 ? occ : 1);
     } else {
         (void)cudaGetLastError();

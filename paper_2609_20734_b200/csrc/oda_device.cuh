@@ -232,9 +232,53 @@ __device__ __forceinline__ void store_out(const AttnParams& p, int layer, int b,
         reinterpret_cast<float*>(p.out)[idx] = val;
 }
 
-// cta_part: [G][D+2] in shared memory holding this CTA's (m, l, o[D]) for the item.
-// If the unit has one chunk, normalise and store.  Otherwise publish the partial, take a
-// ticket, and let the CTA that arrives last merge all chunks in chunk order (deterministic).
+// Split merge.  A unit (layer, request, kv head) with one chunk is normalised and stored by the
+// CTA that computed it.  Otherwise each CTA publishes its partial [G][D+2] = (m, l, o[D]) in
+// its slot, takes a ticket, and the CTA that arrives last (no waiting, one atomic) merges all
+// chunks in chunk order, so the bits do not depend on scheduling.
+
+__device__ __forceinline__ float* partial_slot(const AttnParams& p, const Item& it, int G, int W)
+{
+    return p.partials + (size_t)(it.slot_base + it.chunk) * (G * W);
+}
+
+// one thread calls this after the CTA's partial is visible (threadfence + barrier before)
+__device__ __forceinline__ int take_ticket(const AttnParams& p, const Item& it)
+{
+    int* tk = p.tickets + ((size_t)it.layer * p.max_batch + it.b) * p.num_kv_heads + it.g;
+    int old = atomicAdd(tk, 1);
+    int last = (old == it.nchunks - 1);
+    if (last) *tk = 0;  // ready for the next launch
+    return last;
+}
+
+template <int D, int G>
+__device__ inline void merge_chunks(const AttnParams& p, const Item& it, int tid, int nth)
+{
+    constexpr int W = D + 2;
+    const float kLn2 = 0.6931471805599453f;
+    const float* base = p.partials + (size_t)it.slot_base * (G * W);
+    for (int e = tid; e < G * D; e += nth) {
+        int h = e / D, d = e - h * D;
+        float M = -INFINITY;
+        for (int c = 0; c < it.nchunks; ++c) M = fmaxf(M, __ldcg(base + (size_t)c * (G * W) + h * W));
+        float l = 0.f, o = 0.f;
+        for (int c = 0; c < it.nchunks; ++c) {
+            const float* pc = base + (size_t)c * (G * W) + h * W;
+            float mc = __ldcg(pc);
+            float sc = (mc == -INFINITY) ? 0.f : ex2(mc - M);
+            l += __ldcg(pc + 1) * sc;
+            o += __ldcg(pc + 2 + d) * sc;
+        }
+        store_out<D>(p, it.layer, it.b, it.g * G + h, d, o / l);
+        if (d == 0 && p.lse)
+            p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + it.g * G + h] =
+                (M + log2f(l)) * kLn2;
+    }
+}
+
+// cta_part: [G][D+2] in shared memory holding this CTA's (m, l, o[D]) for the item; called by
+// every thread of the CTA.
 template <int D, int G>
 __device__ inline void finish_item(const AttnParams& p, const Item& it, const float* cta_part,
                                    int* s_is_last)
@@ -255,38 +299,15 @@ __device__ inline void finish_item(const AttnParams& p, const Item& it, const fl
         }
         return;
     }
-    float* slot = p.partials + (size_t)(it.slot_base + it.chunk) * (G * W);
+    float* slot = partial_slot(p, it, G, W);
     for (int e = tid; e < G * W; e += nth) __stcg(slot + e, cta_part[e]);
     __threadfence();
     __syncthreads();
-    if (tid == 0) {
-        int* tk = p.tickets + ((size_t)it.layer * p.max_batch + it.b) * p.num_kv_heads + it.g;
-        int old = atomicAdd(tk, 1);
-        int last = (old == it.nchunks - 1);
-        if (last) *tk = 0;  // ready for the next launch
-        *s_is_last = last;
-    }
+    if (tid == 0) *s_is_last = take_ticket(p, it);
     __syncthreads();
     if (!*s_is_last) return;
     __threadfence();
-    const float* base = p.partials + (size_t)it.slot_base * (G * W);
-    for (int e = tid; e < G * D; e += nth) {
-        int h = e / D, d = e - h * D;
-        float M = -INFINITY;
-        for (int c = 0; c < it.nchunks; ++c) M = fmaxf(M, __ldcg(base + (size_t)c * (G * W) + h * W));
-        float l = 0.f, o = 0.f;
-        for (int c = 0; c < it.nchunks; ++c) {
-            const float* pc = base + (size_t)c * (G * W) + h * W;
-            float mc = __ldcg(pc);
-            float sc = (mc == -INFINITY) ? 0.f : ex2(mc - M);
-            l += __ldcg(pc + 1) * sc;
-            o += __ldcg(pc + 2 + d) * sc;
-        }
-        store_out<D>(p, it.layer, it.b, it.g * G + h, d, o / l);
-        if (d == 0 && p.lse)
-            p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + it.g * G + h] =
-                (M + log2f(l)) * kLn2;
-    }
+    merge_chunks<D, G>(p, it, tid, nth);
 }
 
 }  // namespace oda

@@ -10,6 +10,14 @@ struct AttnParams;
 cudaError_t launch_splitkv_simt(const AttnParams& p, int head_dim, int group, int grid, cudaStream_t st);
 int occupancy_splitkv_simt(int head_dim, int group);
 
+// TMA + tensor-core variant.  kmap / vmap point at 128-byte CUtensorMap objects (host memory).
+bool tma_variant_supported(int head_dim, int64_t layer_stride, int64_t block_stride, int num_layers_phys);
+bool encode_kv_map(void* out_map, const void* base, int head_dim, int num_kv_heads, int64_t token_stride,
+                   int64_t head_stride, int64_t block_stride, int64_t num_blocks_bound);
+cudaError_t launch_splitkv_tma(const AttnParams& p, const void* kmap, const void* vmap, int blocks_per_layer,
+                               int head_dim, int group, int grid, cudaStream_t st);
+int occupancy_splitkv_tma(int head_dim, int group);
+
 struct HeadParams {
     const float* feat_ext;      // [B, d_ext] or nullptr
     const void* attn_out;       // [B, d_attn] fp32 or bf16, or nullptr

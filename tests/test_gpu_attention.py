@@ -10,7 +10,7 @@ from tests.helpers import make_problem, oracle_attention
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [binding.VARIANT_SIMT]
+VARIANTS = [binding.VARIANT_SIMT, binding.VARIANT_TMA_MMA]
 RAGGED = [1, 15, 16, 17, 300, 1000, 2053]
 
 
