@@ -46,6 +46,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--kernel-reps", type=int, default=10)
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="time only the Local and the all-flagged Full attention launches (for ncu captures)")
     return ap.parse_args()
 
 
@@ -254,6 +256,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.kernels_only:
+        args.steps, args.warmup, args.no_sweep, args.no_e2e, args.no_cpu_baseline = 1, 1, True, True, True
     st.seq_lens.copy_(seq0)
     run_steps(0, args.warmup, False)
     sampler = ClockSampler(local_rank)
@@ -271,7 +275,7 @@ def main():
         total_ms = float(t.item())
     realised = float(np.mean([f.mean() for f in flags_h[args.warmup:]]))
     assert ctx.read_device_status() == 0, "device status word set during the timed region"
-    assert int(counters[0, 0].item()) == nsteps, "the recall kernel did not run once per step"
+    assert int(counters[0, 0].item()) == args.warmup + args.steps, "the recall kernel did not run once per step"
     value = world * B * args.steps / (total_ms * 1e-3)
 
     # per-step algorithmic bytes (exact tokens of Eq. 1, not rounded to pages)

@@ -71,7 +71,7 @@ typedef struct {
     int32_t num_kv_heads;
     int32_t head_dim;           /* 64 or 128 */
     int32_t block_size;         /* tokens per KV block: 16 */
-    int32_t max_batch;          /* 1..256 */
+    int32_t max_batch;          /* 1..128 */
     int32_t max_blocks_per_seq; /* row length of block_table */
     int32_t out_dtype;          /* 0 = fp32, 1 = bf16 */
     float sm_scale;             /* logit scale; 0 => 1/sqrt(head_dim) */

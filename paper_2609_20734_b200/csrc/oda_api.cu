@@ -38,8 +38,7 @@ struct oda_ctx {
     int num_sms = 148;
     int variant = ODA_VARIANT_SIMT;
     int grid = 148;
-    int items_per_cta = 4;
-    int min_chunk_pages = 4;
+    int min_span_pages = 8;
     int max_items = 0;
     int head_grid = 1;
     WsLayout lay{};
@@ -144,8 +143,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     p.out_bf16 = f.out_dtype;
     p.mode = mode;
     p.ncls = c->ncls;
-    p.items_per_cta = c->items_per_cta;
-    p.min_chunk_pages = c->min_chunk_pages;
+    p.min_span_pages = c->min_span_pages;
     p.max_items = c->max_items;
     p.scale_log2e = c->scale * 1.4426950408889634f;
     bool any = false;
@@ -244,7 +242,7 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         li.sinks = cfg->layer_sinks[l];
         li.gated = cfg->layer_gated[l] ? 1 : 0;
         li.kv_index = cfg->layer_kv_index ? cfg->layer_kv_index[l] : l;
-        if (li.window < 1 || li.sinks < 0 || li.kv_index < 0) {
+        if (li.window < 1 || li.sinks < 0 || li.kv_index < 0 || li.kv_index > 65535) {
             delete c;
             return ODA_ERR_INVALID_ARG;
         }
@@ -296,7 +294,7 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         c->num_sms = 148;  // no device visible: sizes follow a B200 so that host-only checks still work
         c->grid = 148 * 2;
     }
-    c->max_items = c->grid * c->items_per_cta + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
+    c->max_items = c->grid + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
     c->head_grid = cfg->head_d_hidden > 0 ? recall_head_grid(cfg->head_d_hidden) : 1;
     compute_layout(c);
     *out_ctx = c;

@@ -9,7 +9,7 @@
 namespace oda {
 
 constexpr int kPage = 16;          // tokens per KV block
-constexpr int kMaxBatch = 256;
+constexpr int kMaxBatch = 128;
 constexpr int kMaxLayers = 256;
 constexpr int kMaxClasses = 4;     // distinct (window, sinks, gated) triples in one stack
 
@@ -39,19 +39,29 @@ struct AttnParams {
     int32_t num_q_heads, num_kv_heads, max_blocks_per_seq, out_bf16;
     int32_t mode;          // 0 = Local (Eq. 1 S^L), 1 = gated Full (S^F)
     int32_t ncls;
-    int32_t items_per_cta; // target items per CTA used to size chunks
-    int32_t min_chunk_pages;
+    int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)
     int32_t cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
     int32_t cls_layers_in_call[kMaxClasses];
 };
 
+// Work decomposition.  A unit is one (layer, request, kv head); it owns np pages of KV (the
+// pages of its Eq. 1 window segment, or of the whole history in Full mode).  All units are laid
+// end to end, layer-major then request then kv head, on one axis of P pages; the axis is cut into
+// nseg <= gridDim.x spans of equal length (+-1 page) and CTA j streams span j.  A span that
+// crosses a unit boundary yields one item per unit it touches, so every CTA reads the same number
+// of bytes whatever the mix of lengths and flags is, and the number of partials a unit has is the
+// number of spans it touches.
 struct Plan {  // shared memory, one per CTA
-    int32_t offsets[kMaxClasses][kMaxBatch + 1];  // exclusive prefix of chunks per request
-    int32_t layer_base[kMaxLayers + 1];           // first item id of each layer in the call
-    int32_t chunk_pages;
-    int32_t total_items;
+    int32_t pb[kMaxClasses][kMaxBatch + 1];  // exclusive prefix over requests of pages per kv head
+    int32_t lb[kMaxLayers + 1];              // first axis page of each layer of the call
+    int32_t seq[kMaxBatch];                  // seq_lens, clamped to the table capacity
+    uint16_t kv_index[kMaxLayers];
+    uint8_t cls[kMaxLayers];
+    int32_t total_pages;
+    int32_t nseg;
+    int32_t pad;  // keeps sizeof(Plan) a multiple of 8
 };
 
 struct Item {
@@ -59,10 +69,11 @@ struct Item {
     int32_t chunk, nchunks;     // this split and how many the unit has
     int32_t slot_base;          // partial slot of the unit's chunk 0
     int32_t t;                  // seq_len
-    int32_t win_pg0, win_pg1;   // logical pages of this chunk
+    int32_t win_pg0, win_pg1;   // logical pages of this item
     int32_t win_lo, win_hi;     // valid positions of the window/full segment: [lo, hi)
     int32_t sink_pg1;           // sink pages [0, sink_pg1) (0 = none in this item)
     int32_t sink_hi;            // valid sink positions [0, sink_hi)
+    int32_t kv_layer;           // cache layer slice holding this layer's K/V
 };
 
 // Eq. 1 in 0-based form.  Local: sinks [0, min(s,t)), window [max(0,t-w), t); when they touch
@@ -101,116 +112,128 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
 {
     const int tid = threadIdx.x, nth = blockDim.x;
     const int B = p.batch;
-    for (int idx = tid; idx < p.ncls * B; idx += nth) {
-        int c = idx / B, b = idx - c * B;
+    const int nl = p.layer_end - p.layer_begin;
+    for (int b = tid; b < B; b += nth) {
         int t = p.seq_lens[b];
-        int np = 0;
-        bool active = p.cls_layers_in_call[c] > 0 &&
-                      (p.mode == 0 || (p.cls_gated[c] && p.flags[b] != 0));
-        if (active) {
-            if (t < 1) {
-                atomicOr(p.status, kStatusBadSeqLen);
-            } else {
-                if (t > p.max_blocks_per_seq * kPage) {
-                    t = p.max_blocks_per_seq * kPage;
-                    atomicOr(p.status, kStatusBadSeqLen);
-                }
-                Ranges r = eq1_ranges(p.mode, t, p.cls_window[c], p.cls_sinks[c]);
-                np = r.pg1 - r.pg0;
-            }
+        if (t > p.max_blocks_per_seq * kPage) {
+            t = p.max_blocks_per_seq * kPage;
+            atomicOr(p.status, kStatusBadSeqLen);
         }
-        pl.offsets[c][b + 1] = np;
+        pl.seq[b] = t;
+    }
+    for (int i = tid; i < nl; i += nth) {
+        const LayerInfo li = p.layers[p.layer_begin + i];
+        pl.cls[i] = (uint8_t)li.cls;
+        pl.kv_index[i] = (uint16_t)li.kv_index;
     }
     __syncthreads();
-    if (tid < 32) {
-        long long tot = 0;
-        for (int c = 0; c < p.ncls; ++c) {
-            long long sc = 0;
-            for (int b = tid; b < B; b += 32) sc += pl.offsets[c][b + 1];
-            tot += sc * p.cls_layers_in_call[c];
-        }
-        for (int o = 16; o; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
-        tot *= p.num_kv_heads;
-        long long denom = (long long)gridDim.x * p.items_per_cta;
-        long long cp = (tot + denom - 1) / denom;
-        if (cp < p.min_chunk_pages) cp = p.min_chunk_pages;
-        if (tid == 0) pl.chunk_pages = (int)cp;
-    }
-    __syncthreads();
-    const int cp = pl.chunk_pages;
     const int warp = tid >> 5, lane = tid & 31, nwarps = nth >> 5;
     for (int c = warp; c < p.ncls; c += nwarps) {  // one warp scans one class
         int carry = 0;
         for (int b0 = 0; b0 < B; b0 += 32) {
-            int b = b0 + lane;
-            int np = b < B ? pl.offsets[c][b + 1] : 0;
-            int n = (np + cp - 1) / cp;
-            int x = n;
+            const int b = b0 + lane;
+            int np = 0;
+            if (b < B && p.cls_layers_in_call[c] > 0 && (p.mode == 0 || (p.cls_gated[c] && p.flags[b] != 0))) {
+                const int t = pl.seq[b];
+                if (t < 1) {
+                    atomicOr(p.status, kStatusBadSeqLen);
+                } else {
+                    Ranges r = eq1_ranges(p.mode, t, p.cls_window[c], p.cls_sinks[c]);
+                    np = r.pg1 - r.pg0;
+                }
+            }
+            int x = np;
             for (int o = 1; o < 32; o <<= 1) {
                 int y = __shfl_up_sync(0xffffffffu, x, o);
                 if (lane >= o) x += y;
             }
-            if (b < B) pl.offsets[c][b + 1] = carry + x;
+            if (b < B) pl.pb[c][b + 1] = carry + x;
             carry += __shfl_sync(0xffffffffu, x, 31);
         }
-        if (lane == 0) pl.offsets[c][0] = 0;
+        if (lane == 0) pl.pb[c][0] = 0;
     }
     __syncthreads();
-    if (tid == 0) {
-        int base = 0;
-        for (int l = p.layer_begin; l < p.layer_end; ++l) {
-            pl.layer_base[l - p.layer_begin] = base;
-            base += p.num_kv_heads * pl.offsets[p.layers[l].cls][B];
+    if (tid < 32) {  // exclusive scan over the layers of the call
+        long long carry = 0;
+        for (int i0 = 0; i0 < nl; i0 += 32) {
+            const int i = i0 + lane;
+            long long x = i < nl ? (long long)p.num_kv_heads * pl.pb[pl.cls[i]][B] : 0;
+            const long long own = x;
+            for (int o = 1; o < 32; o <<= 1) {
+                long long y = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += y;
+            }
+            if (i < nl) pl.lb[i] = (int32_t)(carry + x - own);
+            carry += __shfl_sync(0xffffffffu, x, 31);
         }
-        pl.layer_base[p.layer_end - p.layer_begin] = base;
-        if (base > p.max_items) {
-            atomicOr(p.status, kStatusItemOverflow);
-            base = 0;  // refuse to run rather than overrun the partial buffer
+        if (lane == 0) {
+            if (carry > 0x7fffffffll) {  // beyond the 32-bit page axis: refuse rather than wrap
+                atomicOr(p.status, kStatusItemOverflow);
+                carry = 0;
+            }
+            pl.lb[nl] = (int32_t)carry;
+            pl.total_pages = (int32_t)carry;
+            long long n = (carry + p.min_span_pages - 1) / p.min_span_pages;
+            if (n > (long long)gridDim.x) n = gridDim.x;
+            pl.nseg = (int32_t)n;
         }
-        pl.total_items = base;
     }
     __syncthreads();
 }
 
-// item id -> (layer, request, kv head, chunk) and the token ranges it covers
-__device__ inline Item decode_item(const AttnParams& p, const Plan& pl, int id)
+__device__ __forceinline__ int span_begin(const Plan& pl, int j)
 {
-    Item it;
+    return (int)(((long long)j * pl.total_pages) / pl.nseg);
+}
+// the span that contains axis page x
+__device__ __forceinline__ int span_of(const Plan& pl, int x)
+{
+    return (int)((((long long)x + 1) * pl.nseg - 1) / pl.total_pages);
+}
+
+// The item of span j that starts at axis page x (span_begin(j) <= x < x_end = span_begin(j+1)).
+// Returns the number of axis pages it covers (>= 1).
+__device__ inline int decode_item(const AttnParams& p, const Plan& pl, int j, int x, int x_end, Item& it)
+{
     const int nl = p.layer_end - p.layer_begin;
-    int lo = 0, hi = nl;  // last layer with layer_base <= id
+    int lo = 0, hi = nl;  // last layer with lb <= x
     while (hi - lo > 1) {
         int mid = (lo + hi) >> 1;
-        if (pl.layer_base[mid] <= id) lo = mid; else hi = mid;
+        if (pl.lb[mid] <= x) lo = mid; else hi = mid;
     }
-    it.layer = p.layer_begin + lo;
-    const LayerInfo li = p.layers[it.layer];
-    const int c = li.cls;
-    const int totc = pl.offsets[c][p.batch];
-    int rem = id - pl.layer_base[lo];
-    it.g = rem / totc;
-    rem -= it.g * totc;
-    int blo = 0, bhi = p.batch;  // last b with offsets[b] <= rem
+    const int c = pl.cls[lo];
+    const int H = p.num_kv_heads;
+    const int r = x - pl.lb[lo];
+    int blo = 0, bhi = p.batch;  // last request with H * pb <= r
     while (bhi - blo > 1) {
         int mid = (blo + bhi) >> 1;
-        if (pl.offsets[c][mid] <= rem) blo = mid; else bhi = mid;
+        if (H * pl.pb[c][mid] <= r) blo = mid; else bhi = mid;
     }
+    const int np = pl.pb[c][blo + 1] - pl.pb[c][blo];
+    const int r2 = r - H * pl.pb[c][blo];
+    const int g = r2 / np;
+    const int off = r2 - g * np;
+    const int unit0 = x - off;                       // axis page where the unit starts
+    const int take = min(np - off, x_end - x);
+    const int j0 = span_of(pl, unit0), j1 = span_of(pl, unit0 + np - 1);
+    it.layer = p.layer_begin + lo;
     it.b = blo;
-    it.chunk = rem - pl.offsets[c][blo];
-    it.nchunks = pl.offsets[c][blo + 1] - pl.offsets[c][blo];
-    it.slot_base = id - it.chunk;
-    int t = p.seq_lens[it.b];
-    if (t > p.max_blocks_per_seq * kPage) t = p.max_blocks_per_seq * kPage;
+    it.g = g;
+    it.chunk = j - j0;
+    it.nchunks = j1 - j0 + 1;
+    // one slot per (span, unit) pair met along the axis: span index + unit index is unique
+    it.slot_base = j0 + (lo * p.batch + blo) * H + g;
+    it.kv_layer = pl.kv_index[lo];
+    const int t = pl.seq[blo];
     it.t = t;
-    Ranges r = eq1_ranges(p.mode, t, li.window, li.sinks);
-    const int np = r.pg1 - r.pg0;
-    const int per = (np + it.nchunks - 1) / it.nchunks;
-    it.win_pg0 = r.pg0 + it.chunk * per;
-    it.win_pg1 = min(it.win_pg0 + per, r.pg1);
-    it.win_lo = r.lo;
-    it.win_hi = r.hi;
-    it.sink_hi = (it.chunk == 0) ? r.sink_hi : 0;
+    Ranges rg = eq1_ranges(p.mode, t, p.cls_window[c], p.cls_sinks[c]);
+    it.win_pg0 = rg.pg0 + off;
+    it.win_pg1 = it.win_pg0 + take;
+    it.win_lo = rg.lo;
+    it.win_hi = rg.hi;
+    it.sink_hi = (off == 0) ? rg.sink_hi : 0;
     it.sink_pg1 = (it.sink_hi + kPage - 1) / kPage;
-    return it;
+    return take;
 }
 
 __device__ __forceinline__ float ex2(float x)

@@ -51,9 +51,12 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
     const int sub = lane / C::kLPR;               // which row of a warp-wide load this lane reads
     const int dofs = (lane % C::kLPR) * 8;        // this lane's 8 head-dim elements
 
-    for (int id = blockIdx.x; id < plan.total_items; id += gridDim.x) {
-        const Item it = decode_item(p, plan, id);
-        const LayerInfo li = p.layers[it.layer];
+    const int span = blockIdx.x;
+    if (span >= plan.nseg) return;
+    const int x_end = span_begin(plan, span + 1);
+    for (int x = span_begin(plan, span); x < x_end;) {
+        Item it;
+        x += decode_item(p, plan, span, x, x_end, it);
         // q for the G heads of this kv head, pre-multiplied by scale * log2(e)
         float qf[G][8];
         {
@@ -75,7 +78,7 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
 #pragma unroll
             for (int d = 0; d < 8; ++d) o[h][d] = 0.f;
         }
-        const size_t kv_base = (size_t)li.kv_index * p.kv_layer_stride + (size_t)it.g * p.kv_head_stride + dofs;
+        const size_t kv_base = (size_t)it.kv_layer * p.kv_layer_stride + (size_t)it.g * p.kv_head_stride + dofs;
         const int32_t* bt = p.block_table + (size_t)it.b * p.max_blocks_per_seq;
 
         // segment 0: sink pages (only chunk 0 of a two-segment Local set), segment 1: window/full pages

@@ -4,8 +4,9 @@
 // tiled TMA copies (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers); four
 // consumer warps each take one 16-token page of a tile and run the GQA group tile on the
 // tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate): S = Q K^T with the group's query
-// heads in the M rows, online softmax in fp32 registers, O += P V with P split into a bf16
-// high and low part so that the softmax weights keep ~16 bits.  The work is memory bound:
+// heads in the N columns and the tokens in the M rows (S^T = K Q^T, O^T += V^T P^T, so every
+// accumulator register is live), online softmax in fp32 registers, P split into a bf16 high
+// and low part so that the softmax weights keep ~16 bits.  The work is memory bound:
 // the tensor cores are there to take the dot products off the issue slots, not for flops.
 // Serves the Local pass (Eq. 1, S^L) and the gated Full pass (S^F) with one code path.
 #include <cuda.h>
@@ -23,11 +24,12 @@ struct TmaCfg {
     static constexpr int kThreads = (kConsumerWarps + 1) * 32;
     static constexpr int kTilePages = 4;                    // one page per consumer warp
     static constexpr int kPageBytes = kPage * D * 2;        // one tensor, one kv head
-    static constexpr int kSlabs = D / 64;                   // 128-byte-row slabs per page
     static constexpr int kStageBytes = 2 * kTilePages * kPageBytes;  // K and V
     static constexpr int kStages = 98304 / kStageBytes;     // 96 KiB ring
-    static constexpr int kMergeBytes = 2 * 32 * 32 * 4 + 2 * 32 * 2 * 4;
-    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kMergeBytes + (int)sizeof(Plan) + 256;
+    static constexpr int kQSlotBytes = 8 * D * 2;           // q of one kv-head group (up to 8 heads)
+    static constexpr int kMergeBytes = 32 * 32 * 4 + 32 * 4 * 4;  // one warp's O fragment + (m, l) of two heads per lane
+    static constexpr int kBarBytes = 2 * kStages * 8 + 16;
+    static constexpr int kSmemBytes = kStages * (kStageBytes + kQSlotBytes) + kMergeBytes + (int)sizeof(Plan) + kBarBytes;
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -91,6 +93,12 @@ __device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* m
         : "memory");
 }
 
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -101,13 +109,21 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-// D = A(16x16, rows 8..15 zero) * B(16x8) + D, bf16 in, fp32 accumulate
-__device__ __forceinline__ void mma_top(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1)
+// D(16x8) += A(16x16) * B(16x8), bf16 in, fp32 accumulate
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1)
 {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// transpose of an 8x8 matrix of 16-bit elements held as one register per lane
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
@@ -121,8 +137,8 @@ __device__ __forceinline__ void consumer_sync()
 }
 
 // ------------------------------------------------------------------ tile sequence of an item
-// Both the producer and the consumers walk the same sequence: sink pages first (chunk 0 of a
-// two-segment Local set), then the chunk's window / full pages, four pages per tile.
+// Both the producer and the consumers walk the same sequence: sink pages first (the item that
+// starts a two-segment Local set), then the item's window / full pages, four pages per tile.
 struct TileWalk {
     int seg;       // 0 = sinks, 1 = window/full, 2 = done
     int pg;        // first logical page of the current tile
@@ -144,21 +160,31 @@ struct TileWalk {
     __device__ __forceinline__ bool done() const { return seg == 2; }
 };
 
+// Producer's view: runs of up to 32 consecutive logical pages of one item (8 tiles), whose block
+// ids are fetched with one warp-wide load well before the copies that need them are issued.
+struct PageRun {
+    int g, kv_layer, b;
+    const __nv_bfloat16* q;  // q rows of the item, copied with the first tile of the item
+    int pg, n;               // first logical page, pages in the run (1..32)
+    bool first;              // first run of its item
+};
+
 template <int D, int G>
-__global__ void __maxnreg__(200)
+__global__ void __launch_bounds__(TmaCfg<D>::kThreads, 2)
 splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap kmap,
                    const __grid_constant__ CUtensorMap vmap, const int blocks_per_layer)
 {
     using C = TmaCfg<D>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* ring = smem;                                           // kStages * kStageBytes
-    float* mbuf = reinterpret_cast<float*>(ring + C::kStages * C::kStageBytes);   // [2][32][32]
-    float* mlbuf = mbuf + 2 * 32 * 32;                              // [2][32][2]
-    Plan& plan = *reinterpret_cast<Plan*>(mlbuf + 2 * 32 * 2);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(&plan) + ((sizeof(Plan) + 15) & ~size_t(15)));
-    int* s_flags = reinterpret_cast<int*>(bars + 2 * C::kStages);   // [0] abort, [1] is_last
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* ring = smem;                                                 // kStages * kStageBytes
+    uint8_t* qring = ring + C::kStages * C::kStageBytes;                  // kStages * kQSlotBytes
+    float* mbuf = reinterpret_cast<float*>(qring + C::kStages * C::kQSlotBytes);  // [32][32]
+    float* mlbuf = mbuf + 32 * 32;                                        // [32][4]
+    Plan& plan = *reinterpret_cast<Plan*>(mlbuf + 32 * 4);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(&plan) + sizeof(Plan));
+    int* s_flags = reinterpret_cast<int*>(bars + 2 * C::kStages);         // [0] abort, [1] is_last
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + C::kStages);
+    static_assert(sizeof(Plan) % 8 == 0, "barriers must stay 8-byte aligned");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -172,50 +198,80 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     }
     build_plan(p, plan);  // ends with __syncthreads()
     volatile int* abort_flag = s_flags;
-    const int total = plan.total_items;
+    const int span = blockIdx.x;
+    if (span >= plan.nseg) return;
+    const int x0 = span_begin(plan, span), x_end = span_begin(plan, span + 1);
+    constexpr uint32_t kQBytes = G * D * 2;
 
     if (warp == C::kConsumerWarps) {
         // ============================ producer warp ============================
         const uint64_t policy = 0x12F0000000000000ull;  // L2 evict-first: the KV stream is read once
         uint32_t cnt = 0;
-        int id = blockIdx.x;
+        // walker over the runs of the span
+        int x = x0, take = 0, seg = 0, pg = 0;
         Item it;
-        TileWalk tw;
-        int blk = 0;
-        bool have = id < total;
-        if (have) {
-            it = decode_item(p, plan, id);
-            tw.start(it);
-            if (lane < tw.npages) blk = __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + tw.pg + lane);
-        }
-        while (have) {
-            // current tile: (it, tw, blk).  Look up the next tile's pages before blocking.
-            const Item cur_it = it;
-            const int cur_np = tw.npages, cur_blk = blk;
-            const int kv_layer = p.layers[cur_it.layer].kv_index;
-            tw.next(it);
-            if (tw.done()) {
-                id += gridDim.x;
-                have = id < total;
-                if (have) {
-                    it = decode_item(p, plan, id);
-                    tw.start(it);
+        bool more = true, item_first = true;
+        take = decode_item(p, plan, span, x, x_end, it);
+        seg = it.sink_pg1 > 0 ? 0 : 1;
+        pg = seg ? it.win_pg0 : 0;
+        auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when the span is done
+            if (!more) return false;
+            const int end = seg ? it.win_pg1 : it.sink_pg1;
+            r.g = it.g; r.kv_layer = it.kv_layer; r.b = it.b;
+            r.q = p.q + (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + (size_t)it.g * G) * D;
+            r.pg = pg;
+            r.n = min(32, end - pg);
+            r.first = item_first;
+            item_first = false;
+            blk = lane < r.n ? __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + pg + lane) : 0;
+            pg += r.n;
+            if (pg >= end) {
+                if (seg == 0) {
+                    seg = 1;
+                    pg = it.win_pg0;
+                } else {
+                    x += take;
+                    if (x < x_end) {
+                        take = decode_item(p, plan, span, x, x_end, it);
+                        seg = it.sink_pg1 > 0 ? 0 : 1;
+                        pg = seg ? it.win_pg0 : 0;
+                        item_first = true;
+                    } else {
+                        more = false;
+                    }
                 }
             }
-            if (have && lane < tw.npages)
-                blk = __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + tw.pg + lane);
-            const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
-            if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) break;
-            if (lane == 0) mbar_expect_tx(full0 + 8 * s, (uint32_t)cur_np * 2 * C::kPageBytes);
-            __syncwarp();
-            if (lane < cur_np) {
-                const uint32_t kdst = smem_u32(ring + s * C::kStageBytes + lane * C::kPageBytes);
-                const uint32_t vdst = kdst + C::kTilePages * C::kPageBytes;
-                const int bcoord = kv_layer * blocks_per_layer + cur_blk;
-                tma_load_page(kdst, &kmap, full0 + 8 * s, cur_it.g, bcoord, policy);
-                tma_load_page(vdst, &vmap, full0 + 8 * s, cur_it.g, bcoord, policy);
+            return true;
+        };
+        PageRun cur, nxt;
+        int blk_cur = 0, blk_nxt = 0;
+        bool have = fetch(cur, blk_cur);
+        bool dead = false;
+        while (have && !dead) {
+            const bool have_next = fetch(nxt, blk_nxt);  // block ids of the next run are in flight during this one
+            for (int t0 = 0; t0 < cur.n; t0 += 4) {
+                const int np = min(4, cur.n - t0);
+                const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
+                if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { dead = true; break; }
+                const bool with_q = cur.first && t0 == 0;
+                if (lane == 0)
+                    mbar_expect_tx(full0 + 8 * s, (uint32_t)np * 2 * C::kPageBytes + (with_q ? kQBytes : 0u));
+                __syncwarp();
+                const int blk = __shfl_sync(0xffffffffu, blk_cur, t0 + (lane & 3));
+                if (lane < np) {
+                    const uint32_t kdst = smem_u32(ring + s * C::kStageBytes + lane * C::kPageBytes);
+                    const uint32_t vdst = kdst + C::kTilePages * C::kPageBytes;
+                    const int bcoord = cur.kv_layer * blocks_per_layer + blk;
+                    tma_load_page(kdst, &kmap, full0 + 8 * s, cur.g, bcoord, policy);
+                    tma_load_page(vdst, &vmap, full0 + 8 * s, cur.g, bcoord, policy);
+                } else if (lane == 4 && with_q) {
+                    bulk_load(smem_u32(qring + s * C::kQSlotBytes), cur.q, kQBytes, full0 + 8 * s);
+                }
+                ++cnt;
             }
-            ++cnt;
+            cur = nxt;
+            blk_cur = blk_nxt;
+            have = have_next;
         }
         // Do not leave while copies may still be landing in this CTA's shared memory: wait
         // (bounded) until the consumers have released every stage that was armed.
@@ -231,31 +287,37 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     }
 
     // ================================ consumer warps ================================
-    const int row = lane >> 2;           // query head within the group (M row of the fragment)
-    const int qc = (lane & 3) * 2;       // column pair inside an 8-wide fragment
+    // Transposed GQA tile: tokens in the M rows, the group's query heads in the N columns.
+    //   S^T[16 tok x 8 heads] = K[16 tok x D] * Q^T[D x 8 heads]
+    //   O^T[D x 8 heads]     += V^T[D x 16 tok] * P^T[16 tok x 8 heads]
+    // so every accumulator register is a real (d, head) or (token, head) element.
+    const int hrow = lane >> 2;          // B-fragment column: the query head whose q this lane holds
+    const int qc = (lane & 3) * 2;       // accumulator columns: heads qc, qc+1; B-fragment k pair
     // ldmatrix row addresses inside one page (relative to the page base), 128-byte swizzle
-    const int k_tok = (lane & 7) + ((lane >> 4) << 3), k_half = (lane >> 3) & 1;
-    const int v_tok = (lane & 7) + (((lane >> 3) & 1) << 3), v_sel = lane >> 4;
+    const int k_tok = (lane & 7) + (((lane >> 3) & 1) << 3), k_half = lane >> 4;
+    const int v_tok = (lane & 7) + ((lane >> 4) << 3), v_sel = (lane >> 3) & 1;
     const int xr = lane & 7;
     uint32_t cnt = 0;
 
-    for (int id = blockIdx.x; id < total; id += gridDim.x) {
-        const Item it = decode_item(p, plan, id);
-        // Q fragments: rows >= G stay zero
+    for (int x = x0; x < x_end;) {
+        Item it;
+        x += decode_item(p, plan, span, x, x_end, it);
+        // Q^T fragments come with the item's first tile; heads >= G stay zero
         uint32_t qa[D / 16][2];
         {
-            const __nv_bfloat16* qb =
-                p.q + (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + (size_t)it.g * G + row) * D + qc;
+            const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
+            if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) break;
+            const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
 #pragma unroll
             for (int kc = 0; kc < D / 16; ++kc) {
-                qa[kc][0] = row < G ? __ldg(reinterpret_cast<const unsigned int*>(qb + kc * 16)) : 0u;
-                qa[kc][1] = row < G ? __ldg(reinterpret_cast<const unsigned int*>(qb + kc * 16 + 8)) : 0u;
+                qa[kc][0] = hrow < G ? qs[kc * 8] : 0u;
+                qa[kc][1] = hrow < G ? qs[kc * 8 + 4] : 0u;
             }
         }
-        float o[D / 8][4];
+        float o[D / 16][4];
 #pragma unroll
-        for (int n = 0; n < D / 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f;
+        for (int n = 0; n < D / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+        float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;  // heads qc and qc+1
 
         TileWalk tw;
         bool aborted = false;
@@ -269,61 +331,69 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 const bool edge = pos0 < vlo || pos0 + kPage > vhi;
                 const uint32_t kpage = smem_u32(ring + s * C::kStageBytes + warp * C::kPageBytes);
                 const uint32_t vpage = kpage + C::kTilePages * C::kPageBytes;
-                // ---- S = Q K^T for 16 tokens: two n-tiles of 8 ----
-                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                // ---- S^T = K Q^T for 16 tokens ----
+                float st[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int kc = 0; kc < D / 16; ++kc) {
                     const int chunk = (kc & 3) * 2 + k_half;
                     const uint32_t addr = kpage + (kc >> 2) * 2048 + k_tok * 128 + ((chunk ^ xr) << 4);
-                    uint32_t r0, r1, r2, r3;
-                    ldsm_x4(addr, r0, r1, r2, r3);
-                    mma_top(s0, qa[kc][0], qa[kc][1], r0, r1);
-                    mma_top(s1, qa[kc][0], qa[kc][1], r2, r3);
+                    uint32_t a0, a1, a2, a3;
+                    ldsm_x4(addr, a0, a1, a2, a3);
+                    mma16816(st, a0, a1, a2, a3, qa[kc][0], qa[kc][1]);
                 }
-                float x0 = s0[0] * p.scale_log2e, x1 = s0[1] * p.scale_log2e;
-                float x2 = s1[0] * p.scale_log2e, x3 = s1[1] * p.scale_log2e;
+                // st[0],st[1]: token hrow, heads qc,qc+1;  st[2],st[3]: token hrow+8
+                float x0s = st[0] * p.scale_log2e, x1s = st[1] * p.scale_log2e;
+                float x2s = st[2] * p.scale_log2e, x3s = st[3] * p.scale_log2e;
                 uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
                 if (edge) {  // positions outside [vlo, vhi) are not in the set
+                    const int ta = pos0 + hrow;
+                    const bool va = ta >= vlo && ta < vhi, vb = ta + 8 >= vlo && ta + 8 < vhi;
+                    x0s = va ? x0s : -INFINITY; x1s = va ? x1s : -INFINITY;
+                    x2s = vb ? x2s : -INFINITY; x3s = vb ? x3s : -INFINITY;
+                    // V^T fragments hold tokens qc, qc+1 (and +8) in their 16-bit halves
                     const int t0 = pos0 + qc;
                     const bool v0 = t0 >= vlo && t0 < vhi, v1 = t0 + 1 >= vlo && t0 + 1 < vhi;
                     const bool v2 = t0 + 8 >= vlo && t0 + 8 < vhi, v3 = t0 + 9 >= vlo && t0 + 9 < vhi;
-                    x0 = v0 ? x0 : -INFINITY; x1 = v1 ? x1 : -INFINITY;
-                    x2 = v2 ? x2 : -INFINITY; x3 = v3 ? x3 : -INFINITY;
                     mk0 = (v0 ? 0x0000ffffu : 0u) | (v1 ? 0xffff0000u : 0u);
                     mk1 = (v2 ? 0x0000ffffu : 0u) | (v3 ? 0xffff0000u : 0u);
                 }
-                // ---- online softmax (fp32, base 2) ----
-                float mx = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run, mx);
-                const float mu = (m_new == -INFINITY) ? 0.f : m_new;
-                const float alpha = ex2(m_run - mu);
-                const float p0 = ex2(x0 - mu), p1 = ex2(x1 - mu), p2 = ex2(x2 - mu), p3 = ex2(x3 - mu);
-                l_run = l_run * alpha + ((p0 + p1) + (p2 + p3));
-                m_run = m_new;
-                if (!__all_sync(0xffffffffu, alpha == 1.f)) {
+                // ---- online softmax over the 16 tokens (fp32, base 2); tokens live across lanes ----
+                float mxA = fmaxf(x0s, x2s), mxB = fmaxf(x1s, x3s);
 #pragma unroll
-                    for (int n = 0; n < D / 8; ++n) { o[n][0] *= alpha; o[n][1] *= alpha; }
+                for (int off = 4; off < 32; off <<= 1) {
+                    mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, off));
+                    mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, off));
                 }
-                // P as A fragments, split into bf16 high and low parts
-                const uint32_t ph0 = pack_bf16x2(p0, p1), ph1 = pack_bf16x2(p2, p3);
-                const uint32_t pl0 = pack_bf16x2(p0 - __uint_as_float(ph0 << 16), p1 - __uint_as_float(ph0 & 0xffff0000u));
-                const uint32_t pl1 = pack_bf16x2(p2 - __uint_as_float(ph1 << 16), p3 - __uint_as_float(ph1 & 0xffff0000u));
-                // ---- O += P V ----
+                const float mnA = fmaxf(mA, mxA), mnB = fmaxf(mB, mxB);
+                const float muA = (mnA == -INFINITY) ? 0.f : mnA, muB = (mnB == -INFINITY) ? 0.f : mnB;
+                const float alA = ex2(mA - muA), alB = ex2(mB - muB);
+                const float p0 = ex2(x0s - muA), p1 = ex2(x1s - muB), p2 = ex2(x2s - muA), p3 = ex2(x3s - muB);
+                lA = lA * alA + (p0 + p2);
+                lB = lB * alB + (p1 + p3);
+                mA = mnA;
+                mB = mnB;
+                if (!__all_sync(0xffffffffu, alA == 1.f && alB == 1.f)) {
 #pragma unroll
-                for (int np = 0; np < D / 16; ++np) {
-                    const int chunk = (np & 3) * 2 + v_sel;
-                    const uint32_t addr = vpage + (np >> 2) * 2048 + v_tok * 128 + ((chunk ^ xr) << 4);
-                    uint32_t r0, r1, r2, r3;
-                    ldsm_x4_t(addr, r0, r1, r2, r3);
+                    for (int n = 0; n < D / 16; ++n) { o[n][0] *= alA; o[n][1] *= alB; o[n][2] *= alA; o[n][3] *= alB; }
+                }
+                // P^T as B fragments: transpose the two 8x8 (token x head) tiles; bf16 high + low parts
+                const uint32_t hi0 = pack_bf16x2(p0, p1), hi1 = pack_bf16x2(p2, p3);
+                const uint32_t lo0 = pack_bf16x2(p0 - __uint_as_float(hi0 << 16), p1 - __uint_as_float(hi0 & 0xffff0000u));
+                const uint32_t lo1 = pack_bf16x2(p2 - __uint_as_float(hi1 << 16), p3 - __uint_as_float(hi1 & 0xffff0000u));
+                const uint32_t bh0 = movmatrix_t(hi0), bh1 = movmatrix_t(hi1);
+                const uint32_t bl0 = movmatrix_t(lo0), bl1 = movmatrix_t(lo1);
+                // ---- O^T += V^T P^T ----
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) {
+                    const int chunk = (mt & 3) * 2 + v_sel;
+                    const uint32_t addr = vpage + (mt >> 2) * 2048 + v_tok * 128 + ((chunk ^ xr) << 4);
+                    uint32_t a0, a1, a2, a3;
+                    ldsm_x4_t(addr, a0, a1, a2, a3);
                     if (edge) {  // slots outside the set may hold anything, NaN bit patterns included
-                        r0 &= mk0; r1 &= mk1; r2 &= mk0; r3 &= mk1;
+                        a0 &= mk0; a1 &= mk0; a2 &= mk1; a3 &= mk1;
                     }
-                    mma_top(o[2 * np], ph0, ph1, r0, r1);
-                    mma_top(o[2 * np], pl0, pl1, r0, r1);
-                    mma_top(o[2 * np + 1], ph0, ph1, r2, r3);
-                    mma_top(o[2 * np + 1], pl0, pl1, r2, r3);
+                    mma16816(o[mt], a0, a1, a2, a3, bh0, bh1);
+                    mma16816(o[mt], a0, a1, a2, a3, bl0, bl1);
                 }
             }
             __syncwarp();
@@ -331,69 +401,95 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         }
         if (aborted || *abort_flag) break;
 
-        // ---- merge the four warps' streams pairwise through shared memory (same fragment layout) ----
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        // ---- fold warps 1..3 into warp 0 through shared memory (all use the same fragment layout) ----
 #pragma unroll
-        for (int round = 0; round < 2; ++round) {
-            const int nsend = round == 0 ? 2 : 1;  // round 0: warps 2,3 -> 0,1; round 1: warp 1 -> 0
-            if (warp >= nsend && warp < 2 * nsend) {
-                float* dst = mbuf + (warp - nsend) * 32 * 32;
+        for (int off = 4; off < 32; off <<= 1) {
+            lA += __shfl_xor_sync(0xffffffffu, lA, off);
+            lB += __shfl_xor_sync(0xffffffffu, lB, off);
+        }
+#pragma unroll 1
+        for (int src_warp = 1; src_warp < C::kConsumerWarps; ++src_warp) {
+            if (warp == src_warp) {
 #pragma unroll
-                for (int n = 0; n < D / 8; ++n) {
-                    dst[(2 * n) * 32 + lane] = o[n][0];
-                    dst[(2 * n + 1) * 32 + lane] = o[n][1];
+                for (int n = 0; n < D / 16; ++n) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) mbuf[(4 * n + e) * 32 + lane] = o[n][e];
                 }
-                mlbuf[((warp - nsend) * 32 + lane) * 2] = m_run;
-                mlbuf[((warp - nsend) * 32 + lane) * 2 + 1] = l_run;
+                reinterpret_cast<float4*>(mlbuf)[lane] = make_float4(mA, lA, mB, lB);
             }
             consumer_sync();
-            if (warp < nsend) {
-                const float* src = mbuf + warp * 32 * 32;
-                const float m2 = mlbuf[(warp * 32 + lane) * 2], l2 = mlbuf[(warp * 32 + lane) * 2 + 1];
-                const float M = fmaxf(m_run, m2);
-                const float mu = (M == -INFINITY) ? 0.f : M;
-                const float sa = ex2(m_run - mu), sb = ex2(m2 - mu);
+            if (warp == 0) {
+                const float4 ml = reinterpret_cast<const float4*>(mlbuf)[lane];
+                const float MA = fmaxf(mA, ml.x), MB = fmaxf(mB, ml.z);
+                const float muA = (MA == -INFINITY) ? 0.f : MA, muB = (MB == -INFINITY) ? 0.f : MB;
+                const float saA = ex2(mA - muA), sbA = ex2(ml.x - muA);
+                const float saB = ex2(mB - muB), sbB = ex2(ml.z - muB);
 #pragma unroll
-                for (int n = 0; n < D / 8; ++n) {
-                    o[n][0] = o[n][0] * sa + src[(2 * n) * 32 + lane] * sb;
-                    o[n][1] = o[n][1] * sa + src[(2 * n + 1) * 32 + lane] * sb;
+                for (int n = 0; n < D / 16; ++n) {
+                    o[n][0] = o[n][0] * saA + mbuf[(4 * n + 0) * 32 + lane] * sbA;
+                    o[n][1] = o[n][1] * saB + mbuf[(4 * n + 1) * 32 + lane] * sbB;
+                    o[n][2] = o[n][2] * saA + mbuf[(4 * n + 2) * 32 + lane] * sbA;
+                    o[n][3] = o[n][3] * saB + mbuf[(4 * n + 3) * 32 + lane] * sbB;
                 }
-                l_run = l_run * sa + l2 * sb;
-                m_run = M;
+                lA = lA * saA + ml.y * sbA;
+                lB = lB * saB + ml.w * sbB;
+                mA = MA;
+                mB = MB;
             }
             consumer_sync();
         }
         // ---- warp 0 holds the CTA's (m, l, o): store the result or publish the partial ----
+        // o[n][0..1]: d = 16n + hrow, heads qc, qc+1;  o[n][2..3]: d = 16n + 8 + hrow
         constexpr int W = D + 2;
         const float kLn2 = 0.6931471805599453f;
         if (it.nchunks == 1) {
-            if (warp == 0 && row < G) {
-                const float inv = 1.f / l_run;
-                const int h = it.g * G + row;
-                const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + qc;
-                if (p.out_bf16) {
-                    uint32_t* ob = reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(p.out) + idx);
+            if (warp == 0) {
 #pragma unroll
-                    for (int n = 0; n < D / 8; ++n) ob[n * 4] = pack_bf16x2(o[n][0] * inv, o[n][1] * inv);
-                } else {
-                    float2* of = reinterpret_cast<float2*>(reinterpret_cast<float*>(p.out) + idx);
+                for (int e = 0; e < 2; ++e) {
+                    const int hg = qc + e;
+                    if (hg < G) {
+                        const float inv = 1.f / (e ? lB : lA);
+                        const int h = it.g * G + hg;
+                        const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + hrow;
+                        if (p.out_bf16) {
+                            __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) + idx;
 #pragma unroll
-                    for (int n = 0; n < D / 8; ++n) of[n * 4] = make_float2(o[n][0] * inv, o[n][1] * inv);
+                            for (int n = 0; n < D / 16; ++n) {
+                                ob[n * 16] = __float2bfloat16_rn(o[n][e] * inv);
+                                ob[n * 16 + 8] = __float2bfloat16_rn(o[n][2 + e] * inv);
+                            }
+                        } else {
+                            float* of = reinterpret_cast<float*>(p.out) + idx;
+#pragma unroll
+                            for (int n = 0; n < D / 16; ++n) {
+                                of[n * 16] = o[n][e] * inv;
+                                of[n * 16 + 8] = o[n][2 + e] * inv;
+                            }
+                        }
+                        if (p.lse && hrow == 0)
+                            p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] =
+                                ((e ? mB : mA) + log2f(e ? lB : lA)) * kLn2;
+                    }
                 }
-                if (p.lse && (lane & 3) == 0)
-                    p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] = (m_run + log2f(l_run)) * kLn2;
             }
         } else {
-            if (warp == 0 && row < G) {
-                float* slot = partial_slot(p, it, G, W) + row * W;
-                if ((lane & 3) == 0) {
-                    __stcg(slot, m_run);
-                    __stcg(slot + 1, l_run);
-                }
+            if (warp == 0) {
 #pragma unroll
-                for (int n = 0; n < D / 8; ++n)
-                    __stcg(reinterpret_cast<float2*>(slot + 2 + n * 8 + qc), make_float2(o[n][0], o[n][1]));
+                for (int e = 0; e < 2; ++e) {
+                    const int hg = qc + e;
+                    if (hg < G) {
+                        float* slot = partial_slot(p, it, G, W) + hg * W;
+                        if (hrow == 0) {
+                            __stcg(slot, e ? mB : mA);
+                            __stcg(slot + 1, e ? lB : lA);
+                        }
+#pragma unroll
+                        for (int n = 0; n < D / 16; ++n) {
+                            __stcg(slot + 2 + n * 16 + hrow, o[n][e]);
+                            __stcg(slot + 2 + n * 16 + 8 + hrow, o[n][2 + e]);
+                        }
+                    }
+                }
             }
             __threadfence();
             consumer_sync();
@@ -468,6 +564,8 @@ static cudaError_t launch_tma_t(const AttnParams& p, const void* kmap, const voi
         cudaError_t e = cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              TmaCfg<D>::kSmemBytes);
         if (e != cudaSuccess) return e;
+        (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                   cudaSharedmemCarveoutMaxShared);
         attr_set = true;
     }
     splitkv_tma_kernel<D, G><<<grid, TmaCfg<D>::kThreads, TmaCfg<D>::kSmemBytes, st>>>(
@@ -485,6 +583,8 @@ static int occupancy_tma_t()
         (void)cudaGetLastError();
         return 0;
     }
+    (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                               cudaSharedmemCarveoutMaxShared);
     cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, splitkv_tma_kernel<D, G>, TmaCfg<D>::kThreads,
                                                   TmaCfg<D>::kSmemBytes);
     return n;
