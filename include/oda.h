@@ -191,6 +191,37 @@ int32_t oda_resolved_variant(const oda_ctx_t* ctx);
 /* Grid size (CTAs) the attention kernels of this context launch with. */
 int32_t oda_attention_grid(const oda_ctx_t* ctx);
 
+/*
+ * Local pass of ONE attention layer without any workspace.  (The paper has no counterpart:
+ * this entry point exists for integration, not for the method.)
+ *
+ * Some callers of this library cannot allocate device memory at the point where they call
+ * it -- a plugin running inside another runtime's execution callback, a process whose memory
+ * pool was handed out completely at start-up, code that must not disturb an allocator it
+ * does not own -- and so cannot provide the workspace oda_set_workspace() asks for.  For them
+ * the split partials, merge tickets and status word of this call live in a fixed array inside
+ * the library's device image (about 2.2 MiB, held by every GPU that loads the library until
+ * the process exits).  The call performs no device or host allocation.
+ *
+ * Same result as oda_local_decode() for a one-layer stack: q [batch, q_heads, head_dim] bf16,
+ * out [batch, q_heads, head_dim] fp32, lse [batch, q_heads] fp32 (nullable), cache addressed by
+ * block*kv_block_stride + slot*kv_token_stride + head*kv_head_stride + d, Eq. 1 with the given
+ * window and sinks, sm_scale 0 => 1/sqrt(head_dim).  All pointers are device pointers.
+ *
+ * Limits: batch <= 16 and batch*kv_heads <= 256; anything larger returns ODA_ERR_UNSUPPORTED
+ * with nothing enqueued (the scratch is never used beyond its size).
+ * The first call on each device looks up the array's device address (that device must be
+ * current) -- make that first call outside any stream capture.
+ * Every call on a device uses the same array: a call clears what it needs to start from zero,
+ * but two calls that overlap on the GPU (different streams) race.  Serialise them.
+ */
+oda_status_t oda_local_decode_static(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads,
+                                     int32_t head_dim, int32_t window, int32_t sinks, float sm_scale,
+                                     int64_t kv_block_stride, int64_t kv_token_stride,
+                                     int64_t kv_head_stride, int32_t max_blocks_per_seq, const void* q,
+                                     const void* k_cache, const void* v_cache, const int32_t* block_table,
+                                     const int32_t* seq_lens, float* out, float* lse, void* stream);
+
 const char* oda_status_string(oda_status_t s);
 const char* oda_last_error(const oda_ctx_t* ctx); /* host string describing the last failure */
 const char* oda_version(void);

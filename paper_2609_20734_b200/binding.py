@@ -22,7 +22,7 @@ EXPORTS = [
     "oda_create", "oda_destroy", "oda_workspace_bytes", "oda_set_workspace", "oda_local_decode",
     "oda_recall_score", "oda_full_decode_gated", "oda_step", "oda_step_host",
     "oda_read_device_status", "oda_launch_count", "oda_resolved_variant", "oda_attention_grid",
-    "oda_status_string", "oda_last_error", "oda_version",
+    "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
 ]
 
 
@@ -85,6 +85,9 @@ def load_library():
         lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
         lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
                                       ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+        lib.oda_local_decode_static.argtypes = [i32, i32, i32, i32, i32, i32, f32, ctypes.c_int64,
+                                                ctypes.c_int64, ctypes.c_int64, i32, vp, vp, vp, vp, vp,
+                                                vp, vp, vp]
         lib.oda_read_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         lib.oda_launch_count.argtypes = [vp]
         lib.oda_launch_count.restype = ctypes.c_int64
@@ -263,6 +266,20 @@ class OdaContext:
     @property
     def attention_grid(self) -> int:
         return self.lib.oda_attention_grid(self._h)
+
+
+def local_decode_static(batch, num_q_heads, num_kv_heads, head_dim, window, sinks, sm_scale,
+                        kv_block_stride, kv_token_stride, kv_head_stride, max_blocks_per_seq, q,
+                        k_cache, v_cache, block_table, seq_lens, out, lse=None, stream=None) -> None:
+    """Local pass of one layer with no workspace: for callers that cannot allocate device memory
+    (the scratch is a fixed array inside the library).  Limits: batch <= 16, batch*kv_heads <= 256.
+    Calls on one device must not overlap; make the first call on a device outside stream capture."""
+    st = load_library().oda_local_decode_static(
+        batch, num_q_heads, num_kv_heads, head_dim, window, sinks, float(sm_scale), kv_block_stride,
+        kv_token_stride, kv_head_stride, max_blocks_per_seq, _ptr(q), _ptr(k_cache), _ptr(v_cache),
+        _ptr(block_table), _ptr(seq_lens), _ptr(out), _ptr(lse), _stream() if stream is None else stream)
+    if st != 0:
+        raise OdaError(st, "oda_local_decode_static", load_library().oda_status_string(st).decode())
 
 
 def version() -> str:
