@@ -91,7 +91,8 @@ typedef struct {
     int32_t head_d_ext;
     int32_t head_use_attn_out;
     int32_t head_d_hidden;
-    int32_t reserved;
+    int32_t reserved;           /* 0; 1 = launch every kernel fully serialised (no programmatic
+                                 * dependent launch between the kernels of a step) */
 } oda_config_t;
 
 /* Lifetime.  oda_create validates and copies the config (host only, no device work).

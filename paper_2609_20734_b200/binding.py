@@ -125,6 +125,7 @@ class OdaConfig:
     head_d_ext: int = 0
     head_use_attn_out: int = 1
     head_d_hidden: int = 0
+    serialize_launches: int = 0   # 1 = no programmatic dependent launch between the kernels of a step
     _keep: list = field(default_factory=list, repr=False)
 
     def to_c(self) -> _Config:
@@ -141,7 +142,7 @@ class OdaConfig:
             arr(self.layer_window, np.int32), arr(self.layer_sinks, np.int32),
             arr(self.layer_gated, np.uint8), arr(self.layer_kv_index, np.int32),
             self.kv_layer_stride, self.kv_block_stride, self.kv_token_stride, self.kv_head_stride,
-            self.head_d_ext, self.head_use_attn_out, self.head_d_hidden, 0)
+            self.head_d_ext, self.head_use_attn_out, self.head_d_hidden, self.serialize_launches)
 
 
 def _ptr(t) -> Optional[int]:

@@ -52,6 +52,7 @@ struct oda_ctx {
     int blocks_per_layer = 0;
     int64_t blocks_bound = 1;
     int64_t launches = 0;
+    bool use_pdl = true;  // programmatic dependent launch between the kernels of a step
     std::string err;
 };
 
@@ -112,7 +113,8 @@ oda_status_t check_attn_args(oda_ctx* c, int lb, int le, int batch, const void* 
 
 oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, const void* q,
                               const void* k, const void* v, const int32_t* bt, const int32_t* sl,
-                              const uint8_t* flags, void* out, float* lse, cudaStream_t st)
+                              const uint8_t* flags, void* out, float* lse, cudaStream_t st,
+                              int32_t* advance = nullptr, bool* advanced = nullptr)
 {
     const oda_config_t& f = c->cfg;
     AttnParams p;
@@ -157,6 +159,9 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
         if (n && (mode == 0 || c->cls_gated[i])) any = true;
     }
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
+    p.advance_seq_lens = advance;
+    p.done_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 128);
+    if (advanced) *advanced = advance != nullptr;
     cudaError_t e;
     if (c->variant == ODA_VARIANT_TMA_MMA) {
         if (c->kmap_base != k) {
@@ -171,9 +176,9 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
                 return fail(c, ODA_ERR_CUDA, "cuTensorMapEncodeTiled failed for v_cache");
             c->vmap_base = v;
         }
-        e = launch_splitkv_tma(p, c->kmap, c->vmap, c->blocks_per_layer, f.head_dim, c->group, c->grid, st);
+        e = launch_splitkv_tma(p, c->kmap, c->vmap, c->blocks_per_layer, f.head_dim, c->group, c->grid, st, c->use_pdl);
     } else {
-        e = launch_splitkv_simt(p, f.head_dim, c->group, c->grid, st);
+        e = launch_splitkv_simt(p, f.head_dim, c->group, c->grid, st, c->use_pdl);
     }
     if (e != cudaSuccess) return cuda_fail(c, e, "attention kernel launch");
     c->launches += 1;
@@ -281,6 +286,7 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         delete c;
         return ODA_ERR_UNSUPPORTED;  // layer stride is not a whole number of blocks
     }
+    c->use_pdl = cfg->reserved == 0;  // reserved = 1 turns programmatic dependent launch off
     c->variant = cfg->variant == ODA_VARIANT_AUTO ? (tma_ok ? ODA_VARIANT_TMA_MMA : ODA_VARIANT_SIMT) : cfg->variant;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
@@ -388,7 +394,7 @@ oda_status_t oda_recall_score(oda_ctx_t* c, int32_t batch, const float* feat_ext
     p.attn_bf16 = f.out_dtype;
     p.max_batch = f.max_batch;
     p.threshold = threshold;
-    cudaError_t e = launch_recall_head(p, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_recall_head(p, static_cast<cudaStream_t>(stream), c->use_pdl);
     if (e != cudaSuccess) return cuda_fail(c, e, "recall head launch");
     c->launches += 1;
     return ODA_OK;
@@ -417,13 +423,15 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     s = oda_recall_score(c, B, a->feat_ext, attn_last, a->W1, a->b1, a->w2, a->b2, a->threshold,
                          a->override_flags, a->scores, a->logits, a->flags, a->counters, stream);
     if (s != ODA_OK) return s;
+    bool advanced = false;
     if (c->last_gated >= 0) {
+        // the Full kernel is the last reader of seq_lens in the step: it also advances them
         s = launch_attention(c, 1, 0, L, B, qf, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
-                             a->flags, a->out, a->lse, st);
+                             a->flags, a->out, a->lse, st, a->advance_seq_lens ? a->seq_lens : nullptr, &advanced);
         if (s != ODA_OK) return s;
     }
-    if (a->advance_seq_lens) {
-        cudaError_t e = launch_advance_seq_lens(a->seq_lens, B, st);
+    if (a->advance_seq_lens && !advanced) {
+        cudaError_t e = launch_advance_seq_lens(a->seq_lens, B, st, c->use_pdl);
         if (e != cudaSuccess) return cuda_fail(c, e, "seq_lens advance launch");
         c->launches += 1;
     }

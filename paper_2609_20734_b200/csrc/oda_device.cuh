@@ -44,7 +44,15 @@ struct AttnParams {
     float scale_log2e;     // sm_scale * log2(e)
     int32_t cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
     int32_t cls_layers_in_call[kMaxClasses];
+    int32_t* advance_seq_lens;  // nullable: seq_lens to increment once every CTA has read them
+    int32_t* done_counter;      // zero between launches
 };
+
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start while its predecessor in the stream is still running; it must pass griddep_wait() before
+// it touches memory the predecessor reads or writes.  Both are no-ops for an ordinary launch.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Work decomposition.  A unit is one (layer, request, kv head); it owns np pages of KV (the
 // pages of its Eq. 1 window segment, or of the whole history in Full mode).  All units are laid
@@ -179,6 +187,28 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         }
     }
     __syncthreads();
+    // Every CTA now works from its shared-memory copy of seq_lens.  If the step asked for it, the
+    // CTA that gets here last moves the device-side lengths on (no CTA reads them again).
+    if (p.advance_seq_lens && tid == 0) {
+        __threadfence();
+        const int old = atomicAdd(p.done_counter, 1);
+        if (old == (int)gridDim.x - 1) {
+            *p.done_counter = 0;
+            for (int b = 0; b < B; ++b) p.advance_seq_lens[b] += 1;
+        }
+    }
+}
+
+// Warms L2 with the block table while the plan is being built (the table is not produced by the
+// kernels of this library, so this may run before griddep_wait()).
+__device__ __forceinline__ void prefetch_block_table(const AttnParams& p)
+{
+    const size_t bytes = (size_t)p.batch * p.max_blocks_per_seq * sizeof(int32_t);
+    const size_t lines = (bytes + 127) / 128;
+    if (lines > 8192) return;
+    const char* base = reinterpret_cast<const char*>(p.block_table);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < lines; i += (size_t)gridDim.x * blockDim.x)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
 }
 
 __device__ __forceinline__ int span_begin(const Plan& pl, int j)

@@ -7,7 +7,8 @@ namespace oda {
 
 struct AttnParams;
 
-cudaError_t launch_splitkv_simt(const AttnParams& p, int head_dim, int group, int grid, cudaStream_t st);
+cudaError_t launch_splitkv_simt(const AttnParams& p, int head_dim, int group, int grid, cudaStream_t st,
+                                bool pdl = false);
 int occupancy_splitkv_simt(int head_dim, int group);
 
 // TMA + tensor-core variant.  kmap / vmap point at 128-byte CUtensorMap objects (host memory).
@@ -15,7 +16,7 @@ bool tma_variant_supported(int head_dim, int64_t layer_stride, int64_t block_str
 bool encode_kv_map(void* out_map, const void* base, int head_dim, int num_kv_heads, int64_t token_stride,
                    int64_t head_stride, int64_t block_stride, int64_t num_blocks_bound);
 cudaError_t launch_splitkv_tma(const AttnParams& p, const void* kmap, const void* vmap, int blocks_per_layer,
-                               int head_dim, int group, int grid, cudaStream_t st);
+                               int head_dim, int group, int grid, cudaStream_t st, bool pdl = false);
 int occupancy_splitkv_tma(int head_dim, int group);
 
 struct HeadParams {
@@ -34,7 +35,7 @@ struct HeadParams {
 };
 
 int recall_head_grid(int d_hidden);
-cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st);
-cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st);
+cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl = false);
+cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st, bool pdl = false);
 
 }  // namespace oda

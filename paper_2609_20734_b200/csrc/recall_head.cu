@@ -6,6 +6,7 @@
 // arrives last (one atomic ticket, no waiting) adds them in CTA order and writes the flags,
 // so the result does not depend on scheduling.
 #include <cuda_bf16.h>
+#include "launch_ex.cuh"
 #include "oda_launch.h"
 
 namespace oda {
@@ -25,6 +26,8 @@ __global__ void __launch_bounds__(kHeadWarps * 32) recall_head_kernel(const __gr
 {
     __shared__ float s_h[kHeadWarps][256];
     __shared__ int s_last;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the Local output it reads comes from the previous kernel
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j = blockIdx.x * kHeadWarps + warp;
     const int d_in = p.d_ext + p.d_attn;
@@ -95,6 +98,8 @@ __global__ void __launch_bounds__(kHeadWarps * 32) recall_head_kernel(const __gr
 __global__ void copy_flags_kernel(const uint8_t* __restrict__ ov, uint8_t* __restrict__ flags,
                                   float* scores, float* logits, int32_t* counters, int batch)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < batch; b += gridDim.x * blockDim.x) {
         uint8_t f = ov[b] ? 1 : 0;
         flags[b] = f;
@@ -109,25 +114,24 @@ __global__ void copy_flags_kernel(const uint8_t* __restrict__ ov, uint8_t* __res
 
 __global__ void advance_seq_lens_kernel(int32_t* seq_lens, int batch)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < batch; b += gridDim.x * blockDim.x) seq_lens[b] += 1;
 }
 
 int recall_head_grid(int d_hidden) { return (d_hidden + kHeadWarps - 1) / kHeadWarps; }
 
-cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st)
+cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl)
 {
-    if (p.d_hidden <= 0) {
-        copy_flags_kernel<<<1, 256, 0, st>>>(p.override_flags, p.flags, p.scores, p.logits, p.counters, p.batch);
-    } else {
-        recall_head_kernel<<<recall_head_grid(p.d_hidden), kHeadWarps * 32, 0, st>>>(p);
-    }
-    return cudaGetLastError();
+    if (p.d_hidden <= 0)
+        return launch_ex(copy_flags_kernel, dim3(1), dim3(128), 0, st, pdl, p.override_flags, p.flags, p.scores,
+                         p.logits, p.counters, p.batch);
+    return launch_ex(recall_head_kernel, dim3(recall_head_grid(p.d_hidden)), dim3(kHeadWarps * 32), 0, st, pdl, p);
 }
 
-cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st)
+cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st, bool pdl)
 {
-    advance_seq_lens_kernel<<<1, 256, 0, st>>>(seq_lens, batch);
-    return cudaGetLastError();
+    return launch_ex(advance_seq_lens_kernel, dim3(1), dim3(128), 0, st, pdl, seq_lens, batch);
 }
 
 }  // namespace oda

@@ -3,6 +3,7 @@
 // softmax per lane group, then a cross-warp merge and the split merge of oda_device.cuh.
 // Serves both the Local pass (Eq. 1, S^L) and the gated Full pass (S^F).
 #include "oda_device.cuh"
+#include "launch_ex.cuh"
 #include "oda_launch.h"
 
 namespace oda {
@@ -46,7 +47,10 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
     __shared__ float s_part[G][C::kW];
     __shared__ int s_is_last;
 
+    prefetch_block_table(p);
+    griddep_wait();
     build_plan(p, plan);
+    griddep_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sub = lane / C::kLPR;               // which row of a warp-wide load this lane reads
     const int dofs = (lane % C::kLPR) * 8;        // this lane's 8 head-dim elements
@@ -202,10 +206,9 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
 }
 
 template <int D, int G>
-static cudaError_t launch_simt_t(const AttnParams& p, int grid, cudaStream_t st)
+static cudaError_t launch_simt_t(const AttnParams& p, int grid, cudaStream_t st, bool pdl)
 {
-    splitkv_simt_kernel<D, G><<<grid, SimtCfg<D, G>::kThreads, 0, st>>>(p);
-    return cudaGetLastError();
+    return launch_ex(splitkv_simt_kernel<D, G>, dim3(grid), dim3(SimtCfg<D, G>::kThreads), 0, st, pdl, p);
 }
 
 template <int D, int G>
@@ -231,10 +234,10 @@ static int occupancy_simt_t()
         }                                                                              \
     } while (0)
 
-cudaError_t launch_splitkv_simt(const AttnParams& p, int head_dim, int group, int grid, cudaStream_t st)
+cudaError_t launch_splitkv_simt(const AttnParams& p, int head_dim, int group, int grid, cudaStream_t st, bool pdl)
 {
     cudaError_t e = cudaErrorInvalidValue;
-    ODA_DISPATCH_DG(head_dim, group, e = (launch_simt_t<DD, GG>(p, grid, st)));
+    ODA_DISPATCH_DG(head_dim, group, e = (launch_simt_t<DD, GG>(p, grid, st, pdl)));
     return e;
 }
 

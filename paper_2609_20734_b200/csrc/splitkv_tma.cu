@@ -12,11 +12,20 @@
 #include <cuda.h>
 
 #include "oda_device.cuh"
+#include "launch_ex.cuh"
 #include "oda_launch.h"
 
 namespace oda {
 
 constexpr int kStatusWaitTimeout = 4;
+
+#ifdef ODA_TIMELINE
+__device__ unsigned long long g_timeline[1024 * 8];
+#define ODA_TL(slot) do { if ((threadIdx.x & 31) == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_timeline[blockIdx.x * 8 + (slot)] = t_; } } while (0)
+extern "C" int oda_debug_timeline(unsigned long long* host, int n) { return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n); }
+#else
+#define ODA_TL(slot) do { } while (0)
+#endif
 
 template <int D>
 struct TmaCfg {
@@ -187,6 +196,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     static_assert(sizeof(Plan) % 8 == 0, "barriers must stay 8-byte aligned");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) ODA_TL(0);
     if (tid == 0) {
         for (int s = 0; s < C::kStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
@@ -195,8 +205,15 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         s_flags[0] = 0;
         s_flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&kmap)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&vmap)) : "memory");
     }
-    build_plan(p, plan);  // ends with __syncthreads()
+    prefetch_block_table(p);
+    griddep_wait();       // everything above is independent of the previous kernel in the stream
+    if (tid == 0) ODA_TL(1);
+    build_plan(p, plan);  // ends with a barrier
+    griddep_launch_dependents();
+    if (tid == 0) ODA_TL(2);
     volatile int* abort_flag = s_flags;
     const int span = blockIdx.x;
     if (span >= plan.nseg) return;
@@ -254,6 +271,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { dead = true; break; }
                 const bool with_q = cur.first && t0 == 0;
+                if (cnt == 0) ODA_TL(3);
                 if (lane == 0)
                     mbar_expect_tx(full0 + 8 * s, (uint32_t)np * 2 * C::kPageBytes + (with_q ? kQBytes : 0u));
                 __syncwarp();
@@ -307,6 +325,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         {
             const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
             if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) break;
+            if (cnt == 0 && warp == 0) ODA_TL(4);
             const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
 #pragma unroll
             for (int kc = 0; kc < D / 16; ++kc) {
@@ -400,6 +419,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             if (lane == 0) mbar_arrive(empty0 + 8 * s);
         }
         if (aborted || *abort_flag) break;
+        if (warp == 0) ODA_TL(5);
 
         // ---- fold warps 1..3 into warp 0 through shared memory (all use the same fragment layout) ----
 #pragma unroll
@@ -501,6 +521,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             }
             consumer_sync();  // s_flags[1] is reused by the next item
         }
+        if (warp == 0) ODA_TL(6);
     }
 }
 
@@ -557,7 +578,7 @@ bool encode_kv_map(void* out_map, const void* base, int head_dim, int num_kv_hea
 
 template <int D, int G>
 static cudaError_t launch_tma_t(const AttnParams& p, const void* kmap, const void* vmap, int blocks_per_layer,
-                                int grid, cudaStream_t st)
+                                int grid, cudaStream_t st, bool pdl)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -568,10 +589,9 @@ static cudaError_t launch_tma_t(const AttnParams& p, const void* kmap, const voi
                                    cudaSharedmemCarveoutMaxShared);
         attr_set = true;
     }
-    splitkv_tma_kernel<D, G><<<grid, TmaCfg<D>::kThreads, TmaCfg<D>::kSmemBytes, st>>>(
-        p, *reinterpret_cast<const CUtensorMap*>(kmap), *reinterpret_cast<const CUtensorMap*>(vmap),
-        blocks_per_layer);
-    return cudaGetLastError();
+    return launch_ex(splitkv_tma_kernel<D, G>, dim3(grid), dim3(TmaCfg<D>::kThreads), TmaCfg<D>::kSmemBytes, st, pdl,
+                     p, *reinterpret_cast<const CUtensorMap*>(kmap), *reinterpret_cast<const CUtensorMap*>(vmap),
+                     blocks_per_layer);
 }
 
 template <int D, int G>
@@ -606,10 +626,10 @@ static int occupancy_tma_t()
     } while (0)
 
 cudaError_t launch_splitkv_tma(const AttnParams& p, const void* kmap, const void* vmap, int blocks_per_layer,
-                               int head_dim, int group, int grid, cudaStream_t st)
+                               int head_dim, int group, int grid, cudaStream_t st, bool pdl)
 {
     cudaError_t e = cudaErrorInvalidValue;
-    ODA_DISPATCH_DG(head_dim, group, e = (launch_tma_t<DD, GG>(p, kmap, vmap, blocks_per_layer, grid, st)));
+    ODA_DISPATCH_DG(head_dim, group, e = (launch_tma_t<DD, GG>(p, kmap, vmap, blocks_per_layer, grid, st, pdl)));
     return e;
 }
 

@@ -128,7 +128,7 @@ def test_tiny_config_eight_steps_with_learned_flags():
     c = counters.cpu().numpy()
     assert c[0, 0] == wl.steps and c[0, 1] == 2
     assert ctx.read_device_status() == 0
-    assert ctx.launch_count == wl.steps * 4
+    assert ctx.launch_count == wl.steps * 3   # Local, head, gated Full (which also advances seq_lens)
 
 
 def _small_batched():
