@@ -1,7 +1,9 @@
 // C-ABI layer of the ODA decode library: argument validation, workspace layout and
 // stream-ordered kernel launches.  No device memory is allocated here, and nothing
 // synchronises except the two entry points whose contract says so.
+#include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -38,7 +40,10 @@ struct oda_ctx {
     int num_sms = 148;
     int variant = ODA_VARIANT_SIMT;
     int grid = 148;
-    int min_span_pages = 8;
+    int min_span_pages = 16;
+    int first_span_pct = 88;
+    int tail_span_pct = 6;
+    int dynamic_min_fair_pages = 1 << 30;  // dynamic hand-out off: measured slower than the static split (see oda_device.cuh)
     int max_items = 0;
     int head_grid = 1;
     WsLayout lay{};
@@ -82,7 +87,7 @@ void compute_layout(oda_ctx* c)
     w.layers = take(L * sizeof(LayerInfo));
     w.tickets = take(L * B * f.num_kv_heads * sizeof(int32_t));
     w.head_partial = take((size_t)c->head_grid * B * sizeof(float));
-    w.partials = take((size_t)c->max_items * c->group * (D + 2) * sizeof(float));
+    w.partials = take((size_t)c->max_items * c->group * (D + kPartHdr) * sizeof(float));
     w.st_q_local = take(L * B * Hq * D * 2);
     w.st_q_full = take(L * B * Hq * D * 2);
     w.st_feat = take(B * (size_t)(f.head_d_ext > 0 ? f.head_d_ext : 1) * 4);
@@ -146,6 +151,9 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     p.mode = mode;
     p.ncls = c->ncls;
     p.min_span_pages = c->min_span_pages;
+    p.first_span_pct = c->first_span_pct;
+    p.tail_span_pct = c->tail_span_pct;
+    p.dynamic_min_fair_pages = c->dynamic_min_fair_pages;
     p.max_items = c->max_items;
     p.scale_log2e = c->scale * 1.4426950408889634f;
     bool any = false;
@@ -161,6 +169,8 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
     p.advance_seq_lens = advance;
     p.done_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 128);
+    p.span_counter = c->variant == ODA_VARIANT_TMA_MMA ? reinterpret_cast<int32_t*>(c->ws + c->lay.status + 160) : nullptr;
+    p.exit_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 192);
     if (advanced) *advanced = advance != nullptr;
     cudaError_t e;
     if (c->variant == ODA_VARIANT_TMA_MMA) {
@@ -286,6 +296,10 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         delete c;
         return ODA_ERR_UNSUPPORTED;  // layer stride is not a whole number of blocks
     }
+    if (const char* e = std::getenv("ODA_MIN_SPAN_PAGES")) c->min_span_pages = std::max(1, std::atoi(e));
+    if (const char* e = std::getenv("ODA_TAIL_SPAN_PCT")) c->tail_span_pct = std::min(100, std::max(1, std::atoi(e)));
+    if (const char* e = std::getenv("ODA_DYNAMIC_MIN_FAIR")) c->dynamic_min_fair_pages = std::max(1, std::atoi(e));
+    if (const char* e = std::getenv("ODA_FIRST_SPAN_PCT")) c->first_span_pct = std::min(100, std::max(1, std::atoi(e)));
     c->use_pdl = cfg->reserved == 0;  // reserved = 1 turns programmatic dependent launch off
     c->variant = cfg->variant == ODA_VARIANT_AUTO ? (tma_ok ? ODA_VARIANT_TMA_MMA : ODA_VARIANT_SIMT) : cfg->variant;
     int dev = 0, sms = 0;
@@ -300,7 +314,7 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         c->num_sms = 148;  // no device visible: sizes follow a B200 so that host-only checks still work
         c->grid = 148 * 2;
     }
-    c->max_items = c->grid + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
+    c->max_items = c->grid * kMaxLevels + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
     c->head_grid = cfg->head_d_hidden > 0 ? recall_head_grid(cfg->head_d_hidden) : 1;
     compute_layout(c);
     *out_ctx = c;

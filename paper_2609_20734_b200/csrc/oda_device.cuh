@@ -12,6 +12,7 @@ constexpr int kPage = 16;          // tokens per KV block
 constexpr int kMaxBatch = 128;
 constexpr int kMaxLayers = 256;
 constexpr int kMaxClasses = 4;     // distinct (window, sinks, gated) triples in one stack
+constexpr int kPartHdr = 4;        // a partial row is (m, l, -, -, o[D]): o starts 16-byte aligned
 
 // device status bits
 constexpr int kStatusBadSeqLen = 1;
@@ -30,7 +31,7 @@ struct AttnParams {
     const uint8_t* flags;  // Full mode: per-request gate; Local mode: nullptr
     void* out;
     float* lse;
-    float* partials;       // [max_items][G][D+2]: m (log2 units), l, unnormalised o
+    float* partials;       // [max_items][G][kPartHdr + D]: m (log2 units), l, unnormalised o
     int32_t* tickets;      // [num_layers][max_batch][Hkv], zero between launches
     int32_t* status;
     const LayerInfo* layers;
@@ -39,13 +40,18 @@ struct AttnParams {
     int32_t num_q_heads, num_kv_heads, max_blocks_per_seq, out_bf16;
     int32_t mode;          // 0 = Local (Eq. 1 S^L), 1 = gated Full (S^F)
     int32_t ncls;
-    int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
+    int32_t min_span_pages;  // smallest span handed out (unless there are fewer pages)
+    int32_t first_span_pct;  // first-level span length as a percentage of the fair share per CTA
+    int32_t tail_span_pct;   // length of the spans handed out after the first level, same unit
+    int32_t dynamic_min_fair_pages;  // below this fair share the split is one static level
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)
     int32_t cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
     int32_t cls_layers_in_call[kMaxClasses];
     int32_t* advance_seq_lens;  // nullable: seq_lens to increment once every CTA has read them
     int32_t* done_counter;      // zero between launches
+    int32_t* span_counter;      // dynamic span hand-out (TMA variant), zero between launches
+    int32_t* exit_counter;      // CTAs that finished taking spans, zero between launches
 };
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
@@ -55,22 +61,38 @@ __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wa
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Work decomposition.  A unit is one (layer, request, kv head); it owns np pages of KV (the
-// pages of its Eq. 1 window segment, or of the whole history in Full mode).  All units are laid
-// end to end, layer-major then request then kv head, on one axis of P pages; the axis is cut into
-// nseg <= gridDim.x spans of equal length (+-1 page) and CTA j streams span j.  A span that
-// crosses a unit boundary yields one item per unit it touches, so every CTA reads the same number
-// of bytes whatever the mix of lengths and flags is, and the number of partials a unit has is the
-// number of spans it touches.
+// pages of its Eq. 1 window segment, or of the whole history in Full mode; requests that are not
+// flagged and layers that are not gated own none).  All units are laid end to end, layer-major
+// then request then kv head, on one axis of P pages.  The axis is cut into spans in levels.
+// With little work per CTA there is one level: span j is the j-th fair share P / gridDim.
+// Otherwise level 0 has one span per CTA of first_span_pct % of the fair share and the rest of
+// the axis is cut into short spans (tail_span_pct % of the fair share) in further levels.
+// A span that crosses a unit boundary yields one item per unit it touches; a unit touched by
+// several spans has that many partials.  The SIMT variant gives CTA c the spans c, c + grid, ...
+// (one per level); the TMA variant hands out the spans after level 0 through an atomic counter,
+// so CTAs that stream faster (the measured spread between CTAs is +-10 %) take more of the
+// short spans at the end.  On the 4.3 GB Full pass of the 32-layer benchmark the hand-out measured
+// slower than the one-level static split (692-950 us against 665 us: every short span costs a
+// partial, a fence and a ticket in the epilogue warp), so it is off by default
+// (dynamic_min_fair_pages = 2^30) and kept for experiments.
+constexpr int kMaxLevels = 16;
+
 struct Plan {  // shared memory, one per CTA
     int32_t pb[kMaxClasses][kMaxBatch + 1];  // exclusive prefix over requests of pages per kv head
     int32_t lb[kMaxLayers + 1];              // first axis page of each layer of the call
     int32_t seq[kMaxBatch];                  // seq_lens, clamped to the table capacity
     uint16_t kv_index[kMaxLayers];
     uint8_t cls[kMaxLayers];
+    uint8_t active[kMaxBatch];               // request takes part in this launch (Full mode: flagged)
+    int32_t lvl_base[kMaxLevels + 1];        // first axis page of each level
+    int32_t lvl_span0[kMaxLevels + 1];       // first span index of each level
+    int32_t lvl_size[kMaxLevels];            // span length of each level
+    int32_t nlevels;
     int32_t total_pages;
     int32_t nseg;
-    int32_t pad;  // keeps sizeof(Plan) a multiple of 8
+    int32_t pad[2];
 };
+static_assert(sizeof(Plan) % 8 == 0, "Plan is followed by 8-byte aligned barriers in shared memory");
 
 struct Item {
     int32_t layer, b, g;        // layer, request, kv head
@@ -121,19 +143,25 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     const int tid = threadIdx.x, nth = blockDim.x;
     const int B = p.batch;
     const int nl = p.layer_end - p.layer_begin;
-    for (int b = tid; b < B; b += nth) {
-        int t = p.seq_lens[b];
+    // issue every global load of the plan before using any of them: one memory latency, not three
+    const bool has_b = tid < B;  // blockDim.x >= kMaxBatch
+    const int t_raw = has_b ? p.seq_lens[tid] : 1;
+    const int fl_raw = (has_b && p.mode == 1) ? p.flags[tid] : 1;
+    LayerInfo li0, li1;
+    li0.cls = li0.kv_index = li1.cls = li1.kv_index = 0;
+    if (tid < nl) li0 = p.layers[p.layer_begin + tid];
+    if (tid + nth < nl) li1 = p.layers[p.layer_begin + tid + nth];
+    if (has_b) {
+        int t = t_raw;
         if (t > p.max_blocks_per_seq * kPage) {
             t = p.max_blocks_per_seq * kPage;
             atomicOr(p.status, kStatusBadSeqLen);
         }
-        pl.seq[b] = t;
+        pl.seq[tid] = t;
+        pl.active[tid] = fl_raw != 0;
     }
-    for (int i = tid; i < nl; i += nth) {
-        const LayerInfo li = p.layers[p.layer_begin + i];
-        pl.cls[i] = (uint8_t)li.cls;
-        pl.kv_index[i] = (uint16_t)li.kv_index;
-    }
+    if (tid < nl) { pl.cls[tid] = (uint8_t)li0.cls; pl.kv_index[tid] = (uint16_t)li0.kv_index; }
+    if (tid + nth < nl) { pl.cls[tid + nth] = (uint8_t)li1.cls; pl.kv_index[tid + nth] = (uint16_t)li1.kv_index; }
     __syncthreads();
     const int warp = tid >> 5, lane = tid & 31, nwarps = nth >> 5;
     for (int c = warp; c < p.ncls; c += nwarps) {  // one warp scans one class
@@ -141,7 +169,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         for (int b0 = 0; b0 < B; b0 += 32) {
             const int b = b0 + lane;
             int np = 0;
-            if (b < B && p.cls_layers_in_call[c] > 0 && (p.mode == 0 || (p.cls_gated[c] && p.flags[b] != 0))) {
+            if (b < B && p.cls_layers_in_call[c] > 0 && (p.mode == 0 || (p.cls_gated[c] && pl.active[b]))) {
                 const int t = pl.seq[b];
                 if (t < 1) {
                     atomicOr(p.status, kStatusBadSeqLen);
@@ -181,9 +209,36 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             }
             pl.lb[nl] = (int32_t)carry;
             pl.total_pages = (int32_t)carry;
-            long long n = (carry + p.min_span_pages - 1) / p.min_span_pages;
-            if (n > (long long)gridDim.x) n = gridDim.x;
-            pl.nseg = (int32_t)n;
+            // span levels
+            const int g = (int)gridDim.x;
+            const int P = (int)carry;
+            const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
+            const long long fair = ((long long)P + g - 1) / g;
+            // little work per CTA: one level, the whole fair share at once (nothing to gain from a
+            // hand-out whose per-span cost is comparable to the work)
+            const bool dynamic = p.span_counter != nullptr && fair >= p.dynamic_min_fair_pages;
+            int size = dynamic ? (int)((fair * p.first_span_pct + 99) / 100) : (int)fair;
+            int tail = (int)((fair * p.tail_span_pct + 99) / 100);
+            if (tail < minS) tail = minS;
+            int done = 0, spans = 0, lv = 0;
+            while (done < P) {
+                if (size < minS) size = minS;
+                int rem = P - done;
+                if (lv == kMaxLevels - 1) size = (rem + g - 1) / g;  // last level takes whatever is left
+                int n = (rem + size - 1) / size;
+                if (n > g) n = g;
+                pl.lvl_base[lv] = done;
+                pl.lvl_span0[lv] = spans;
+                pl.lvl_size[lv] = size;
+                done += (long long)n * size > rem ? rem : n * size;
+                spans += n;
+                ++lv;
+                size = tail;
+            }
+            pl.lvl_base[lv] = P;
+            pl.lvl_span0[lv] = spans;
+            pl.nlevels = lv;
+            pl.nseg = spans;
         }
     }
     __syncthreads();
@@ -211,17 +266,22 @@ __device__ __forceinline__ void prefetch_block_table(const AttnParams& p)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
 }
 
-__device__ __forceinline__ int span_begin(const Plan& pl, int j)
+__device__ __forceinline__ void span_range(const Plan& pl, int j, int& x0, int& x1)
 {
-    return (int)(((long long)j * pl.total_pages) / pl.nseg);
+    int lv = 0;
+    while (lv + 1 < pl.nlevels && pl.lvl_span0[lv + 1] <= j) ++lv;
+    x0 = pl.lvl_base[lv] + (j - pl.lvl_span0[lv]) * pl.lvl_size[lv];
+    x1 = min(x0 + pl.lvl_size[lv], pl.lvl_base[lv + 1]);
 }
 // the span that contains axis page x
 __device__ __forceinline__ int span_of(const Plan& pl, int x)
 {
-    return (int)((((long long)x + 1) * pl.nseg - 1) / pl.total_pages);
+    int lv = 0;
+    while (lv + 1 < pl.nlevels && pl.lvl_base[lv + 1] <= x) ++lv;
+    return pl.lvl_span0[lv] + (x - pl.lvl_base[lv]) / pl.lvl_size[lv];
 }
 
-// The item of span j that starts at axis page x (span_begin(j) <= x < x_end = span_begin(j+1)).
+// The item of span j that starts at axis page x (x0 <= x < x_end of span_range(j)).
 // Returns the number of axis pages it covers (>= 1).
 __device__ inline int decode_item(const AttnParams& p, const Plan& pl, int j, int x, int x_end, Item& it)
 {
@@ -308,42 +368,73 @@ __device__ __forceinline__ int take_ticket(const AttnParams& p, const Item& it)
 template <int D, int G>
 __device__ inline void merge_chunks(const AttnParams& p, const Item& it, int tid, int nth)
 {
-    constexpr int W = D + 2;
+    constexpr int W = D + kPartHdr;
+    constexpr int kBatch = 8;  // chunks whose loads are all issued before the first use
     const float kLn2 = 0.6931471805599453f;
     const float* base = p.partials + (size_t)it.slot_base * (G * W);
-    for (int e = tid; e < G * D; e += nth) {
-        int h = e / D, d = e - h * D;
-        float M = -INFINITY;
-        for (int c = 0; c < it.nchunks; ++c) M = fmaxf(M, __ldcg(base + (size_t)c * (G * W) + h * W));
-        float l = 0.f, o = 0.f;
-        for (int c = 0; c < it.nchunks; ++c) {
-            const float* pc = base + (size_t)c * (G * W) + h * W;
-            float mc = __ldcg(pc);
-            float sc = (mc == -INFINITY) ? 0.f : ex2(mc - M);
-            l += __ldcg(pc + 1) * sc;
-            o += __ldcg(pc + 2 + d) * sc;
+    for (int e = tid; e < G * (D / 4); e += nth) {
+        const int h = e / (D / 4), d = (e - h * (D / 4)) * 4;
+        float M = -INFINITY, l = 0.f;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c0 = 0; c0 < it.nchunks; c0 += kBatch) {  // chunk order is fixed: same bits every run
+            float mc[kBatch], lc[kBatch];
+            float4 oc[kBatch];
+#pragma unroll
+            for (int c = 0; c < kBatch; ++c) {
+                if (c0 + c < it.nchunks) {
+                    const float* pc = base + (size_t)(c0 + c) * (G * W) + h * W;
+                    mc[c] = __ldcg(pc);
+                    lc[c] = __ldcg(pc + 1);
+                    oc[c] = __ldcg(reinterpret_cast<const float4*>(pc + kPartHdr + d));
+                }
+            }
+            float Mn = M;
+#pragma unroll
+            for (int c = 0; c < kBatch; ++c)
+                if (c0 + c < it.nchunks) Mn = fmaxf(Mn, mc[c]);
+            const float mu = (Mn == -INFINITY) ? 0.f : Mn;
+            const float a = ex2(M - mu);  // M = -inf -> 0
+            l *= a;
+            o.x *= a; o.y *= a; o.z *= a; o.w *= a;
+            M = Mn;
+#pragma unroll
+            for (int c = 0; c < kBatch; ++c) {
+                if (c0 + c < it.nchunks) {
+                    const float sc = ex2(mc[c] - mu);
+                    l += lc[c] * sc;
+                    o.x += oc[c].x * sc; o.y += oc[c].y * sc; o.z += oc[c].z * sc; o.w += oc[c].w * sc;
+                }
+            }
         }
-        store_out<D>(p, it.layer, it.b, it.g * G + h, d, o / l);
+        const float inv = 1.f / l;
+        const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + it.g * G + h) * D + d;
+        if (p.out_bf16) {
+            __nv_bfloat162* ob = reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(p.out) + idx);
+            ob[0] = __floats2bfloat162_rn(o.x * inv, o.y * inv);
+            ob[1] = __floats2bfloat162_rn(o.z * inv, o.w * inv);
+        } else {
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + idx) =
+                make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv);
+        }
         if (d == 0 && p.lse)
-            p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + it.g * G + h] =
-                (M + log2f(l)) * kLn2;
+            p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + it.g * G + h] = (M + log2f(l)) * kLn2;
     }
 }
 
-// cta_part: [G][D+2] in shared memory holding this CTA's (m, l, o[D]) for the item; called by
-// every thread of the CTA.
+// cta_part: [G][kPartHdr + D] in shared memory holding this CTA's (m, l, -, -, o[D]) for the item;
+// called by every thread of the CTA.
 template <int D, int G>
 __device__ inline void finish_item(const AttnParams& p, const Item& it, const float* cta_part,
                                    int* s_is_last)
 {
-    constexpr int W = D + 2;
+    constexpr int W = D + kPartHdr;
     const int tid = threadIdx.x, nth = blockDim.x;
     const float kLn2 = 0.6931471805599453f;
     if (it.nchunks == 1) {
         for (int e = tid; e < G * D; e += nth) {
             int h = e / D, d = e - h * D;
             float l = cta_part[h * W + 1];
-            store_out<D>(p, it.layer, it.b, it.g * G + h, d, cta_part[h * W + 2 + d] / l);
+            store_out<D>(p, it.layer, it.b, it.g * G + h, d, cta_part[h * W + kPartHdr + d] / l);
         }
         if (p.lse && tid < G) {
             float m = cta_part[tid * W], l = cta_part[tid * W + 1];

@@ -17,7 +17,7 @@ struct SimtCfg {
     static constexpr int kLoads = kPage / kRPL;   // loads per page per tensor
     static constexpr int kBatch = (G * kLoads <= 32) ? kLoads : (32 / G);  // rows per softmax update
     static constexpr int kSubs = kWarps * kRPL;   // independent online-softmax streams per CTA
-    static constexpr int kW = D + 2;
+    static constexpr int kW = D + kPartHdr;
 };
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p)
@@ -55,10 +55,11 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
     const int sub = lane / C::kLPR;               // which row of a warp-wide load this lane reads
     const int dofs = (lane % C::kLPR) * 8;        // this lane's 8 head-dim elements
 
-    const int span = blockIdx.x;
-    if (span >= plan.nseg) return;
-    const int x_end = span_begin(plan, span + 1);
-    for (int x = span_begin(plan, span); x < x_end;) {
+    for (int span = blockIdx.x; span < plan.nseg; span += gridDim.x)
+    {
+    int x_begin, x_end;
+    span_range(plan, span, x_begin, x_end);
+    for (int x = x_begin; x < x_end;) {
         Item it;
         x += decode_item(p, plan, span, x, x_end, it);
         // q for the G heads of this kv head, pre-multiplied by scale * log2(e)
@@ -176,9 +177,11 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
             if ((lane % C::kLPR) == 0) {
                 s_sub[sidx][h][0] = m[h];
                 s_sub[sidx][h][1] = l[h];
+                s_sub[sidx][h][2] = 0.f;
+                s_sub[sidx][h][3] = 0.f;
             }
 #pragma unroll
-            for (int d = 0; d < 8; ++d) s_sub[sidx][h][2 + dofs + d] = o[h][d];
+            for (int d = 0; d < 8; ++d) s_sub[sidx][h][kPartHdr + dofs + d] = o[h][d];
         }
         __syncthreads();
         for (int e = tid; e < G * C::kW; e += C::kThreads) {
@@ -202,6 +205,7 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
         __syncthreads();
         finish_item<D, G>(p, it, &s_part[0][0], &s_is_last);
         __syncthreads();
+    }
     }
 }
 

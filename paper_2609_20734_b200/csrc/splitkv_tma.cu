@@ -1,13 +1,18 @@
 // Split-KV paged decode attention, TMA + tensor-core variant for sm_100a.
 //
-// One producer warp streams KV pages from the paged cache into a shared-memory ring with
-// tiled TMA copies (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers); four
-// consumer warps each take one 16-token page of a tile and run the GQA group tile on the
-// tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate): S = Q K^T with the group's query
-// heads in the N columns and the tokens in the M rows (S^T = K Q^T, O^T += V^T P^T, so every
-// accumulator register is live), online softmax in fp32 registers, P split into a bf16 high
-// and low part so that the softmax weights keep ~16 bits.  The work is memory bound:
-// the tensor cores are there to take the dot products off the issue slots, not for flops.
+// Six warps per CTA, two CTAs per SM, persistent:
+//  * one producer warp takes spans of the page axis (its first one statically, the rest from
+//    an atomic counter), looks up block ids a run of 32 pages ahead, and streams KV pages into a
+//    96 KiB shared-memory ring with tiled TMA copies (cp.async.bulk.tensor, 128-byte swizzle,
+//    completion on mbarriers); each item's q rows ride along with its first tile;
+//  * four consumer warps each take one 16-token page of a tile and run the GQA group tile on the
+//    tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate), transposed so that every accumulator
+//    register is live: S^T = K Q^T (tokens x heads), O^T += V^T P^T (head_dim x heads); online
+//    softmax in fp32 registers; P split into a bf16 high and low part so the weights keep ~16 bits;
+//  * one epilogue warp receives each finished item through shared memory and does everything that
+//    waits on global memory -- result store, or partial store + ticket + merge of the unit's
+//    partials -- so the consumers move straight on to the next item.
+// The work is memory bound: the tensor cores take the dot products off the issue slots.
 // Serves the Local pass (Eq. 1, S^L) and the gated Full pass (S^F) with one code path.
 #include <cuda.h>
 
@@ -27,18 +32,35 @@ extern "C" int oda_debug_timeline(unsigned long long* host, int n) { return (int
 #define ODA_TL(slot) do { } while (0)
 #endif
 
+constexpr int kMaxStages = 6;
+
+struct EpiMeta {  // what the epilogue warp needs to know about a finished item
+    int32_t layer, b, g, chunk, nchunks, slot_base, valid, pad;
+};
+
+struct Ctl {  // barriers and small hand-off slots, after the Plan in shared memory
+    uint64_t full[kMaxStages], empty[kMaxStages];
+    uint64_t efull, efree;
+    int32_t span_slot[kMaxStages];  // span id delivered with the first tile of a span (-1: no more work)
+    int32_t abort;
+    int32_t pad;
+    EpiMeta meta;
+};
+
 template <int D>
 struct TmaCfg {
     static constexpr int kConsumerWarps = 4;
-    static constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    static constexpr int kProducerWarp = 4;
+    static constexpr int kEpilogueWarp = 5;
+    static constexpr int kThreads = 6 * 32;
     static constexpr int kTilePages = 4;                    // one page per consumer warp
     static constexpr int kPageBytes = kPage * D * 2;        // one tensor, one kv head
     static constexpr int kStageBytes = 2 * kTilePages * kPageBytes;  // K and V
     static constexpr int kStages = 98304 / kStageBytes;     // 96 KiB ring
     static constexpr int kQSlotBytes = 8 * D * 2;           // q of one kv-head group (up to 8 heads)
     static constexpr int kMergeBytes = 32 * 32 * 4 + 32 * 4 * 4;  // one warp's O fragment + (m, l) of two heads per lane
-    static constexpr int kBarBytes = 2 * kStages * 8 + 16;
-    static constexpr int kSmemBytes = kStages * (kStageBytes + kQSlotBytes) + kMergeBytes + (int)sizeof(Plan) + kBarBytes;
+    static constexpr int kSmemBytes = kStages * (kStageBytes + kQSlotBytes) + kMergeBytes + (int)sizeof(Plan) + (int)sizeof(Ctl);
+    static_assert(kStages <= kMaxStages, "ring deeper than the control block");
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -175,7 +197,9 @@ struct PageRun {
     int g, kv_layer, b;
     const __nv_bfloat16* q;  // q rows of the item, copied with the first tile of the item
     int pg, n;               // first logical page, pages in the run (1..32)
+    int span;                // span the run belongs to
     bool first;              // first run of its item
+    bool span_first;         // first run of its span
 };
 
 template <int D, int G>
@@ -190,10 +214,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     float* mbuf = reinterpret_cast<float*>(qring + C::kStages * C::kQSlotBytes);  // [32][32]
     float* mlbuf = mbuf + 32 * 32;                                        // [32][4]
     Plan& plan = *reinterpret_cast<Plan*>(mlbuf + 32 * 4);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(&plan) + sizeof(Plan));
-    int* s_flags = reinterpret_cast<int*>(bars + 2 * C::kStages);         // [0] abort, [1] is_last
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + C::kStages);
-    static_assert(sizeof(Plan) % 8 == 0, "barriers must stay 8-byte aligned");
+    Ctl& ctl = *reinterpret_cast<Ctl*>(reinterpret_cast<uint8_t*>(&plan) + sizeof(Plan));
+    const uint32_t full0 = smem_u32(ctl.full), empty0 = smem_u32(ctl.empty);
+    const uint32_t efull = smem_u32(&ctl.efull), efree = smem_u32(&ctl.efree);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) ODA_TL(0);
@@ -202,8 +225,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, C::kConsumerWarps);
         }
-        s_flags[0] = 0;
-        s_flags[1] = 0;
+        mbar_init(efull, 1);
+        mbar_init(efree, 1);
+        ctl.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&kmap)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&vmap)) : "memory");
@@ -214,32 +238,44 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     build_plan(p, plan);  // ends with a barrier
     griddep_launch_dependents();
     if (tid == 0) ODA_TL(2);
-    volatile int* abort_flag = s_flags;
-    const int span = blockIdx.x;
-    if (span >= plan.nseg) return;
-    const int x0 = span_begin(plan, span), x_end = span_begin(plan, span + 1);
+    volatile int* abort_flag = &ctl.abort;
     constexpr uint32_t kQBytes = G * D * 2;
 
-    if (warp == C::kConsumerWarps) {
+    if (warp == C::kProducerWarp) {
         // ============================ producer warp ============================
         const uint64_t policy = 0x12F0000000000000ull;  // L2 evict-first: the KV stream is read once
         uint32_t cnt = 0;
-        // walker over the runs of the span
-        int x = x0, take = 0, seg = 0, pg = 0;
+        bool dead = false;
+        // Walker over the runs of all the spans this CTA takes.  The first span is the CTA's own;
+        // every further one comes from the counter, asked for one span ahead so that the answer
+        // is there when the current span runs out and the stream of copies never pauses.
+        int span = (int)blockIdx.x < plan.nseg ? (int)blockIdx.x : -1;
+        int pending = 0;   // lane 0: span id requested from the counter, not yet used
+        int x = 0, x_end = 0, take = 0, seg = 0, pg = 0;
         Item it;
-        bool more = true, item_first = true;
-        take = decode_item(p, plan, span, x, x_end, it);
-        seg = it.sink_pg1 > 0 ? 0 : 1;
-        pg = seg ? it.win_pg0 : 0;
-        auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when the span is done
-            if (!more) return false;
+        bool item_first = true, span_first = true;
+        auto open_span = [&]() {  // span >= 0: position the walker on its first item and ask for the next span
+            if (lane == 0) pending = atomicAdd(p.span_counter, 1) + (int)gridDim.x;
+            span_range(plan, span, x, x_end);
+            take = decode_item(p, plan, span, x, x_end, it);
+            seg = it.sink_pg1 > 0 ? 0 : 1;
+            pg = seg ? it.win_pg0 : 0;
+            item_first = true;
+            span_first = true;
+        };
+        if (span >= 0) open_span();
+        auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when there is no more work
+            if (span < 0) return false;
             const int end = seg ? it.win_pg1 : it.sink_pg1;
             r.g = it.g; r.kv_layer = it.kv_layer; r.b = it.b;
             r.q = p.q + (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + (size_t)it.g * G) * D;
             r.pg = pg;
             r.n = min(32, end - pg);
+            r.span = span;
             r.first = item_first;
+            r.span_first = span_first;
             item_first = false;
+            span_first = false;
             blk = lane < r.n ? __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + pg + lane) : 0;
             pg += r.n;
             if (pg >= end) {
@@ -254,7 +290,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                         pg = seg ? it.win_pg0 : 0;
                         item_first = true;
                     } else {
-                        more = false;
+                        const int nx = __shfl_sync(0xffffffffu, pending, 0);
+                        span = nx < plan.nseg ? nx : -1;
+                        if (span >= 0) open_span();
                     }
                 }
             }
@@ -263,7 +301,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         PageRun cur, nxt;
         int blk_cur = 0, blk_nxt = 0;
         bool have = fetch(cur, blk_cur);
-        bool dead = false;
         while (have && !dead) {
             const bool have_next = fetch(nxt, blk_nxt);  // block ids of the next run are in flight during this one
             for (int t0 = 0; t0 < cur.n; t0 += 4) {
@@ -272,8 +309,10 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { dead = true; break; }
                 const bool with_q = cur.first && t0 == 0;
                 if (cnt == 0) ODA_TL(3);
-                if (lane == 0)
+                if (lane == 0) {
+                    if (cur.span_first && t0 == 0) ctl.span_slot[s] = cur.span;  // ordered before the arrive below
                     mbar_expect_tx(full0 + 8 * s, (uint32_t)np * 2 * C::kPageBytes + (with_q ? kQBytes : 0u));
+                }
                 __syncwarp();
                 const int blk = __shfl_sync(0xffffffffu, blk_cur, t0 + (lane & 3));
                 if (lane < np) {
@@ -291,15 +330,113 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             blk_cur = blk_nxt;
             have = have_next;
         }
+        if (!dead) {  // tell the consumers that nothing more will come
+            const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
+            if (mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) {
+                if (lane == 0) {
+                    ctl.span_slot[s] = -1;
+                    mbar_arrive(full0 + 8 * s);
+                }
+                ++cnt;
+            }
+        }
+        // This CTA will not touch the span counter again: the CTA that notes this last re-arms
+        // both counters for the next launch.
+        if (lane == 0) {
+            __threadfence();
+            const int old = atomicAdd(p.exit_counter, 1);
+            if (old == (int)gridDim.x - 1) {
+                *p.span_counter = 0;
+                *p.exit_counter = 0;
+            }
+        }
         // Do not leave while copies may still be landing in this CTA's shared memory: wait
         // (bounded) until the consumers have released every stage that was armed.
-        for (uint32_t k = 0; k < (uint32_t)C::kStages && k < cnt; ++k) {
-            const uint32_t c2 = cnt - 1 - k;
+        for (uint32_t k = 1; k < (uint32_t)C::kStages + 1 && k < cnt; ++k) {
+            const uint32_t c2 = cnt - 1 - k;  // (the last count is the end marker, which carries no copy)
             const uint32_t s = c2 % C::kStages, ph = (c2 / C::kStages) & 1;
             if (!mbar_wait(empty0 + 8 * s, ph, abort_flag, p.status)) break;
         }
         if (*abort_flag) {  // abandoned waits: give in-flight copies time to land before the CTA retires
             for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        }
+        return;
+    }
+
+    if (warp == C::kEpilogueWarp) {
+        // ============================ epilogue warp ============================
+        // Fragment layout of the item it receives (same as the consumers' accumulators):
+        // o[n][0..1]: d = 16n + hrow, heads qc, qc+1;  o[n][2..3]: d = 16n + 8 + hrow.
+        const int hrow = lane >> 2, qc = (lane & 3) * 2;
+        constexpr int W = D + kPartHdr;
+        const float kLn2 = 0.6931471805599453f;
+        for (uint32_t k = 0;; ++k) {
+            if (!mbar_wait(efull, k & 1, abort_flag, p.status)) break;
+            const EpiMeta m = ctl.meta;
+            if (!m.valid) break;
+            float o[D / 16][4];
+#pragma unroll
+            for (int n = 0; n < D / 16; ++n) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) o[n][e] = mbuf[(4 * n + e) * 32 + lane];
+            }
+            const float4 ml = reinterpret_cast<const float4*>(mlbuf)[lane];  // mA, lA, mB, lB
+            __syncwarp();
+            if (lane == 0) mbar_arrive(efree);  // the consumers may reuse the hand-off buffer
+            Item it;
+            it.layer = m.layer; it.b = m.b; it.g = m.g; it.chunk = m.chunk; it.nchunks = m.nchunks;
+            it.slot_base = m.slot_base;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int hg = qc + e;
+                if (hg >= G) continue;
+                const float mm = e ? ml.z : ml.x, ll = e ? ml.w : ml.y;
+                if (it.nchunks == 1) {
+                    const float inv = 1.f / ll;
+                    const int h = it.g * G + hg;
+                    const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + hrow;
+                    if (p.out_bf16) {
+                        __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) + idx;
+#pragma unroll
+                        for (int n = 0; n < D / 16; ++n) {
+                            ob[n * 16] = __float2bfloat16_rn(o[n][e] * inv);
+                            ob[n * 16 + 8] = __float2bfloat16_rn(o[n][2 + e] * inv);
+                        }
+                    } else {
+                        float* of = reinterpret_cast<float*>(p.out) + idx;
+#pragma unroll
+                        for (int n = 0; n < D / 16; ++n) {
+                            of[n * 16] = o[n][e] * inv;
+                            of[n * 16 + 8] = o[n][2 + e] * inv;
+                        }
+                    }
+                    if (p.lse && hrow == 0)
+                        p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] = (mm + log2f(ll)) * kLn2;
+                } else {
+                    float* slot = partial_slot(p, it, G, W) + hg * W;
+                    if (hrow == 0) {
+                        __stcg(slot, mm);
+                        __stcg(slot + 1, ll);
+                    }
+#pragma unroll
+                    for (int n = 0; n < D / 16; ++n) {
+                        __stcg(slot + kPartHdr + n * 16 + hrow, o[n][e]);
+                        __stcg(slot + kPartHdr + n * 16 + 8 + hrow, o[n][2 + e]);
+                    }
+                }
+            }
+            if (it.nchunks > 1) {
+                __threadfence();
+                __syncwarp();
+                int last = 0;
+                if (lane == 0) last = take_ticket(p, it);
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    __threadfence();
+                    merge_chunks<D, G>(p, it, lane, 32);
+                }
+            }
+            ODA_TL(6);
         }
         return;
     }
@@ -315,213 +452,191 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     const int k_tok = (lane & 7) + (((lane >> 3) & 1) << 3), k_half = lane >> 4;
     const int v_tok = (lane & 7) + ((lane >> 4) << 3), v_sel = (lane >> 3) & 1;
     const int xr = lane & 7;
-    uint32_t cnt = 0;
+    uint32_t cnt = 0;    // tiles consumed
+    uint32_t ecnt = 0;   // items handed to the epilogue warp
+    bool aborted = false;
 
-    for (int x = x0; x < x_end;) {
-        Item it;
-        x += decode_item(p, plan, span, x, x_end, it);
-        // Q^T fragments come with the item's first tile; heads >= G stay zero
-        uint32_t qa[D / 16][2];
-        {
+    while (!aborted) {
+        int span;
+        {   // the first tile of a span carries the span id
             const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
-            if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) break;
-            if (cnt == 0 && warp == 0) ODA_TL(4);
-            const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
-#pragma unroll
-            for (int kc = 0; kc < D / 16; ++kc) {
-                qa[kc][0] = hrow < G ? qs[kc * 8] : 0u;
-                qa[kc][1] = hrow < G ? qs[kc * 8 + 4] : 0u;
-            }
-        }
-        float o[D / 16][4];
-#pragma unroll
-        for (int n = 0; n < D / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-        float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;  // heads qc and qc+1
-
-        TileWalk tw;
-        bool aborted = false;
-        for (tw.start(it); !tw.done(); tw.next(it)) {
-            const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
-            ++cnt;
             if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
-            if (warp < tw.npages) {
-                const int pos0 = (tw.pg + warp) * kPage;
-                const int vlo = tw.seg ? it.win_lo : 0, vhi = tw.seg ? it.win_hi : it.sink_hi;
-                const bool edge = pos0 < vlo || pos0 + kPage > vhi;
-                const uint32_t kpage = smem_u32(ring + s * C::kStageBytes + warp * C::kPageBytes);
-                const uint32_t vpage = kpage + C::kTilePages * C::kPageBytes;
-                // ---- S^T = K Q^T for 16 tokens ----
-                float st[4] = {0.f, 0.f, 0.f, 0.f};
+            span = ctl.span_slot[s];
+        }
+        if (span < 0) break;
+        int x, x_end;
+        span_range(plan, span, x, x_end);
+        while (x < x_end && !aborted) {
+            Item it;
+            x += decode_item(p, plan, span, x, x_end, it);
+            // Q^T fragments come with the item's first tile; heads >= G stay zero
+            uint32_t qa[D / 16][2];
+            {
+                const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
+                if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
+                if (cnt == 0 && warp == 0) ODA_TL(4);
+                const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
 #pragma unroll
                 for (int kc = 0; kc < D / 16; ++kc) {
-                    const int chunk = (kc & 3) * 2 + k_half;
-                    const uint32_t addr = kpage + (kc >> 2) * 2048 + k_tok * 128 + ((chunk ^ xr) << 4);
-                    uint32_t a0, a1, a2, a3;
-                    ldsm_x4(addr, a0, a1, a2, a3);
-                    mma16816(st, a0, a1, a2, a3, qa[kc][0], qa[kc][1]);
-                }
-                // st[0],st[1]: token hrow, heads qc,qc+1;  st[2],st[3]: token hrow+8
-                float x0s = st[0] * p.scale_log2e, x1s = st[1] * p.scale_log2e;
-                float x2s = st[2] * p.scale_log2e, x3s = st[3] * p.scale_log2e;
-                uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
-                if (edge) {  // positions outside [vlo, vhi) are not in the set
-                    const int ta = pos0 + hrow;
-                    const bool va = ta >= vlo && ta < vhi, vb = ta + 8 >= vlo && ta + 8 < vhi;
-                    x0s = va ? x0s : -INFINITY; x1s = va ? x1s : -INFINITY;
-                    x2s = vb ? x2s : -INFINITY; x3s = vb ? x3s : -INFINITY;
-                    // V^T fragments hold tokens qc, qc+1 (and +8) in their 16-bit halves
-                    const int t0 = pos0 + qc;
-                    const bool v0 = t0 >= vlo && t0 < vhi, v1 = t0 + 1 >= vlo && t0 + 1 < vhi;
-                    const bool v2 = t0 + 8 >= vlo && t0 + 8 < vhi, v3 = t0 + 9 >= vlo && t0 + 9 < vhi;
-                    mk0 = (v0 ? 0x0000ffffu : 0u) | (v1 ? 0xffff0000u : 0u);
-                    mk1 = (v2 ? 0x0000ffffu : 0u) | (v3 ? 0xffff0000u : 0u);
-                }
-                // ---- online softmax over the 16 tokens (fp32, base 2); tokens live across lanes ----
-                float mxA = fmaxf(x0s, x2s), mxB = fmaxf(x1s, x3s);
-#pragma unroll
-                for (int off = 4; off < 32; off <<= 1) {
-                    mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, off));
-                    mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, off));
-                }
-                const float mnA = fmaxf(mA, mxA), mnB = fmaxf(mB, mxB);
-                const float muA = (mnA == -INFINITY) ? 0.f : mnA, muB = (mnB == -INFINITY) ? 0.f : mnB;
-                const float alA = ex2(mA - muA), alB = ex2(mB - muB);
-                const float p0 = ex2(x0s - muA), p1 = ex2(x1s - muB), p2 = ex2(x2s - muA), p3 = ex2(x3s - muB);
-                lA = lA * alA + (p0 + p2);
-                lB = lB * alB + (p1 + p3);
-                mA = mnA;
-                mB = mnB;
-                if (!__all_sync(0xffffffffu, alA == 1.f && alB == 1.f)) {
-#pragma unroll
-                    for (int n = 0; n < D / 16; ++n) { o[n][0] *= alA; o[n][1] *= alB; o[n][2] *= alA; o[n][3] *= alB; }
-                }
-                // P^T as B fragments: transpose the two 8x8 (token x head) tiles; bf16 high + low parts
-                const uint32_t hi0 = pack_bf16x2(p0, p1), hi1 = pack_bf16x2(p2, p3);
-                const uint32_t lo0 = pack_bf16x2(p0 - __uint_as_float(hi0 << 16), p1 - __uint_as_float(hi0 & 0xffff0000u));
-                const uint32_t lo1 = pack_bf16x2(p2 - __uint_as_float(hi1 << 16), p3 - __uint_as_float(hi1 & 0xffff0000u));
-                const uint32_t bh0 = movmatrix_t(hi0), bh1 = movmatrix_t(hi1);
-                const uint32_t bl0 = movmatrix_t(lo0), bl1 = movmatrix_t(lo1);
-                // ---- O^T += V^T P^T ----
-#pragma unroll
-                for (int mt = 0; mt < D / 16; ++mt) {
-                    const int chunk = (mt & 3) * 2 + v_sel;
-                    const uint32_t addr = vpage + (mt >> 2) * 2048 + v_tok * 128 + ((chunk ^ xr) << 4);
-                    uint32_t a0, a1, a2, a3;
-                    ldsm_x4_t(addr, a0, a1, a2, a3);
-                    if (edge) {  // slots outside the set may hold anything, NaN bit patterns included
-                        a0 &= mk0; a1 &= mk0; a2 &= mk1; a3 &= mk1;
-                    }
-                    mma16816(o[mt], a0, a1, a2, a3, bh0, bh1);
-                    mma16816(o[mt], a0, a1, a2, a3, bl0, bl1);
+                    qa[kc][0] = hrow < G ? qs[kc * 8] : 0u;
+                    qa[kc][1] = hrow < G ? qs[kc * 8 + 4] : 0u;
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * s);
-        }
-        if (aborted || *abort_flag) break;
-        if (warp == 0) ODA_TL(5);
-
-        // ---- fold warps 1..3 into warp 0 through shared memory (all use the same fragment layout) ----
+            float o[D / 16][4];
 #pragma unroll
-        for (int off = 4; off < 32; off <<= 1) {
-            lA += __shfl_xor_sync(0xffffffffu, lA, off);
-            lB += __shfl_xor_sync(0xffffffffu, lB, off);
-        }
+            for (int n = 0; n < D / 16; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+            float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;  // heads qc and qc+1
+
+            TileWalk tw;
+            for (tw.start(it); !tw.done(); tw.next(it)) {
+                const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
+                ++cnt;
+                if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
+                if (warp < tw.npages) {
+                    const int pos0 = (tw.pg + warp) * kPage;
+                    const int vlo = tw.seg ? it.win_lo : 0, vhi = tw.seg ? it.win_hi : it.sink_hi;
+                    const bool edge = pos0 < vlo || pos0 + kPage > vhi;
+                    const uint32_t kpage = smem_u32(ring + s * C::kStageBytes + warp * C::kPageBytes);
+                    const uint32_t vpage = kpage + C::kTilePages * C::kPageBytes;
+                    // ---- S^T = K Q^T for 16 tokens ----
+                    float st[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int kc = 0; kc < D / 16; ++kc) {
+                        const int chunk = (kc & 3) * 2 + k_half;
+                        const uint32_t addr = kpage + (kc >> 2) * 2048 + k_tok * 128 + ((chunk ^ xr) << 4);
+                        uint32_t a0, a1, a2, a3;
+                        ldsm_x4(addr, a0, a1, a2, a3);
+                        mma16816(st, a0, a1, a2, a3, qa[kc][0], qa[kc][1]);
+                    }
+                    // st[0],st[1]: token hrow, heads qc,qc+1;  st[2],st[3]: token hrow+8
+                    float x0s = st[0] * p.scale_log2e, x1s = st[1] * p.scale_log2e;
+                    float x2s = st[2] * p.scale_log2e, x3s = st[3] * p.scale_log2e;
+                    uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
+                    if (edge) {  // positions outside [vlo, vhi) are not in the set
+                        const int ta = pos0 + hrow;
+                        const bool va = ta >= vlo && ta < vhi, vb = ta + 8 >= vlo && ta + 8 < vhi;
+                        x0s = va ? x0s : -INFINITY; x1s = va ? x1s : -INFINITY;
+                        x2s = vb ? x2s : -INFINITY; x3s = vb ? x3s : -INFINITY;
+                        // V^T fragments hold tokens qc, qc+1 (and +8) in their 16-bit halves
+                        const int t0 = pos0 + qc;
+                        const bool v0 = t0 >= vlo && t0 < vhi, v1 = t0 + 1 >= vlo && t0 + 1 < vhi;
+                        const bool v2 = t0 + 8 >= vlo && t0 + 8 < vhi, v3 = t0 + 9 >= vlo && t0 + 9 < vhi;
+                        mk0 = (v0 ? 0x0000ffffu : 0u) | (v1 ? 0xffff0000u : 0u);
+                        mk1 = (v2 ? 0x0000ffffu : 0u) | (v3 ? 0xffff0000u : 0u);
+                    }
+                    // ---- online softmax over the 16 tokens (fp32, base 2); tokens live across lanes ----
+                    float mxA = fmaxf(x0s, x2s), mxB = fmaxf(x1s, x3s);
+#pragma unroll
+                    for (int off = 4; off < 32; off <<= 1) {
+                        mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, off));
+                        mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, off));
+                    }
+                    const float mnA = fmaxf(mA, mxA), mnB = fmaxf(mB, mxB);
+                    const float muA = (mnA == -INFINITY) ? 0.f : mnA, muB = (mnB == -INFINITY) ? 0.f : mnB;
+                    const float alA = ex2(mA - muA), alB = ex2(mB - muB);
+                    const float p0 = ex2(x0s - muA), p1 = ex2(x1s - muB), p2 = ex2(x2s - muA), p3 = ex2(x3s - muB);
+                    lA = lA * alA + (p0 + p2);
+                    lB = lB * alB + (p1 + p3);
+                    mA = mnA;
+                    mB = mnB;
+                    if (!__all_sync(0xffffffffu, alA == 1.f && alB == 1.f)) {
+#pragma unroll
+                        for (int n = 0; n < D / 16; ++n) { o[n][0] *= alA; o[n][1] *= alB; o[n][2] *= alA; o[n][3] *= alB; }
+                    }
+                    // P^T as B fragments: transpose the two 8x8 (token x head) tiles; bf16 high + low parts
+                    const uint32_t hi0 = pack_bf16x2(p0, p1), hi1 = pack_bf16x2(p2, p3);
+                    const uint32_t lo0 = pack_bf16x2(p0 - __uint_as_float(hi0 << 16), p1 - __uint_as_float(hi0 & 0xffff0000u));
+                    const uint32_t lo1 = pack_bf16x2(p2 - __uint_as_float(hi1 << 16), p3 - __uint_as_float(hi1 & 0xffff0000u));
+                    const uint32_t bh0 = movmatrix_t(hi0), bh1 = movmatrix_t(hi1);
+                    const uint32_t bl0 = movmatrix_t(lo0), bl1 = movmatrix_t(lo1);
+                    // ---- O^T += V^T P^T ----
+#pragma unroll
+                    for (int mt = 0; mt < D / 16; ++mt) {
+                        const int chunk = (mt & 3) * 2 + v_sel;
+                        const uint32_t addr = vpage + (mt >> 2) * 2048 + v_tok * 128 + ((chunk ^ xr) << 4);
+                        uint32_t a0, a1, a2, a3;
+                        ldsm_x4_t(addr, a0, a1, a2, a3);
+                        if (edge) {  // slots outside the set may hold anything, NaN bit patterns included
+                            a0 &= mk0; a1 &= mk0; a2 &= mk1; a3 &= mk1;
+                        }
+                        mma16816(o[mt], a0, a1, a2, a3, bh0, bh1);
+                        mma16816(o[mt], a0, a1, a2, a3, bl0, bl1);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * s);
+            }
+            if (aborted || *abort_flag) { aborted = true; break; }
+            if (warp == 0) ODA_TL(5);
+
+            // ---- fold warps 1..3 into warp 0 through shared memory (all use the same fragment
+            //      layout), then leave the item to the epilogue warp ----
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                lA += __shfl_xor_sync(0xffffffffu, lA, off);
+                lB += __shfl_xor_sync(0xffffffffu, lB, off);
+            }
+            // the hand-off buffer doubles as the merge buffer: wait until the epilogue warp has
+            // taken the previous item out of it
+            if (!mbar_wait(efree, (ecnt & 1) ^ 1, abort_flag, p.status)) { aborted = true; break; }
 #pragma unroll 1
-        for (int src_warp = 1; src_warp < C::kConsumerWarps; ++src_warp) {
-            if (warp == src_warp) {
+            for (int src_warp = 1; src_warp < C::kConsumerWarps; ++src_warp) {
+                if (warp == src_warp) {
+#pragma unroll
+                    for (int n = 0; n < D / 16; ++n) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) mbuf[(4 * n + e) * 32 + lane] = o[n][e];
+                    }
+                    reinterpret_cast<float4*>(mlbuf)[lane] = make_float4(mA, lA, mB, lB);
+                }
+                consumer_sync();
+                if (warp == 0) {
+                    const float4 ml = reinterpret_cast<const float4*>(mlbuf)[lane];
+                    const float MA = fmaxf(mA, ml.x), MB = fmaxf(mB, ml.z);
+                    const float muA = (MA == -INFINITY) ? 0.f : MA, muB = (MB == -INFINITY) ? 0.f : MB;
+                    const float saA = ex2(mA - muA), sbA = ex2(ml.x - muA);
+                    const float saB = ex2(mB - muB), sbB = ex2(ml.z - muB);
+#pragma unroll
+                    for (int n = 0; n < D / 16; ++n) {
+                        o[n][0] = o[n][0] * saA + mbuf[(4 * n + 0) * 32 + lane] * sbA;
+                        o[n][1] = o[n][1] * saB + mbuf[(4 * n + 1) * 32 + lane] * sbB;
+                        o[n][2] = o[n][2] * saA + mbuf[(4 * n + 2) * 32 + lane] * sbA;
+                        o[n][3] = o[n][3] * saB + mbuf[(4 * n + 3) * 32 + lane] * sbB;
+                    }
+                    lA = lA * saA + ml.y * sbA;
+                    lB = lB * saB + ml.w * sbB;
+                    mA = MA;
+                    mB = MB;
+                }
+                consumer_sync();
+            }
+            if (warp == 0) {
 #pragma unroll
                 for (int n = 0; n < D / 16; ++n) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) mbuf[(4 * n + e) * 32 + lane] = o[n][e];
                 }
                 reinterpret_cast<float4*>(mlbuf)[lane] = make_float4(mA, lA, mB, lB);
-            }
-            consumer_sync();
-            if (warp == 0) {
-                const float4 ml = reinterpret_cast<const float4*>(mlbuf)[lane];
-                const float MA = fmaxf(mA, ml.x), MB = fmaxf(mB, ml.z);
-                const float muA = (MA == -INFINITY) ? 0.f : MA, muB = (MB == -INFINITY) ? 0.f : MB;
-                const float saA = ex2(mA - muA), sbA = ex2(ml.x - muA);
-                const float saB = ex2(mB - muB), sbB = ex2(ml.z - muB);
-#pragma unroll
-                for (int n = 0; n < D / 16; ++n) {
-                    o[n][0] = o[n][0] * saA + mbuf[(4 * n + 0) * 32 + lane] * sbA;
-                    o[n][1] = o[n][1] * saB + mbuf[(4 * n + 1) * 32 + lane] * sbB;
-                    o[n][2] = o[n][2] * saA + mbuf[(4 * n + 2) * 32 + lane] * sbA;
-                    o[n][3] = o[n][3] * saB + mbuf[(4 * n + 3) * 32 + lane] * sbB;
+                if (lane == 0) {
+                    EpiMeta m;
+                    m.layer = it.layer; m.b = it.b; m.g = it.g; m.chunk = it.chunk; m.nchunks = it.nchunks;
+                    m.slot_base = it.slot_base; m.valid = 1; m.pad = 0;
+                    ctl.meta = m;
                 }
-                lA = lA * saA + ml.y * sbA;
-                lB = lB * saB + ml.w * sbB;
-                mA = MA;
-                mB = MB;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(efull);
             }
-            consumer_sync();
+            ++ecnt;
         }
-        // ---- warp 0 holds the CTA's (m, l, o): store the result or publish the partial ----
-        // o[n][0..1]: d = 16n + hrow, heads qc, qc+1;  o[n][2..3]: d = 16n + 8 + hrow
-        constexpr int W = D + 2;
-        const float kLn2 = 0.6931471805599453f;
-        if (it.nchunks == 1) {
-            if (warp == 0) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int hg = qc + e;
-                    if (hg < G) {
-                        const float inv = 1.f / (e ? lB : lA);
-                        const int h = it.g * G + hg;
-                        const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + hrow;
-                        if (p.out_bf16) {
-                            __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) + idx;
-#pragma unroll
-                            for (int n = 0; n < D / 16; ++n) {
-                                ob[n * 16] = __float2bfloat16_rn(o[n][e] * inv);
-                                ob[n * 16 + 8] = __float2bfloat16_rn(o[n][2 + e] * inv);
-                            }
-                        } else {
-                            float* of = reinterpret_cast<float*>(p.out) + idx;
-#pragma unroll
-                            for (int n = 0; n < D / 16; ++n) {
-                                of[n * 16] = o[n][e] * inv;
-                                of[n * 16 + 8] = o[n][2 + e] * inv;
-                            }
-                        }
-                        if (p.lse && hrow == 0)
-                            p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] =
-                                ((e ? mB : mA) + log2f(e ? lB : lA)) * kLn2;
-                    }
-                }
+    }
+    // end marker for the epilogue warp (also on the abort path, where its own waits are bounded)
+    if (warp == 0) {
+        if (mbar_wait(efree, (ecnt & 1) ^ 1, abort_flag, p.status)) {
+            if (lane == 0) {
+                ctl.meta.valid = 0;
+                mbar_arrive(efull);
             }
-        } else {
-            if (warp == 0) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int hg = qc + e;
-                    if (hg < G) {
-                        float* slot = partial_slot(p, it, G, W) + hg * W;
-                        if (hrow == 0) {
-                            __stcg(slot, e ? mB : mA);
-                            __stcg(slot + 1, e ? lB : lA);
-                        }
-#pragma unroll
-                        for (int n = 0; n < D / 16; ++n) {
-                            __stcg(slot + 2 + n * 16 + hrow, o[n][e]);
-                            __stcg(slot + 2 + n * 16 + 8 + hrow, o[n][2 + e]);
-                        }
-                    }
-                }
-            }
-            __threadfence();
-            consumer_sync();
-            if (tid == 0) s_flags[1] = take_ticket(p, it);
-            consumer_sync();
-            if (s_flags[1]) {
-                __threadfence();
-                merge_chunks<D, G>(p, it, tid, C::kConsumerWarps * 32);
-            }
-            consumer_sync();  // s_flags[1] is reused by the next item
         }
-        if (warp == 0) ODA_TL(6);
     }
 }
 
