@@ -300,16 +300,27 @@ def main():
         ones = torch.ones(B, dtype=torch.uint8, device="cuda")
         st.seq_lens.copy_(seq0)
         kt = {"local": [], "full": []}
+        # each launch is captured in a graph of its own, so that the events time the kernel and
+        # not the host's launch path
+        kgraphs = {}
+        for name in ("local", "full"):
+            gk = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(gk, stream=side):
+                    if name == "local":
+                        ctx.local_decode(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table, st.seq_lens,
+                                         out, lse, stream=side.cuda_stream)
+                    else:
+                        ctx.full_decode_gated(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table,
+                                              st.seq_lens, ones, out, lse, stream=side.cuda_stream)
+            kgraphs[name] = gk
+        torch.cuda.synchronize()
         for r in range(reps + 2):
             for name in ("local", "full"):
                 flush.fill_(r)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                if name == "local":
-                    ctx.local_decode(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, lse)
-                else:
-                    ctx.full_decode_gated(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table,
-                                          st.seq_lens, ones, out, lse)
+                kgraphs[name].replay()
                 e1.record()
                 torch.cuda.synchronize()
                 if r >= 2:
