@@ -42,10 +42,15 @@ def parse():
     ap.add_argument("--recall-rate", type=float, default=0.25)
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 SIMT, 2 TMA+MMA")
     ap.add_argument("--sinks", type=int, default=None)
+    ap.add_argument("--phys-layers", type=int, default=0,
+                    help="alias the layers onto this many physical cache slices (bounds memory for the large "
+                         "configs); -1 = one slice per layer")
+    ap.add_argument("--context", type=int, default=0, help="override every request's context length")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--kernel-reps", type=int, default=10)
+    ap.add_argument("--no-calibrate", action="store_true", help="keep the equal split of work across CTAs")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the Local and the all-flagged Full attention launches (for ncu captures)")
     return ap.parse_args()
@@ -175,6 +180,12 @@ def main():
     if args.sinks is not None:
         wl.sinks = [args.sinks if g else s for g, s in zip(wl.gated, wl.sinks)]
     wl.steps = args.steps + args.warmup + 1
+    if args.phys_layers > 0:
+        wl.kv_index = [l % args.phys_layers for l in range(wl.L)]
+    elif args.phys_layers < 0:
+        wl.kv_index = None
+    if args.context > 0:
+        wl.seq_lens0 = np.full(wl.B, args.context, np.int32)
     if args.impl == "reference":
         reference_arm(args, wl)
         return
@@ -221,6 +232,14 @@ def main():
     step_args = ctx.step_args(B, q_s, st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, scores,
                               flags, feat_ext=fe_s, head=st.head, threshold=wl.threshold,
                               override_flags=ov_s, lse=lse, counters=counters, advance_seq_lens=True)
+    calib = 0.0
+    if not args.no_calibrate:  # set-up, once: per-SM streaming rates measured on two all-flagged Full passes
+        ctx.calibration_begin()
+        for _ in range(2):
+            ctx.full_decode_gated(0, L, B, qs[0], st.k_cache, st.v_cache, st.block_table, st.seq_lens,
+                                  torch.ones(B, dtype=torch.uint8, device="cuda"), out, lse)
+        calib = ctx.calibration_end()
+
     # capture one step; every replay reads lengths and flags on the device
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -291,6 +310,7 @@ def main():
             "step_gbs": step_bytes / (total_ms / args.steps * 1e-3) / 1e9,
             "variant": {1: "simt", 2: "tma_mma"}.get(ctx.variant, str(ctx.variant)),
             "attention_grid": ctx.attention_grid,
+            "sm_bandwidth_calibration": {"applied": calib > 0, "slowest_over_fastest_sm": calib},
             "wall_s_timed_region_incl_flush": t_wall}
 
     if rank == 0:

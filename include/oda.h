@@ -107,6 +107,23 @@ oda_status_t oda_workspace_bytes(const oda_ctx_t* ctx, size_t* bytes);
 oda_status_t oda_set_workspace(oda_ctx_t* ctx, void* dev_ptr, size_t bytes, void* stream);
 
 /*
+ * Optional calibration of the split of work across SMs.  HBM bandwidth is not shared evenly among
+ * the SMs of a GPU (on a B200, equal spans of KV finish +-10 % apart, in a pattern that is a fixed
+ * property of the chip).  Between oda_calibration_begin() and oda_calibration_end() the attention
+ * kernels record, per SM, how many pages they streamed in how much time; run one or more large
+ * passes in between (e.g. one oda_full_decode_gated with every request flagged: only launches
+ * that give every CTA work are counted).  oda_calibration_end() synchronises the stream, and from
+ * then on cuts the work of large attention launches in proportion to the measured rate of the SM
+ * each CTA runs on, so that all CTAs finish together.  Results stay deterministic (the table is
+ * fixed once measured) and agree with the uncalibrated ones up to summation order.  Has no effect
+ * for the SIMT variant.  oda_set_workspace() discards the table.  Do not capture these two calls.
+ */
+oda_status_t oda_calibration_begin(oda_ctx_t* ctx, void* stream);
+oda_status_t oda_calibration_end(oda_ctx_t* ctx, void* stream);
+/* slowest / fastest SM streaming rate found by the calibration (0 if not calibrated) */
+double oda_calibration_spread(const oda_ctx_t* ctx);
+
+/*
  * Local pass (Eq. 1, S^L) for layers [layer_begin, layer_end) and requests 0..batch-1:
  * split-KV partials + log-sum-exp merge.  Writes out/lse rows of those layers.
  * lse may be NULL.  batch = 0 is a no-op.

@@ -23,6 +23,7 @@ EXPORTS = [
     "oda_recall_score", "oda_full_decode_gated", "oda_step", "oda_step_host",
     "oda_read_device_status", "oda_launch_count", "oda_resolved_variant", "oda_attention_grid",
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
+    "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
 ]
 
 
@@ -88,6 +89,10 @@ def load_library():
         lib.oda_local_decode_static.argtypes = [i32, i32, i32, i32, i32, i32, f32, ctypes.c_int64,
                                                 ctypes.c_int64, ctypes.c_int64, i32, vp, vp, vp, vp, vp,
                                                 vp, vp, vp]
+        lib.oda_calibration_begin.argtypes = [vp, vp]
+        lib.oda_calibration_end.argtypes = [vp, vp]
+        lib.oda_calibration_spread.argtypes = [vp]
+        lib.oda_calibration_spread.restype = ctypes.c_double
         lib.oda_read_device_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         lib.oda_launch_count.argtypes = [vp]
         lib.oda_launch_count.restype = ctypes.c_int64
@@ -201,6 +206,18 @@ class OdaContext:
     def set_workspace(self, ptr: int, nbytes: int, stream: Optional[int] = None):
         self._check(self.lib.oda_set_workspace(self._h, ptr, nbytes, _stream() if stream is None else stream),
                     "oda_set_workspace")
+
+    def calibration_begin(self, stream=None):
+        """Start recording per-SM streaming rates in the attention launches that follow."""
+        self._check(self.lib.oda_calibration_begin(self._h, _stream() if stream is None else stream),
+                    "oda_calibration_begin")
+
+    def calibration_end(self, stream=None) -> float:
+        """Fix the split of work across SMs from the recorded rates.  Returns slowest/fastest
+        rate (0: not applied, e.g. no large launch was seen)."""
+        self._check(self.lib.oda_calibration_end(self._h, _stream() if stream is None else stream),
+                    "oda_calibration_end")
+        return self.lib.oda_calibration_spread(self._h)
 
     # ---- the four calls of the path -------------------------------------------------
     def local_decode(self, layer_begin, layer_end, batch, q, k_cache, v_cache, block_table, seq_lens,

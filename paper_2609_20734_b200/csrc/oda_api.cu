@@ -22,7 +22,7 @@ constexpr size_t kAlign = 256;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct WsLayout {
-    size_t status, layers, tickets, head_partial, partials;
+    size_t status, layers, tickets, head_partial, sm_claims, sm_bytes, cum_share, partials;
     size_t st_q_local, st_q_full, st_feat, st_override, st_out, st_lse, st_scores, st_logits, st_flags;
     size_t total;
 };
@@ -40,10 +40,10 @@ struct oda_ctx {
     int num_sms = 148;
     int variant = ODA_VARIANT_SIMT;
     int grid = 148;
-    int min_span_pages = 16;
-    int first_span_pct = 88;
-    int tail_span_pct = 6;
-    int dynamic_min_fair_pages = 1 << 30;  // dynamic hand-out off: measured slower than the static split (see oda_device.cuh)
+    int min_span_pages = 8;
+    bool calibrated = false;  // the per-SM split table in the workspace is valid
+    bool calibrating = false; // attention launches record per-SM streaming rates
+    double calib_spread = 0.0; // slowest / fastest SM share seen by oda_calibrate
     int max_items = 0;
     int head_grid = 1;
     WsLayout lay{};
@@ -87,6 +87,9 @@ void compute_layout(oda_ctx* c)
     w.layers = take(L * sizeof(LayerInfo));
     w.tickets = take(L * B * f.num_kv_heads * sizeof(int32_t));
     w.head_partial = take((size_t)c->head_grid * B * sizeof(float));
+    w.sm_claims = take(1024 * sizeof(int32_t));
+    w.sm_bytes = take(2 * 1024 * sizeof(unsigned long long));
+    w.cum_share = take((kMaxGrid + 1) * sizeof(uint16_t));
     w.partials = take((size_t)c->max_items * c->group * (D + kPartHdr) * sizeof(float));
     w.st_q_local = take(L * B * Hq * D * 2);
     w.st_q_full = take(L * B * Hq * D * 2);
@@ -151,9 +154,6 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     p.mode = mode;
     p.ncls = c->ncls;
     p.min_span_pages = c->min_span_pages;
-    p.first_span_pct = c->first_span_pct;
-    p.tail_span_pct = c->tail_span_pct;
-    p.dynamic_min_fair_pages = c->dynamic_min_fair_pages;
     p.max_items = c->max_items;
     p.scale_log2e = c->scale * 1.4426950408889634f;
     bool any = false;
@@ -169,8 +169,13 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
     p.advance_seq_lens = advance;
     p.done_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 128);
-    p.span_counter = c->variant == ODA_VARIANT_TMA_MMA ? reinterpret_cast<int32_t*>(c->ws + c->lay.status + 160) : nullptr;
     p.exit_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 192);
+    p.num_sms = c->num_sms;
+    if (c->calibrating) p.sm_stats = reinterpret_cast<unsigned long long*>(c->ws + c->lay.sm_bytes);
+    if (c->calibrated) {
+        p.cum_share = reinterpret_cast<const uint16_t*>(c->ws + c->lay.cum_share);
+        p.sm_claims = reinterpret_cast<int32_t*>(c->ws + c->lay.sm_claims);
+    }
     if (advanced) *advanced = advance != nullptr;
     cudaError_t e;
     if (c->variant == ODA_VARIANT_TMA_MMA) {
@@ -296,10 +301,6 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         delete c;
         return ODA_ERR_UNSUPPORTED;  // layer stride is not a whole number of blocks
     }
-    if (const char* e = std::getenv("ODA_MIN_SPAN_PAGES")) c->min_span_pages = std::max(1, std::atoi(e));
-    if (const char* e = std::getenv("ODA_TAIL_SPAN_PCT")) c->tail_span_pct = std::min(100, std::max(1, std::atoi(e)));
-    if (const char* e = std::getenv("ODA_DYNAMIC_MIN_FAIR")) c->dynamic_min_fair_pages = std::max(1, std::atoi(e));
-    if (const char* e = std::getenv("ODA_FIRST_SPAN_PCT")) c->first_span_pct = std::min(100, std::max(1, std::atoi(e)));
     c->use_pdl = cfg->reserved == 0;  // reserved = 1 turns programmatic dependent launch off
     c->variant = cfg->variant == ODA_VARIANT_AUTO ? (tma_ok ? ODA_VARIANT_TMA_MMA : ODA_VARIANT_SIMT) : cfg->variant;
     int dev = 0, sms = 0;
@@ -314,7 +315,7 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         c->num_sms = 148;  // no device visible: sizes follow a B200 so that host-only checks still work
         c->grid = 148 * 2;
     }
-    c->max_items = c->grid * kMaxLevels + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
+    c->max_items = c->grid + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
     c->head_grid = cfg->head_d_hidden > 0 ? recall_head_grid(cfg->head_d_hidden) : 1;
     compute_layout(c);
     *out_ctx = c;
@@ -346,8 +347,62 @@ oda_status_t oda_set_workspace(oda_ctx_t* c, void* dev_ptr, size_t bytes, void* 
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(c, e, "workspace initialisation");
     c->ws = ws;
+    c->calibrated = false;  // the table lives in the workspace
     return ODA_OK;
 }
+
+oda_status_t oda_calibration_begin(oda_ctx_t* c, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    cudaError_t e = cudaMemsetAsync(c->ws + c->lay.sm_bytes, 0, 2 * 1024 * sizeof(unsigned long long),
+                                    static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(c, e, "calibration memset");
+    c->calibrated = false;  // measure under the equal split
+    c->calibrating = true;
+    return ODA_OK;
+}
+
+oda_status_t oda_calibration_end(oda_ctx_t* c, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    if (!c->calibrating) return fail(c, ODA_ERR_INVALID_ARG, "oda_calibration_begin has not been called");
+    c->calibrating = false;
+    // the weighted split assumes two resident CTAs per SM (the TMA variant's launch shape)
+    if (c->variant != ODA_VARIANT_TMA_MMA || c->grid != 2 * c->num_sms || c->grid > kMaxGrid || c->num_sms > 1024)
+        return ODA_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<unsigned long long> h(2 * 1024);
+    cudaError_t e = cudaMemcpyAsync(h.data(), c->ws + c->lay.sm_bytes, h.size() * sizeof(unsigned long long),
+                                    cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "calibration read-back");
+    std::vector<double> rate(c->num_sms);
+    double total = 0.0, lo = 1e300, hi = 0.0;
+    for (int i = 0; i < c->num_sms; ++i) {
+        if (h[2 * i] == 0 || h[2 * i + 1] == 0) return ODA_OK;  // an SM saw no large launch: keep the equal split
+        rate[i] = (double)h[2 * i] / (double)h[2 * i + 1];
+        total += rate[i];
+        lo = std::min(lo, rate[i]);
+        hi = std::max(hi, rate[i]);
+    }
+    std::vector<uint16_t> cum(kMaxGrid + 1, 0);
+    double acc = 0.0;
+    for (int v = 0; v < c->grid; ++v) {
+        cum[v] = (uint16_t)std::min(65535.0, std::floor(acc / total * 65536.0 + 0.5));
+        acc += 0.5 * rate[v / 2];
+    }
+    e = cudaMemcpyAsync(c->ws + c->lay.cum_share, cum.data(), cum.size() * sizeof(uint16_t), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->lay.sm_claims, 0, 1024 * sizeof(int32_t), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "calibration table upload");
+    c->calibrated = true;
+    c->calib_spread = lo / hi;
+    return ODA_OK;
+}
+
+double oda_calibration_spread(const oda_ctx_t* c) { return c && c->calibrated ? c->calib_spread : 0.0; }
 
 oda_status_t oda_local_decode(oda_ctx_t* c, int32_t lb, int32_t le, int32_t batch, const void* q,
                               const void* k, const void* v, const int32_t* bt, const int32_t* sl,

@@ -40,18 +40,21 @@ struct AttnParams {
     int32_t num_q_heads, num_kv_heads, max_blocks_per_seq, out_bf16;
     int32_t mode;          // 0 = Local (Eq. 1 S^L), 1 = gated Full (S^F)
     int32_t ncls;
-    int32_t min_span_pages;  // smallest span handed out (unless there are fewer pages)
-    int32_t first_span_pct;  // first-level span length as a percentage of the fair share per CTA
-    int32_t tail_span_pct;   // length of the spans handed out after the first level, same unit
-    int32_t dynamic_min_fair_pages;  // below this fair share the split is one static level
+    int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)
     int32_t cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
     int32_t cls_layers_in_call[kMaxClasses];
     int32_t* advance_seq_lens;  // nullable: seq_lens to increment once every CTA has read them
     int32_t* done_counter;      // zero between launches
-    int32_t* span_counter;      // dynamic span hand-out (TMA variant), zero between launches
-    int32_t* exit_counter;      // CTAs that finished taking spans, zero between launches
+    // Optional per-SM weighting of the split (oda_calibrate): cum_share[v] / 65536 is the part of
+    // the page axis that lies before span v; spans 2*sm and 2*sm+1 belong to SM `sm`.  nullptr =>
+    // equal spans, span = blockIdx.x.
+    const uint16_t* cum_share;
+    int32_t* sm_claims;         // [num_sms] CTAs that have claimed a span of that SM; zero between launches
+    int32_t* exit_counter;      // CTAs past their claim; zero between launches
+    unsigned long long* sm_stats;  // calibration run: per SM (pages streamed, nanoseconds); else nullptr
+    int32_t num_sms;
 };
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
@@ -63,19 +66,16 @@ __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("grid
 // Work decomposition.  A unit is one (layer, request, kv head); it owns np pages of KV (the
 // pages of its Eq. 1 window segment, or of the whole history in Full mode; requests that are not
 // flagged and layers that are not gated own none).  All units are laid end to end, layer-major
-// then request then kv head, on one axis of P pages.  The axis is cut into spans in levels.
-// With little work per CTA there is one level: span j is the j-th fair share P / gridDim.
-// Otherwise level 0 has one span per CTA of first_span_pct % of the fair share and the rest of
-// the axis is cut into short spans (tail_span_pct % of the fair share) in further levels.
-// A span that crosses a unit boundary yields one item per unit it touches; a unit touched by
-// several spans has that many partials.  The SIMT variant gives CTA c the spans c, c + grid, ...
-// (one per level); the TMA variant hands out the spans after level 0 through an atomic counter,
-// so CTAs that stream faster (the measured spread between CTAs is +-10 %) take more of the
-// short spans at the end.  On the 4.3 GB Full pass of the 32-layer benchmark the hand-out measured
-// slower than the one-level static split (692-950 us against 665 us: every short span costs a
-// partial, a fence and a ticket in the epilogue warp), so it is off by default
-// (dynamic_min_fair_pages = 2^30) and kept for experiments.
-constexpr int kMaxLevels = 16;
+// then request then kv head, on one axis of P pages; the axis is cut into nseg <= gridDim.x spans
+// and every CTA streams one span.  A span that crosses a unit boundary yields one item per unit it
+// touches; a unit touched by several spans has that many partials.  By default the spans are
+// equal (+-1 page): every CTA reads the same number of bytes whatever the mix of lengths and
+// flags is.  SMs do not all get the same share of HBM bandwidth, though (on a B200 the streaming
+// time of equal spans spreads over +-10 % and the pattern is a fixed property of the SM), so
+// after a calibration run (oda_calibration_begin/end) the span lengths follow the measured rate
+// of the SM the CTA runs on:
+// the CTA reads %smid, claims one of that SM's two spans, and all CTAs finish together.
+constexpr int kMaxGrid = 320;
 
 struct Plan {  // shared memory, one per CTA
     int32_t pb[kMaxClasses][kMaxBatch + 1];  // exclusive prefix over requests of pages per kv head
@@ -84,13 +84,12 @@ struct Plan {  // shared memory, one per CTA
     uint16_t kv_index[kMaxLayers];
     uint8_t cls[kMaxLayers];
     uint8_t active[kMaxBatch];               // request takes part in this launch (Full mode: flagged)
-    int32_t lvl_base[kMaxLevels + 1];        // first axis page of each level
-    int32_t lvl_span0[kMaxLevels + 1];       // first span index of each level
-    int32_t lvl_size[kMaxLevels];            // span length of each level
-    int32_t nlevels;
+    uint16_t cum[kMaxGrid];                  // weighted split: share of the axis before span v (x 2^-16)
+    int32_t weighted;                        // cum[] is in use
+    int32_t my_span;                         // the span this CTA streams (-1: none)
     int32_t total_pages;
     int32_t nseg;
-    int32_t pad[2];
+    int32_t pad;
 };
 static_assert(sizeof(Plan) % 8 == 0, "Plan is followed by 8-byte aligned barriers in shared memory");
 
@@ -143,6 +142,19 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     const int tid = threadIdx.x, nth = blockDim.x;
     const int B = p.batch;
     const int nl = p.layer_end - p.layer_begin;
+    // weighted split: claim one of the two spans of the SM this CTA runs on (answer used at the end)
+    const bool weighted = p.cum_share != nullptr && (int)gridDim.x == 2 * p.num_sms && (int)gridDim.x <= kMaxGrid;
+    int claim_sm = 0, claim_slot = 0;
+    if (weighted && tid == 0) {
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(claim_sm));
+        if (claim_sm >= p.num_sms) claim_sm = p.num_sms - 1;
+        claim_slot = atomicAdd(p.sm_claims + claim_sm, 1);
+    }
+    uint16_t cum0 = 0, cum1 = 0;
+    if (weighted) {
+        if (tid < (int)gridDim.x) cum0 = p.cum_share[tid];
+        if (tid + nth < (int)gridDim.x) cum1 = p.cum_share[tid + nth];
+    }
     // issue every global load of the plan before using any of them: one memory latency, not three
     const bool has_b = tid < B;  // blockDim.x >= kMaxBatch
     const int t_raw = has_b ? p.seq_lens[tid] : 1;
@@ -162,6 +174,10 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     }
     if (tid < nl) { pl.cls[tid] = (uint8_t)li0.cls; pl.kv_index[tid] = (uint16_t)li0.kv_index; }
     if (tid + nth < nl) { pl.cls[tid + nth] = (uint8_t)li1.cls; pl.kv_index[tid + nth] = (uint16_t)li1.kv_index; }
+    if (weighted) {
+        if (tid < (int)gridDim.x) pl.cum[tid] = cum0;
+        if (tid + nth < (int)gridDim.x) pl.cum[tid + nth] = cum1;
+    }
     __syncthreads();
     const int warp = tid >> 5, lane = tid & 31, nwarps = nth >> 5;
     for (int c = warp; c < p.ncls; c += nwarps) {  // one warp scans one class
@@ -209,36 +225,29 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             }
             pl.lb[nl] = (int32_t)carry;
             pl.total_pages = (int32_t)carry;
-            // span levels
             const int g = (int)gridDim.x;
-            const int P = (int)carry;
             const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
-            const long long fair = ((long long)P + g - 1) / g;
-            // little work per CTA: one level, the whole fair share at once (nothing to gain from a
-            // hand-out whose per-span cost is comparable to the work)
-            const bool dynamic = p.span_counter != nullptr && fair >= p.dynamic_min_fair_pages;
-            int size = dynamic ? (int)((fair * p.first_span_pct + 99) / 100) : (int)fair;
-            int tail = (int)((fair * p.tail_span_pct + 99) / 100);
-            if (tail < minS) tail = minS;
-            int done = 0, spans = 0, lv = 0;
-            while (done < P) {
-                if (size < minS) size = minS;
-                int rem = P - done;
-                if (lv == kMaxLevels - 1) size = (rem + g - 1) / g;  // last level takes whatever is left
-                int n = (rem + size - 1) / size;
-                if (n > g) n = g;
-                pl.lvl_base[lv] = done;
-                pl.lvl_span0[lv] = spans;
-                pl.lvl_size[lv] = size;
-                done += (long long)n * size > rem ? rem : n * size;
-                spans += n;
-                ++lv;
-                size = tail;
+            long long n = (carry + minS - 1) / minS;
+            if (n > g) n = g;
+            pl.nseg = (int32_t)n;
+            // the weighted split needs every CTA to have real work; small launches stay equal
+            pl.weighted = weighted && n == g;
+            int span = (int)blockIdx.x;
+            if (pl.weighted) {
+                span = -1;
+                if (claim_slot < 2) {
+                    span = 2 * claim_sm + claim_slot;
+                } else {
+                    // more than two CTAs landed on this SM (not expected with two resident CTAs per
+                    // SM): take any span that is still free
+                    for (int k = 1; k < p.num_sms && span < 0; ++k) {
+                        const int sm = (claim_sm + k) % p.num_sms;
+                        const int slot = atomicAdd(p.sm_claims + sm, 1);
+                        if (slot < 2) span = 2 * sm + slot;
+                    }
+                }
             }
-            pl.lvl_base[lv] = P;
-            pl.lvl_span0[lv] = spans;
-            pl.nlevels = lv;
-            pl.nseg = spans;
+            pl.my_span = span >= 0 && span < pl.nseg ? span : -1;
         }
     }
     __syncthreads();
@@ -250,6 +259,15 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         if (old == (int)gridDim.x - 1) {
             *p.done_counter = 0;
             for (int b = 0; b < B; ++b) p.advance_seq_lens[b] += 1;
+        }
+    }
+    // Every CTA has made its claim(s) by now; the one that notes this last re-arms the table.
+    if (weighted && tid == 0) {
+        __threadfence();
+        const int old = atomicAdd(p.exit_counter, 1);
+        if (old == (int)gridDim.x - 1) {
+            *p.exit_counter = 0;
+            for (int i = 0; i < p.num_sms; ++i) p.sm_claims[i] = 0;
         }
     }
 }
@@ -266,19 +284,27 @@ __device__ __forceinline__ void prefetch_block_table(const AttnParams& p)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
 }
 
+__device__ __forceinline__ int span_begin(const Plan& pl, int j)
+{
+    if (j >= pl.nseg) return pl.total_pages;
+    if (pl.weighted) return (int)(((long long)pl.cum[j] * pl.total_pages) >> 16);
+    return (int)(((long long)j * pl.total_pages) / pl.nseg);
+}
 __device__ __forceinline__ void span_range(const Plan& pl, int j, int& x0, int& x1)
 {
-    int lv = 0;
-    while (lv + 1 < pl.nlevels && pl.lvl_span0[lv + 1] <= j) ++lv;
-    x0 = pl.lvl_base[lv] + (j - pl.lvl_span0[lv]) * pl.lvl_size[lv];
-    x1 = min(x0 + pl.lvl_size[lv], pl.lvl_base[lv + 1]);
+    x0 = span_begin(pl, j);
+    x1 = span_begin(pl, j + 1);
 }
-// the span that contains axis page x
+// the last span that begins at or before axis page x (the span that contains x)
 __device__ __forceinline__ int span_of(const Plan& pl, int x)
 {
-    int lv = 0;
-    while (lv + 1 < pl.nlevels && pl.lvl_base[lv + 1] <= x) ++lv;
-    return pl.lvl_span0[lv] + (x - pl.lvl_base[lv]) / pl.lvl_size[lv];
+    if (!pl.weighted) return (int)((((long long)x + 1) * pl.nseg - 1) / pl.total_pages);
+    int lo = 0, hi = pl.nseg;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (span_begin(pl, mid) <= x) lo = mid; else hi = mid;
+    }
+    return lo;
 }
 
 // The item of span j that starts at axis page x (x0 <= x < x_end of span_range(j)).

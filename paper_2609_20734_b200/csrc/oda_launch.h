@@ -19,6 +19,7 @@ cudaError_t launch_splitkv_tma(const AttnParams& p, const void* kmap, const void
                                int head_dim, int group, int grid, cudaStream_t st, bool pdl = false);
 int occupancy_splitkv_tma(int head_dim, int group);
 
+
 struct HeadParams {
     const float* feat_ext;      // [B, d_ext] or nullptr
     const void* attn_out;       // [B, d_attn] fp32 or bf16, or nullptr

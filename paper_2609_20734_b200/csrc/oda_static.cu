@@ -14,7 +14,7 @@ namespace {
 constexpr int kStaticMaxBatch = 16;
 constexpr int kStaticMaxUnits = 256;   // batch * kv heads
 constexpr int kStaticMaxGrid = 148;
-constexpr int kStaticMaxItems = 2 * kStaticMaxGrid + kStaticMaxUnits;  // spans (two levels at most) + units
+constexpr int kStaticMaxItems = kStaticMaxGrid + kStaticMaxUnits;  // one partial slot per (span, unit) pair
 constexpr size_t kOffStatus = 0;                              // int32
 constexpr size_t kOffLayer = 256;                             // one LayerInfo
 constexpr size_t kOffTickets = 512;                           // kStaticMaxUnits int32
@@ -112,9 +112,6 @@ extern "C" oda_status_t oda_local_decode_static(int32_t batch, int32_t num_q_hea
     p.max_blocks_per_seq = max_blocks_per_seq;
     p.ncls = 1;
     p.min_span_pages = 8;
-    p.first_span_pct = 100;
-    p.tail_span_pct = 100;
-    p.dynamic_min_fair_pages = 1 << 30;  // one static level: at most gridDim spans, as the scratch assumes
     p.max_items = kStaticMaxItems;
     p.scale_log2e = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;
     p.cls_window[0] = window;

@@ -55,7 +55,8 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
     const int sub = lane / C::kLPR;               // which row of a warp-wide load this lane reads
     const int dofs = (lane % C::kLPR) * 8;        // this lane's 8 head-dim elements
 
-    for (int span = blockIdx.x; span < plan.nseg; span += gridDim.x)
+    const int span = plan.my_span;
+    if (span < 0) return;
     {
     int x_begin, x_end;
     span_range(plan, span, x_begin, x_end);

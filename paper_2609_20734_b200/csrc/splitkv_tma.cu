@@ -1,9 +1,8 @@
 // Split-KV paged decode attention, TMA + tensor-core variant for sm_100a.
 //
 // Six warps per CTA, two CTAs per SM, persistent:
-//  * one producer warp takes spans of the page axis (its first one statically, the rest from
-//    an atomic counter), looks up block ids a run of 32 pages ahead, and streams KV pages into a
-//    96 KiB shared-memory ring with tiled TMA copies (cp.async.bulk.tensor, 128-byte swizzle,
+//  * one producer warp walks the CTA's span of the page axis, looks up block ids a run of 32
+//    pages ahead, and streams KV pages into a 96 KiB shared-memory ring with tiled TMA copies (cp.async.bulk.tensor, 128-byte swizzle,
 //    completion on mbarriers); each item's q rows ride along with its first tile;
 //  * four consumer warps each take one 16-token page of a tile and run the GQA group tile on the
 //    tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate), transposed so that every accumulator
@@ -41,7 +40,6 @@ struct EpiMeta {  // what the epilogue warp needs to know about a finished item
 struct Ctl {  // barriers and small hand-off slots, after the Plan in shared memory
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t efull, efree;
-    int32_t span_slot[kMaxStages];  // span id delivered with the first tile of a span (-1: no more work)
     int32_t abort;
     int32_t pad;
     EpiMeta meta;
@@ -197,9 +195,7 @@ struct PageRun {
     int g, kv_layer, b;
     const __nv_bfloat16* q;  // q rows of the item, copied with the first tile of the item
     int pg, n;               // first logical page, pages in the run (1..32)
-    int span;                // span the run belongs to
     bool first;              // first run of its item
-    bool span_first;         // first run of its span
 };
 
 template <int D, int G>
@@ -240,42 +236,31 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     if (tid == 0) ODA_TL(2);
     volatile int* abort_flag = &ctl.abort;
     constexpr uint32_t kQBytes = G * D * 2;
+    const int span = plan.my_span;  // the one span this CTA streams
+    if (span < 0) return;
 
     if (warp == C::kProducerWarp) {
         // ============================ producer warp ============================
         const uint64_t policy = 0x12F0000000000000ull;  // L2 evict-first: the KV stream is read once
         uint32_t cnt = 0;
         bool dead = false;
-        // Walker over the runs of all the spans this CTA takes.  The first span is the CTA's own;
-        // every further one comes from the counter, asked for one span ahead so that the answer
-        // is there when the current span runs out and the stream of copies never pauses.
-        int span = (int)blockIdx.x < plan.nseg ? (int)blockIdx.x : -1;
-        int pending = 0;   // lane 0: span id requested from the counter, not yet used
-        int x = 0, x_end = 0, take = 0, seg = 0, pg = 0;
+        // walker over the runs of the CTA's span
+        int x, x_end;
+        span_range(plan, span, x, x_end);
         Item it;
-        bool item_first = true, span_first = true;
-        auto open_span = [&]() {  // span >= 0: position the walker on its first item and ask for the next span
-            if (lane == 0) pending = atomicAdd(p.span_counter, 1) + (int)gridDim.x;
-            span_range(plan, span, x, x_end);
-            take = decode_item(p, plan, span, x, x_end, it);
-            seg = it.sink_pg1 > 0 ? 0 : 1;
-            pg = seg ? it.win_pg0 : 0;
-            item_first = true;
-            span_first = true;
-        };
-        if (span >= 0) open_span();
-        auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when there is no more work
-            if (span < 0) return false;
+        int take = decode_item(p, plan, span, x, x_end, it);
+        int seg = it.sink_pg1 > 0 ? 0 : 1;
+        int pg = seg ? it.win_pg0 : 0;
+        bool more = true, item_first = true;
+        auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when the span is done
+            if (!more) return false;
             const int end = seg ? it.win_pg1 : it.sink_pg1;
             r.g = it.g; r.kv_layer = it.kv_layer; r.b = it.b;
             r.q = p.q + (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + (size_t)it.g * G) * D;
             r.pg = pg;
             r.n = min(32, end - pg);
-            r.span = span;
             r.first = item_first;
-            r.span_first = span_first;
             item_first = false;
-            span_first = false;
             blk = lane < r.n ? __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + pg + lane) : 0;
             pg += r.n;
             if (pg >= end) {
@@ -290,9 +275,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                         pg = seg ? it.win_pg0 : 0;
                         item_first = true;
                     } else {
-                        const int nx = __shfl_sync(0xffffffffu, pending, 0);
-                        span = nx < plan.nseg ? nx : -1;
-                        if (span >= 0) open_span();
+                        more = false;
                     }
                 }
             }
@@ -309,10 +292,8 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { dead = true; break; }
                 const bool with_q = cur.first && t0 == 0;
                 if (cnt == 0) ODA_TL(3);
-                if (lane == 0) {
-                    if (cur.span_first && t0 == 0) ctl.span_slot[s] = cur.span;  // ordered before the arrive below
+                if (lane == 0)
                     mbar_expect_tx(full0 + 8 * s, (uint32_t)np * 2 * C::kPageBytes + (with_q ? kQBytes : 0u));
-                }
                 __syncwarp();
                 const int blk = __shfl_sync(0xffffffffu, blk_cur, t0 + (lane & 3));
                 if (lane < np) {
@@ -330,30 +311,10 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             blk_cur = blk_nxt;
             have = have_next;
         }
-        if (!dead) {  // tell the consumers that nothing more will come
-            const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
-            if (mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) {
-                if (lane == 0) {
-                    ctl.span_slot[s] = -1;
-                    mbar_arrive(full0 + 8 * s);
-                }
-                ++cnt;
-            }
-        }
-        // This CTA will not touch the span counter again: the CTA that notes this last re-arms
-        // both counters for the next launch.
-        if (lane == 0) {
-            __threadfence();
-            const int old = atomicAdd(p.exit_counter, 1);
-            if (old == (int)gridDim.x - 1) {
-                *p.span_counter = 0;
-                *p.exit_counter = 0;
-            }
-        }
         // Do not leave while copies may still be landing in this CTA's shared memory: wait
         // (bounded) until the consumers have released every stage that was armed.
-        for (uint32_t k = 1; k < (uint32_t)C::kStages + 1 && k < cnt; ++k) {
-            const uint32_t c2 = cnt - 1 - k;  // (the last count is the end marker, which carries no copy)
+        for (uint32_t k = 0; k < (uint32_t)C::kStages && k < cnt; ++k) {
+            const uint32_t c2 = cnt - 1 - k;
             const uint32_t s = c2 % C::kStages, ph = (c2 / C::kStages) & 1;
             if (!mbar_wait(empty0 + 8 * s, ph, abort_flag, p.status)) break;
         }
@@ -456,16 +417,12 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     uint32_t ecnt = 0;   // items handed to the epilogue warp
     bool aborted = false;
 
-    while (!aborted) {
-        int span;
-        {   // the first tile of a span carries the span id
-            const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
-            if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
-            span = ctl.span_slot[s];
-        }
-        if (span < 0) break;
+    int span_pages = 0;
+    uint64_t t_first = 0;
+    {
         int x, x_end;
         span_range(plan, span, x, x_end);
+        span_pages = x_end - x;
         while (x < x_end && !aborted) {
             Item it;
             x += decode_item(p, plan, span, x, x_end, it);
@@ -475,6 +432,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
                 if (cnt == 0 && warp == 0) ODA_TL(4);
+                if (cnt == 0 && p.sm_stats) t_first = globaltimer_ns();
                 const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
 #pragma unroll
                 for (int kc = 0; kc < D / 16; ++kc) {
@@ -627,6 +585,15 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (lane == 0) mbar_arrive(efull);
             }
             ++ecnt;
+        }
+    }
+    // calibration run: how long this SM took to stream how many pages
+    if (p.sm_stats && tid == 0 && !aborted && plan.nseg == (int)gridDim.x) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        if ((int)smid < p.num_sms) {
+            atomicAdd(p.sm_stats + 2 * smid, (unsigned long long)span_pages);
+            atomicAdd(p.sm_stats + 2 * smid + 1, (unsigned long long)(globaltimer_ns() - t_first));
         }
     }
     // end marker for the epilogue warp (also on the abort path, where its own waits are bounded)

@@ -173,28 +173,31 @@ def test_peaked_softmax_short_sequences(variant):
     gh.assert_close(out2.cpu().numpy(), reff, gh.ATOL_OUT, "peaked full")
 
 
-def test_dynamic_span_handout_gives_the_same_result(monkeypatch):
-    """The optional two-level split with an atomic hand-out of the short spans (off by default)
-    computes the same attention: same oracle bar, and the same bits on a second run."""
-    monkeypatch.setenv("ODA_DYNAMIC_MIN_FAIR", "1")
-    monkeypatch.setenv("ODA_FIRST_SPAN_PCT", "60")
-    monkeypatch.setenv("ODA_TAIL_SPAN_PCT", "10")
-    monkeypatch.setenv("ODA_MIN_SPAN_PAGES", "2")
-    seq = [4100, 700, 33, 2053, 1]
+def test_calibrated_split_gives_the_same_result():
+    """After a calibration run the spans follow the measured per-SM streaming rates: same oracle
+    bar, same bits on a second run, and agreement with the equal split up to summation order."""
+    seq = [40000, 700, 33, 20530, 1]
     prob = make_problem(29, 3, len(seq), 8, 2, 128, seq)
     windows, sinks, gated = [512, 64, 512], [4, 0, 4], [1, 0, 1]
     ctx = gh.make_ctx(prob, windows, sinks, gated, variant=binding.VARIANT_TMA_MMA)
     dev = gh.upload(prob)
+    ones = torch.ones(len(seq), dtype=torch.uint8, device="cuda")
+    before, _ = gh.new_out(prob)
+    ctx.calibration_begin()
+    ctx.full_decode_gated(0, 3, len(seq), dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], ones, before, None)
+    spread = ctx.calibration_end()
+    assert 0.3 < spread <= 1.0
     out, lse = gh.gpu_local(ctx, prob, dev)
     ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8)
-    gh.assert_close(out, ref, gh.ATOL_OUT, "dynamic local")
+    gh.assert_close(out, ref, gh.ATOL_OUT, "calibrated local")
     again, _ = gh.gpu_local(ctx, prob, dev)
     np.testing.assert_array_equal(again, out)
     full, flse = gh.new_out(prob)
-    ctx.full_decode_gated(0, 3, len(seq), dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
-                          torch.ones(len(seq), dtype=torch.uint8, device="cuda"), full, flse)
+    for _ in range(2):   # twice: the per-SM claim table must be re-armed between launches
+        ctx.full_decode_gated(0, 3, len(seq), dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], ones, full, flse)
     torch.cuda.synchronize()
     reff, _ = oracle_attention(prob, "full", windows, sinks, nthreads=8)
     for l in (0, 2):
-        gh.assert_close(full[l].cpu().numpy(), reff[l], gh.ATOL_OUT, f"dynamic full layer {l}")
+        gh.assert_close(full[l].cpu().numpy(), reff[l], gh.ATOL_OUT, f"calibrated full layer {l}")
+        np.testing.assert_allclose(full[l].cpu().numpy(), before[l].cpu().numpy(), rtol=0, atol=1e-5)
     assert ctx.read_device_status() == 0
