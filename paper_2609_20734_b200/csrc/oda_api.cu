@@ -22,7 +22,7 @@ constexpr size_t kAlign = 256;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct WsLayout {
-    size_t status, layers, tickets, head_partial, sm_claims, sm_bytes, cum_share, partials;
+    size_t status, layers, tickets, head_partial, head_pre, head_rb_tickets, sm_claims, sm_bytes, cum_share, partials;
     size_t st_q_local, st_q_full, st_feat, st_override, st_out, st_lse, st_scores, st_logits, st_flags;
     size_t total;
 };
@@ -87,6 +87,11 @@ void compute_layout(oda_ctx* c)
     w.layers = take(L * sizeof(LayerInfo));
     w.tickets = take(L * B * f.num_kv_heads * sizeof(int32_t));
     w.head_partial = take((size_t)c->head_grid * B * sizeof(float));
+    w.head_rb_tickets = take((size_t)c->head_grid * sizeof(int32_t));
+    {
+        const size_t d_in = (size_t)std::max(0, f.head_d_ext) + (f.head_use_attn_out ? Hq * D : 0);
+        w.head_pre = take((size_t)recall_head_ksplits((int)d_in) * (size_t)std::max(1, f.head_d_hidden) * B * sizeof(float));
+    }
     w.sm_claims = take(1024 * sizeof(int32_t));
     w.sm_bytes = take(2 * 1024 * sizeof(unsigned long long));
     w.cum_share = take((kMaxGrid + 1) * sizeof(uint16_t));
@@ -458,11 +463,15 @@ oda_status_t oda_recall_score(oda_ctx_t* c, int32_t batch, const float* feat_ext
     p.flags = flags;
     p.counters = counters;
     p.partial = reinterpret_cast<float*>(c->ws + c->lay.head_partial);
+    p.pre = reinterpret_cast<float*>(c->ws + c->lay.head_pre);
+    p.rb_tickets = reinterpret_cast<int32_t*>(c->ws + c->lay.head_rb_tickets);
     p.ticket = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 64);
     p.batch = batch;
     p.attn_bf16 = f.out_dtype;
     p.max_batch = f.max_batch;
     p.threshold = threshold;
+    p.vec4 = (p.d_ext % 4 == 0) && (p.d_attn % 4 == 0) && aligned16(W1) && aligned16(feat_ext) &&
+             aligned16(attn_out_last);
     cudaError_t e = launch_recall_head(p, static_cast<cudaStream_t>(stream), c->use_pdl);
     if (e != cudaSuccess) return cuda_fail(c, e, "recall head launch");
     c->launches += 1;

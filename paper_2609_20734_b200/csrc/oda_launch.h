@@ -29,13 +29,19 @@ struct HeadParams {
     float* logits;
     uint8_t* flags;
     int32_t* counters;
-    float* partial;             // [grid][max_batch] scratch
+    float* partial;             // [row blocks][max_batch] scratch
+    float* pre;                 // [K slices][d_hidden][max_batch] partial pre-activations
     int32_t* ticket;            // one int, zero between launches
+    int32_t* rb_tickets;        // [row blocks], zero between launches
     int32_t batch, d_ext, d_attn, d_hidden, attn_bf16, max_batch;
+    int32_t vec4;               // 128-bit loads are legal: widths multiples of 4, pointers 16-byte aligned
     float threshold;
 };
 
+constexpr int kMaxHeadBatch = 128;
+
 int recall_head_grid(int d_hidden);
+int recall_head_ksplits(int d_in);
 cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl = false);
 cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st, bool pdl = false);
 

@@ -11,85 +11,165 @@
 
 namespace oda {
 
-constexpr int kHeadWarps = 4;
-constexpr int kHeadBT = 8;  // requests per register tile
+constexpr int kHeadRows = 8;                  // hidden rows per CTA, one warp each
+constexpr int kHeadThreads = kHeadRows * 32;
+constexpr int kHeadBT = 16;                   // requests per tile
+constexpr int kHeadKT = 512;                  // input features per CTA (split-K)
 
 __device__ __forceinline__ float head_x(const HeadParams& p, int b, int i)
 {
     if (i < p.d_ext) return __ldg(p.feat_ext + (size_t)b * p.d_ext + i);
     size_t k = (size_t)b * p.d_attn + (i - p.d_ext);
     if (p.attn_bf16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.attn_out)[k]);
-    return __ldcg(reinterpret_cast<const float*>(p.attn_out) + k);
+    return reinterpret_cast<const float*>(p.attn_out)[k];
 }
 
-__global__ void __launch_bounds__(kHeadWarps * 32) recall_head_kernel(const __grid_constant__ HeadParams p)
+// four consecutive input features of request b starting at feature i (i % 4 == 0, vector path)
+__device__ __forceinline__ float4 head_x4(const HeadParams& p, int b, int i)
 {
-    __shared__ float s_h[kHeadWarps][256];
+    if (i < p.d_ext) return __ldg(reinterpret_cast<const float4*>(p.feat_ext + (size_t)b * p.d_ext + i));
+    const size_t k = (size_t)b * p.d_attn + (i - p.d_ext);
+    if (p.attn_bf16) {
+        const uint2 r = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(p.attn_out) + k);
+        return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
+                           __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+    }
+    return *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.attn_out) + k);
+}
+
+// Split-K GEMV: CTA (rb, ks) multiplies kHeadRows rows of W1 (HBM, read once, 128-bit loads) by
+// one 512-feature tile of the inputs x of up to 16 requests (staged in shared memory), and
+// publishes the partial pre-activations.  The last CTA of a row block (atomic ticket, no
+// waiting) adds the K slices in order, applies bias, SiLU and w2; the last row block adds the
+// row blocks' sums in a fixed tree and writes score, logit, flag and counters.  Every sum has a
+// fixed order, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_constant__ HeadParams p)
+{
+    __shared__ __align__(16) float s_x[kHeadBT][kHeadKT];
+    __shared__ float s_h[kHeadRows][kMaxHeadBatch];
     __shared__ int s_last;
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the Local output it reads comes from the previous kernel
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int j = blockIdx.x * kHeadWarps + warp;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rb = blockIdx.x, ks = blockIdx.y, n_rb = gridDim.x, n_ks = gridDim.y;
+    const int j = rb * kHeadRows + warp;
     const int d_in = p.d_ext + p.d_attn;
+    const int k0 = ks * kHeadKT;
+    // this lane's 16 weights of row j: features k0 + c*128 + lane*4 + e
+    float w[4][4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const int i = k0 + c * 128 + lane * 4;
+        if (j < p.d_hidden && p.vec4 && i < d_in) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(p.W1 + (size_t)j * d_in + i));
+            w[c][0] = v.x; w[c][1] = v.y; w[c][2] = v.z; w[c][3] = v.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                w[c][e] = (j < p.d_hidden && i + e < d_in) ? __ldg(p.W1 + (size_t)j * d_in + i + e) : 0.f;
+        }
+    }
     for (int b0 = 0; b0 < p.batch; b0 += kHeadBT) {
+        if (b0) __syncthreads();
+        // stage x[b0 .. b0+16)[k0 .. k0+512): every load of the tile is in flight together
+        if (p.vec4) {
+#pragma unroll
+            for (int t = 0; t < kHeadBT * kHeadKT / 4 / kHeadThreads; ++t) {
+                const int idx = tid + t * kHeadThreads;
+                const int u = idx / (kHeadKT / 4), q = idx - u * (kHeadKT / 4);
+                const bool ok = b0 + u < p.batch && k0 + q * 4 < d_in;
+                reinterpret_cast<float4*>(&s_x[u][0])[q] =
+                    ok ? head_x4(p, b0 + u, k0 + q * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        } else {
+            for (int idx = tid; idx < kHeadBT * kHeadKT; idx += kHeadThreads) {
+                const int u = idx / kHeadKT, i = idx - u * kHeadKT;
+                s_x[u][i] = (b0 + u < p.batch && k0 + i < d_in) ? head_x(p, b0 + u, k0 + i) : 0.f;
+            }
+        }
+        __syncthreads();
         float acc[kHeadBT];
 #pragma unroll
-        for (int u = 0; u < kHeadBT; ++u) acc[u] = 0.f;
-        if (j < p.d_hidden) {
-            const float* wrow = p.W1 + (size_t)j * d_in;
-            for (int i = lane; i < d_in; i += 32) {
-                const float w = __ldg(wrow + i);
+        for (int u = 0; u < kHeadBT; ++u) {
+            float a = 0.f;
 #pragma unroll
-                for (int u = 0; u < kHeadBT; ++u)
-                    if (b0 + u < p.batch) acc[u] = fmaf(w, head_x(p, b0 + u, i), acc[u]);
+            for (int c = 0; c < 4; ++c) {
+                const float4 x = reinterpret_cast<const float4*>(&s_x[u][0])[c * 32 + lane];
+                a = fmaf(w[c][0], x.x, a);
+                a = fmaf(w[c][1], x.y, a);
+                a = fmaf(w[c][2], x.z, a);
+                a = fmaf(w[c][3], x.w, a);
             }
+            acc[u] = a;
         }
 #pragma unroll
         for (int u = 0; u < kHeadBT; ++u) {
             float a = acc[u];
             for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-            if (lane == 0 && b0 + u < p.batch) {
-                float hv = 0.f;
-                if (j < p.d_hidden) {
-                    a += __ldg(p.b1 + j);
-                    hv = __ldg(p.w2 + j) * (a / (1.f + expf(-a)));
-                }
-                s_h[warp][b0 + u] = hv;
-            }
+            if (lane == 0 && b0 + u < p.batch && j < p.d_hidden)
+                __stcg(p.pre + ((size_t)ks * p.d_hidden + j) * p.max_batch + b0 + u, a);
         }
     }
-    __syncthreads();
-    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) {
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < kHeadWarps; ++w) s += s_h[w][b];
-        __stcg(p.partial + (size_t)blockIdx.x * p.max_batch + b, s);
-    }
+    // ---- row block complete?  (last of its n_ks K slices)
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int old = atomicAdd(p.ticket, 1);
-        s_last = (old == (int)gridDim.x - 1);
+    if (tid == 0) {
+        const int old = atomicAdd(p.rb_tickets + rb, 1);
+        s_last = (old == n_ks - 1);
+        if (s_last) p.rb_tickets[rb] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
+        const int r = e / p.batch, b = e - r * p.batch;
+        const int jj = rb * kHeadRows + r;
+        float hv = 0.f;
+        if (jj < p.d_hidden) {
+            float a = __ldg(p.b1 + jj);
+            for (int s = 0; s < n_ks; ++s) a += __ldcg(p.pre + ((size_t)s * p.d_hidden + jj) * p.max_batch + b);
+            hv = __ldg(p.w2 + jj) * (a / (1.f + expf(-a)));
+        }
+        s_h[r][b] = hv;
+    }
+    __syncthreads();
+    for (int b = tid; b < p.batch; b += kHeadThreads) {
+        float s = 0.f;
+#pragma unroll
+        for (int r = 0; r < kHeadRows; ++r) s += s_h[r][b];
+        __stcg(p.partial + (size_t)rb * p.max_batch + b, s);
+    }
+    // ---- head complete?  (last of the n_rb row blocks)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int old = atomicAdd(p.ticket, 1);
+        s_last = (old == n_rb - 1);
         if (s_last) *p.ticket = 0;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) {
-        float z = __ldg(p.b2);
-        for (int c = 0; c < (int)gridDim.x; ++c) z += __ldcg(p.partial + (size_t)c * p.max_batch + b);
-        const float score = 1.f / (1.f + expf(-z));
-        uint8_t f;
-        if (p.override_flags)
-            f = p.override_flags[b] ? 1 : 0;
-        else
-            f = (!isfinite(z) || score > p.threshold) ? 1 : 0;
-        p.scores[b] = score;
-        if (p.logits) p.logits[b] = z;
-        p.flags[b] = f;
-        if (p.counters) {
-            p.counters[2 * b] += 1;
-            p.counters[2 * b + 1] += f;
+    // one warp per request: lanes take the row blocks' sums 32 apart, then a fixed shuffle tree
+    for (int b = warp; b < p.batch; b += kHeadRows) {
+        float zp = 0.f;
+        for (int c = lane; c < n_rb; c += 32) zp += __ldcg(p.partial + (size_t)c * p.max_batch + b);
+        for (int o = 16; o; o >>= 1) zp += __shfl_xor_sync(0xffffffffu, zp, o);
+        if (lane == 0) {
+            const float z = __ldg(p.b2) + zp;
+            const float score = 1.f / (1.f + expf(-z));
+            uint8_t f;
+            if (p.override_flags)
+                f = p.override_flags[b] ? 1 : 0;
+            else
+                f = (!isfinite(z) || score > p.threshold) ? 1 : 0;
+            p.scores[b] = score;
+            if (p.logits) p.logits[b] = z;
+            p.flags[b] = f;
+            if (p.counters) {
+                p.counters[2 * b] += 1;
+                p.counters[2 * b + 1] += f;
+            }
         }
     }
 }
@@ -119,14 +199,16 @@ __global__ void advance_seq_lens_kernel(int32_t* seq_lens, int batch)
     for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < batch; b += gridDim.x * blockDim.x) seq_lens[b] += 1;
 }
 
-int recall_head_grid(int d_hidden) { return (d_hidden + kHeadWarps - 1) / kHeadWarps; }
+int recall_head_grid(int d_hidden) { return (d_hidden + kHeadRows - 1) / kHeadRows; }
+int recall_head_ksplits(int d_in) { return d_in > 0 ? (d_in + kHeadKT - 1) / kHeadKT : 1; }
 
 cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl)
 {
     if (p.d_hidden <= 0)
         return launch_ex(copy_flags_kernel, dim3(1), dim3(128), 0, st, pdl, p.override_flags, p.flags, p.scores,
                          p.logits, p.counters, p.batch);
-    return launch_ex(recall_head_kernel, dim3(recall_head_grid(p.d_hidden)), dim3(kHeadWarps * 32), 0, st, pdl, p);
+    return launch_ex(recall_head_kernel, dim3(recall_head_grid(p.d_hidden), recall_head_ksplits(p.d_ext + p.d_attn)),
+                     dim3(kHeadThreads), 0, st, pdl, p);
 }
 
 cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st, bool pdl)
