@@ -95,7 +95,7 @@ void compute_layout(oda_ctx* c)
     w.sm_claims = take(1024 * sizeof(int32_t));
     w.sm_bytes = take(2 * 1024 * sizeof(unsigned long long));
     w.cum_share = take((kMaxGrid + 1) * sizeof(uint16_t));
-    w.partials = take((size_t)c->max_items * c->group * (D + kPartHdr) * sizeof(float));
+    w.partials = take((size_t)c->max_items * std::max<size_t>(c->group * (D + kPartHdr), tma_partial_slot_floats()) * sizeof(float));
     w.st_q_local = take(L * B * Hq * D * 2);
     w.st_q_full = take(L * B * Hq * D * 2);
     w.st_feat = take(B * (size_t)(f.head_d_ext > 0 ? f.head_d_ext : 1) * 4);

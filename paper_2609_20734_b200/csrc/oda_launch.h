@@ -18,6 +18,7 @@ bool encode_kv_map(void* out_map, const void* base, int head_dim, int num_kv_hea
 cudaError_t launch_splitkv_tma(const AttnParams& p, const void* kmap, const void* vmap, int blocks_per_layer,
                                int head_dim, int group, int grid, cudaStream_t st, bool pdl = false);
 int occupancy_splitkv_tma(int head_dim, int group);
+int tma_partial_slot_floats();
 
 
 struct HeadParams {

@@ -32,6 +32,9 @@ extern "C" int oda_debug_timeline(unsigned long long* host, int n) { return (int
 #endif
 
 constexpr int kMaxStages = 6;
+// a partial of the TMA variant: the epilogue warp's fragment, 9 rows of one float4 per lane
+// (8 rows of O^T accumulators, 1 row of (m, l) pairs)
+constexpr int kFragSlotFloats = 9 * 32 * 4;
 
 struct EpiMeta {  // what the epilogue warp needs to know about a finished item
     int32_t layer, b, g, chunk, nchunks, slot_base, valid, pad;
@@ -326,11 +329,42 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
 
     if (warp == C::kEpilogueWarp) {
         // ============================ epilogue warp ============================
-        // Fragment layout of the item it receives (same as the consumers' accumulators):
-        // o[n][0..1]: d = 16n + hrow, heads qc, qc+1;  o[n][2..3]: d = 16n + 8 + hrow.
+        // It receives each finished item in the consumers' fragment layout
+        //   o[n][0..1]: d = 16n + hrow, heads qc, qc+1;  o[n][2..3]: d = 16n + 8 + hrow;
+        //   ml = (m, l) of head qc, (m, l) of head qc+1,
+        // and keeps partials in global memory in the same layout (one float4 per lane and row), so
+        // that the CTA that completes a unit folds the other chunks into registers with coalesced
+        // 128-bit loads and stores the result straight from the fragment.
         const int hrow = lane >> 2, qc = (lane & 3) * 2;
-        constexpr int W = D + kPartHdr;
         const float kLn2 = 0.6931471805599453f;
+        auto store_final = [&](const Item& it, const float (&o)[D / 16][4], const float4& ml) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int hg = qc + e;
+                if (hg >= G) continue;
+                const float mm = e ? ml.z : ml.x, ll = e ? ml.w : ml.y;
+                const float inv = 1.f / ll;
+                const int h = it.g * G + hg;
+                const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + hrow;
+                if (p.out_bf16) {
+                    __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) + idx;
+#pragma unroll
+                    for (int n = 0; n < D / 16; ++n) {
+                        ob[n * 16] = __float2bfloat16_rn(o[n][e] * inv);
+                        ob[n * 16 + 8] = __float2bfloat16_rn(o[n][2 + e] * inv);
+                    }
+                } else {
+                    float* of = reinterpret_cast<float*>(p.out) + idx;
+#pragma unroll
+                    for (int n = 0; n < D / 16; ++n) {
+                        of[n * 16] = o[n][e] * inv;
+                        of[n * 16 + 8] = o[n][2 + e] * inv;
+                    }
+                }
+                if (p.lse && hrow == 0)
+                    p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] = (mm + log2f(ll)) * kLn2;
+            }
+        };
         for (uint32_t k = 0;; ++k) {
             if (!mbar_wait(efull, k & 1, abort_flag, p.status)) break;
             const EpiMeta m = ctl.meta;
@@ -347,46 +381,14 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             Item it;
             it.layer = m.layer; it.b = m.b; it.g = m.g; it.chunk = m.chunk; it.nchunks = m.nchunks;
             it.slot_base = m.slot_base;
+            if (it.nchunks == 1) {
+                store_final(it, o, ml);
+            } else {
+                float4* slots = reinterpret_cast<float4*>(p.partials) + (size_t)it.slot_base * (kFragSlotFloats / 4);
+                float4* mine = slots + (size_t)it.chunk * (kFragSlotFloats / 4);
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int hg = qc + e;
-                if (hg >= G) continue;
-                const float mm = e ? ml.z : ml.x, ll = e ? ml.w : ml.y;
-                if (it.nchunks == 1) {
-                    const float inv = 1.f / ll;
-                    const int h = it.g * G + hg;
-                    const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + hrow;
-                    if (p.out_bf16) {
-                        __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) + idx;
-#pragma unroll
-                        for (int n = 0; n < D / 16; ++n) {
-                            ob[n * 16] = __float2bfloat16_rn(o[n][e] * inv);
-                            ob[n * 16 + 8] = __float2bfloat16_rn(o[n][2 + e] * inv);
-                        }
-                    } else {
-                        float* of = reinterpret_cast<float*>(p.out) + idx;
-#pragma unroll
-                        for (int n = 0; n < D / 16; ++n) {
-                            of[n * 16] = o[n][e] * inv;
-                            of[n * 16 + 8] = o[n][2 + e] * inv;
-                        }
-                    }
-                    if (p.lse && hrow == 0)
-                        p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] = (mm + log2f(ll)) * kLn2;
-                } else {
-                    float* slot = partial_slot(p, it, G, W) + hg * W;
-                    if (hrow == 0) {
-                        __stcg(slot, mm);
-                        __stcg(slot + 1, ll);
-                    }
-#pragma unroll
-                    for (int n = 0; n < D / 16; ++n) {
-                        __stcg(slot + kPartHdr + n * 16 + hrow, o[n][e]);
-                        __stcg(slot + kPartHdr + n * 16 + 8 + hrow, o[n][2 + e]);
-                    }
-                }
-            }
-            if (it.nchunks > 1) {
+                for (int n = 0; n < D / 16; ++n) __stcg(mine + n * 32 + lane, make_float4(o[n][0], o[n][1], o[n][2], o[n][3]));
+                __stcg(mine + 8 * 32 + lane, ml);
                 __threadfence();
                 __syncwarp();
                 int last = 0;
@@ -394,7 +396,63 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 last = __shfl_sync(0xffffffffu, last, 0);
                 if (last) {
                     __threadfence();
-                    merge_chunks<D, G>(p, it, lane, 32);
+                    // fold the chunks in index order (this CTA's own chunk comes from its registers);
+                    // the next chunk is in flight while the current one is folded
+                    float ro[D / 16][4], no[D / 16][4];
+                    float4 rml = make_float4(0.f, 0.f, 0.f, 0.f), nml = rml;
+                    auto fetch = [&](int c) {
+                        if (c >= it.nchunks) return;
+                        if (c == it.chunk) {
+#pragma unroll
+                            for (int n = 0; n < D / 16; ++n) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) no[n][e] = o[n][e];
+                            }
+                            nml = ml;
+                        } else {
+                            const float4* src = slots + (size_t)c * (kFragSlotFloats / 4);
+#pragma unroll
+                            for (int n = 0; n < D / 16; ++n) {
+                                const float4 v = __ldcg(src + n * 32 + lane);
+                                no[n][0] = v.x; no[n][1] = v.y; no[n][2] = v.z; no[n][3] = v.w;
+                            }
+                            nml = __ldcg(src + 8 * 32 + lane);
+                        }
+                    };
+                    fetch(0);
+#pragma unroll 1
+                    for (int c = 0; c < it.nchunks; ++c) {
+                        float co[D / 16][4];
+#pragma unroll
+                        for (int n = 0; n < D / 16; ++n) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) co[n][e] = no[n][e];
+                        }
+                        const float4 cml = nml;
+                        fetch(c + 1);
+                        if (c == 0) {
+#pragma unroll
+                            for (int n = 0; n < D / 16; ++n) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) ro[n][e] = co[n][e];
+                            }
+                            rml = cml;
+                        } else {
+                            const float MA = fmaxf(rml.x, cml.x), MB = fmaxf(rml.z, cml.z);
+                            const float muA = (MA == -INFINITY) ? 0.f : MA, muB = (MB == -INFINITY) ? 0.f : MB;
+                            const float saA = ex2(rml.x - muA), sbA = ex2(cml.x - muA);
+                            const float saB = ex2(rml.z - muB), sbB = ex2(cml.z - muB);
+#pragma unroll
+                            for (int n = 0; n < D / 16; ++n) {
+                                ro[n][0] = ro[n][0] * saA + co[n][0] * sbA;
+                                ro[n][1] = ro[n][1] * saB + co[n][1] * sbB;
+                                ro[n][2] = ro[n][2] * saA + co[n][2] * sbA;
+                                ro[n][3] = ro[n][3] * saB + co[n][3] * sbB;
+                            }
+                            rml = make_float4(MA, rml.y * saA + cml.y * sbA, MB, rml.w * saB + cml.w * sbB);
+                        }
+                    }
+                    store_final(it, ro, rml);
                 }
             }
             ODA_TL(6);
@@ -714,6 +772,8 @@ cudaError_t launch_splitkv_tma(const AttnParams& p, const void* kmap, const void
     ODA_DISPATCH_DG(head_dim, group, e = (launch_tma_t<DD, GG>(p, kmap, vmap, blocks_per_layer, grid, st, pdl)));
     return e;
 }
+
+int tma_partial_slot_floats() { return kFragSlotFloats; }
 
 int occupancy_splitkv_tma(int head_dim, int group)
 {
