@@ -127,7 +127,8 @@ oda_status_t check_attn_args(oda_ctx* c, int lb, int le, int batch, const void* 
 oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, const void* q,
                               const void* k, const void* v, const int32_t* bt, const int32_t* sl,
                               const uint8_t* flags, void* out, float* lse, cudaStream_t st,
-                              int32_t* advance = nullptr, bool* advanced = nullptr)
+                              int32_t* advance = nullptr, bool* advanced = nullptr,
+                              const oda_step_args_t* publish = nullptr)
 {
     const oda_config_t& f = c->cfg;
     AttnParams p;
@@ -173,6 +174,12 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     }
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
     p.advance_seq_lens = advance;
+    if (publish) {
+        p.flags_out = publish->flags;
+        p.scores_out = publish->scores;
+        p.logits_out = publish->logits;
+        p.counters_out = publish->counters;
+    }
     p.done_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 128);
     p.exit_counter = reinterpret_cast<int32_t*>(c->ws + c->lay.status + 192);
     p.num_sms = c->num_sms;
@@ -498,14 +505,20 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     const char* attn_last = nullptr;
     if (c->last_gated >= 0 && f.head_use_attn_out)
         attn_last = static_cast<const char*>(a->out) + (size_t)c->last_gated * B * f.num_q_heads * f.head_dim * out_elem(c);
-    s = oda_recall_score(c, B, a->feat_ext, attn_last, a->W1, a->b1, a->w2, a->b2, a->threshold,
-                         a->override_flags, a->scores, a->logits, a->flags, a->counters, stream);
-    if (s != ODA_OK) return s;
+    // Without a head the decision is the caller's forced flags: the Full kernel reads them
+    // directly and publishes them, which saves the decision kernel's launch.
+    const bool fused_decision = f.head_d_hidden == 0 && c->last_gated >= 0;
+    if (!fused_decision) {
+        s = oda_recall_score(c, B, a->feat_ext, attn_last, a->W1, a->b1, a->w2, a->b2, a->threshold,
+                             a->override_flags, a->scores, a->logits, a->flags, a->counters, stream);
+        if (s != ODA_OK) return s;
+    }
     bool advanced = false;
     if (c->last_gated >= 0) {
         // the Full kernel is the last reader of seq_lens in the step: it also advances them
         s = launch_attention(c, 1, 0, L, B, qf, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
-                             a->flags, a->out, a->lse, st, a->advance_seq_lens ? a->seq_lens : nullptr, &advanced);
+                             fused_decision ? a->override_flags : a->flags, a->out, a->lse, st,
+                             a->advance_seq_lens ? a->seq_lens : nullptr, &advanced, fused_decision ? a : nullptr);
         if (s != ODA_OK) return s;
     }
     if (a->advance_seq_lens && !advanced) {

@@ -47,6 +47,12 @@ struct AttnParams {
     int32_t cls_layers_in_call[kMaxClasses];
     int32_t* advance_seq_lens;  // nullable: seq_lens to increment once every CTA has read them
     int32_t* done_counter;      // zero between launches
+    // Full pass of a step without a recall head: `flags` are the caller's forced flags, and the
+    // CTA that finishes the plan last also publishes them as the step's decision (nullable).
+    uint8_t* flags_out;
+    float* scores_out;
+    float* logits_out;
+    int32_t* counters_out;
     // Optional per-SM weighting of the split (oda_calibrate): cum_share[v] / 65536 is the part of
     // the page axis that lies before span v; spans 2*sm and 2*sm+1 belong to SM `sm`.  nullptr =>
     // equal spans, span = blockIdx.x.
@@ -253,12 +259,25 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     __syncthreads();
     // Every CTA now works from its shared-memory copy of seq_lens.  If the step asked for it, the
     // CTA that gets here last moves the device-side lengths on (no CTA reads them again).
-    if (p.advance_seq_lens && tid == 0) {
+    if ((p.advance_seq_lens || p.flags_out) && tid == 0) {
         __threadfence();
         const int old = atomicAdd(p.done_counter, 1);
         if (old == (int)gridDim.x - 1) {
             *p.done_counter = 0;
-            for (int b = 0; b < B; ++b) p.advance_seq_lens[b] += 1;
+            if (p.advance_seq_lens)
+                for (int b = 0; b < B; ++b) p.advance_seq_lens[b] += 1;
+            if (p.flags_out) {
+                for (int b = 0; b < B; ++b) {
+                    const uint8_t f = pl.active[b] ? 1 : 0;
+                    p.flags_out[b] = f;
+                    if (p.scores_out) p.scores_out[b] = 0.5f;
+                    if (p.logits_out) p.logits_out[b] = 0.f;
+                    if (p.counters_out) {
+                        p.counters_out[2 * b] += 1;
+                        p.counters_out[2 * b + 1] += f;
+                    }
+                }
+            }
         }
     }
     // Every CTA has made its claim(s) by now; the one that notes this last re-arms the table.
