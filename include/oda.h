@@ -161,6 +161,21 @@ oda_status_t oda_full_decode_gated(oda_ctx_t* ctx, int32_t layer_begin, int32_t 
                                    const int32_t* seq_lens, const uint8_t* flags, void* out,
                                    float* lse, void* stream);
 
+/*
+ * Commit of the current token (Algorithm 1, line 8; the fused KV commitment of the appendix on
+ * selected-state execution): for every layer and every request with mask[b] != 0 (mask NULL =
+ * all), writes k_cur/v_cur[l,b,:,:] ([L,B,Hkv,D] bf16) into the paged cache at position
+ * seq_lens[b]-1.  One launch for all layers.  A request with seq_len < 1 or beyond the block
+ * table sets the device status word and is skipped.
+ */
+oda_status_t oda_write_current_kv(oda_ctx_t* ctx, int32_t batch, const void* k_cur, const void* v_cur,
+                                  const uint8_t* mask, void* k_cache, void* v_cache,
+                                  const int32_t* block_table, const int32_t* seq_lens, void* stream);
+/* Selected-state rule for per-request rows (h_t = h_t^{b_t}): out[b] = flags[b] ? full[b] : local[b];
+ * rows of row_bytes bytes (a multiple of 16), 16-byte aligned device pointers. */
+oda_status_t oda_select_rows(oda_ctx_t* ctx, int32_t batch, const void* local, const void* full,
+                             const uint8_t* flags, void* out, int64_t row_bytes, void* stream);
+
 typedef struct {
     int32_t batch;
     int32_t advance_seq_lens; /* 1 => seq_lens[b] += 1 on the device at the end of the step */
@@ -181,10 +196,22 @@ typedef struct {
     float* logits;            /* [B] nullable */
     uint8_t* flags;           /* [B] */
     int32_t* counters;        /* [B,2] nullable */
+    /* Optional selected-state commit (Algorithm 1, line 8).  If k_cur_local/v_cur_local
+     * ([L,B,Hkv,D] bf16, the Local branch's K/V of the current token) are given, the step first
+     * writes them at position seq_len-1 of every request; if k_cur_full/v_cur_full are given, the
+     * Full branch's candidates replace them for the requests that recall, before the Full pass:
+     * the cache then holds the selected candidate.  k_cache/v_cache must be writable.  If
+     * hidden_out is given, hidden_out[b] = flag ? hidden_full[b] : hidden_local[b]
+     * (rows of hidden_row_bytes bytes, a multiple of 16). */
+    const void *k_cur_local, *v_cur_local, *k_cur_full, *v_cur_full;
+    const void *hidden_local, *hidden_full;
+    void* hidden_out;
+    int64_t hidden_row_bytes;
 } oda_step_args_t;
 
-/* One whole step (Algorithm 1, lines 1-7): Local on all layers -> recall score on the last
- * gated layer's Local output -> flags -> gated Full -> optional seq_lens advance. */
+/* One whole step (Algorithm 1, lines 1-7, and line 8 when the commit fields are given): Local on
+ * all layers -> recall score on the last gated layer's Local output -> flags -> gated Full ->
+ * optional seq_lens advance. */
 oda_status_t oda_step(oda_ctx_t* ctx, const oda_step_args_t* args, void* stream);
 
 /*

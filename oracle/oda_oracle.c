@@ -32,6 +32,9 @@
  * output of the last gated layer], score = sigmoid(z), flag = override if one
  * is given, else (z nonfinite) or (score > threshold), strictly.
  *
+ * Algorithm 1, line 8 (commit of the selected candidate) is oda_oracle_write_current_kv +
+ * oda_oracle_select_rows, composed into a step by step_with_commit() of the wrapper.
+ *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py
  * (brute force over literal 1-based sets in extended precision, an independent
  * masked-attention library routine, closed forms, set identities quoted from
@@ -299,6 +302,51 @@ int oda_oracle_step(const oracle_shape_t *sh, const int32_t *layer_window,
     free(z);
     free(score);
     return rc;
+}
+
+/*
+ * Commit of the current token (Algorithm 1, line 8, C_t = C_{t-1} || dC_t; "fused commitment"
+ * paragraph of the appendix on selected-state execution): for every layer and every request
+ * with mask[b] != 0 (mask NULL = every request), the K and V vectors of the current token are
+ * written into the paged cache at position seq_len - 1.  k_cur, v_cur: [L,B,Hkv,D] bf16 bits.
+ * Used twice in a step: the Local candidate for every request before the Local pass, and the
+ * Full candidate of the requests that recall before the Full pass (the selected candidate is
+ * then the one the cache keeps).
+ */
+int oda_oracle_write_current_kv(const oracle_shape_t *sh, const int32_t *layer_kv_index,
+                                const uint16_t *k_cur, const uint16_t *v_cur, const uint8_t *mask,
+                                uint16_t *k_cache, uint16_t *v_cache, const int32_t *block_table,
+                                const int32_t *seq_lens)
+{
+    if (!sh || !k_cur || !v_cur || !k_cache || !v_cache || !block_table || !seq_lens) return -1;
+    const int L = sh->num_layers, B = sh->batch, H = sh->num_kv_heads, D = sh->head_dim;
+    for (int l = 0; l < L; ++l) {
+        const int kvl = layer_kv_index ? layer_kv_index[l] : l;
+        for (int b = 0; b < B; ++b) {
+            if (mask && !mask[b]) continue;
+            const int t = seq_lens[b];
+            if (t < 1) return -1;
+            for (int g = 0; g < H; ++g) {
+                const int64_t src = (((int64_t)l * B + b) * H + g) * D;
+                /* same addressing as the reads: position t-1 of request b */
+                uint16_t *kd = (uint16_t *)kv_row(sh, k_cache, kvl, block_table, b, t - 1, g);
+                uint16_t *vd = (uint16_t *)kv_row(sh, v_cache, kvl, block_table, b, t - 1, g);
+                memcpy(kd, k_cur + src, sizeof(uint16_t) * (size_t)D);
+                memcpy(vd, v_cur + src, sizeof(uint16_t) * (size_t)D);
+            }
+        }
+    }
+    return 0;
+}
+
+/* Selected-state rule for a per-request row (h_t = h_t^{b_t}): out[b] = flags[b] ? full[b] : local[b]. */
+int oda_oracle_select_rows(int batch, int64_t row_bytes, const uint8_t *local, const uint8_t *full,
+                           const uint8_t *flags, uint8_t *out)
+{
+    if (batch < 0 || row_bytes < 0 || !local || !full || !flags || !out) return -1;
+    for (int b = 0; b < batch; ++b)
+        memcpy(out + (int64_t)b * row_bytes, (flags[b] ? full : local) + (int64_t)b * row_bytes, (size_t)row_bytes);
+    return 0;
 }
 
 int oda_oracle_max_threads(void)

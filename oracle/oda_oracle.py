@@ -60,6 +60,8 @@ def lib():
         _lib.oda_oracle_flags.restype = ctypes.c_int
         _lib.oda_oracle_step.restype = ctypes.c_int
         _lib.oda_oracle_max_threads.restype = ctypes.c_int
+        _lib.oda_oracle_write_current_kv.restype = ctypes.c_int
+        _lib.oda_oracle_select_rows.restype = ctypes.c_int
     return _lib
 
 
@@ -257,3 +259,85 @@ def step(q_local: np.ndarray, q_full: Optional[np.ndarray], k_cache: np.ndarray,
     if rc:
         raise ValueError(f"oda_oracle_step rejected its arguments ({rc})")
     return StepResult(out, lse, out_l, lse_l, z, score, fl)
+
+
+def write_current_kv(k_cur: np.ndarray, v_cur: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray,
+                     block_table: np.ndarray, seq_lens: np.ndarray, *, block_size: int, layout: KVLayout,
+                     mask: Optional[np.ndarray] = None, layer_kv_index: Optional[Sequence[int]] = None) -> None:
+    """Commit of the current token: k_cur/v_cur [L,B,Hkv,D] (bf16 bits) are written IN PLACE into
+    the flat uint16 caches at position seq_len-1 of every request with mask != 0 (None = all)."""
+    L, B, Hkv, D = k_cur.shape
+    assert k_cache.dtype == np.uint16 and k_cache.flags["C_CONTIGUOUS"] and k_cache.flags["WRITEABLE"]
+    assert v_cache.dtype == np.uint16 and v_cache.flags["C_CONTIGUOUS"] and v_cache.flags["WRITEABLE"]
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32).reshape(B, -1)
+    sh = _Shape(L, B, Hkv, Hkv, D, block_size, block_table.shape[1], 0, layout.layer_stride,
+                layout.block_stride, layout.token_stride, layout.head_stride, 1.0)
+    a = _Args()
+    rc = lib().oda_oracle_write_current_kv(
+        ctypes.byref(sh), a(layer_kv_index, np.int32), a(k_cur, np.uint16), a(v_cur, np.uint16),
+        a(mask, np.uint8), _out(k_cache.reshape(-1), np.uint16), _out(v_cache.reshape(-1), np.uint16),
+        a(block_table, np.int32), a(seq_lens, np.int32))
+    if rc:
+        raise ValueError(f"oda_oracle_write_current_kv rejected its arguments ({rc})")
+
+
+def select_rows(local: np.ndarray, full: np.ndarray, flags: np.ndarray) -> np.ndarray:
+    """Selected-state rule per request: out[b] = flags[b] ? full[b] : local[b]."""
+    assert local.shape == full.shape and local.dtype == full.dtype
+    B = local.shape[0]
+    lo = np.ascontiguousarray(local)
+    fu = np.ascontiguousarray(full)
+    out = np.empty_like(lo)
+    a = _Args()
+    rc = lib().oda_oracle_select_rows(
+        ctypes.c_int(B), ctypes.c_int64(lo.nbytes // max(B, 1)), ctypes.c_void_p(lo.ctypes.data),
+        ctypes.c_void_p(fu.ctypes.data), a(flags, np.uint8), ctypes.c_void_p(out.ctypes.data))
+    if rc:
+        raise ValueError(f"oda_oracle_select_rows rejected its arguments ({rc})")
+    return out
+
+
+@dataclass
+class CommitStepResult:
+    out: np.ndarray
+    out_local: np.ndarray
+    z: np.ndarray
+    score: np.ndarray
+    flags: np.ndarray
+    hidden: Optional[np.ndarray]
+
+
+def step_with_commit(q_local, q_full, k_cache, v_cache, block_table, seq_lens, *, k_cur_local, v_cur_local,
+                     k_cur_full, v_cur_full, num_kv_heads, block_size, layout, layer_window, layer_sinks,
+                     layer_gated, head=None, feat_ext=None, tau=0.5, override_flags=None,
+                     hidden_local=None, hidden_full=None, layer_kv_index=None, nthreads=1) -> CommitStepResult:
+    """Algorithm 1, lines 1-8, on the attention stack, with the current token's K/V supplied as
+    candidates: the Local candidate is written at position seq_len-1 and Local runs; the head
+    decides; for requests that recall, the Full candidate replaces it and Full runs on the gated
+    layers; the selected branch supplies the output, the hidden row, and is what the caches
+    (modified in place) keep."""
+    L, B, Hq, D = q_local.shape
+    kw = dict(num_kv_heads=num_kv_heads, block_size=block_size, layout=layout, layer_window=layer_window,
+              layer_sinks=layer_sinks, layer_kv_index=layer_kv_index, nthreads=nthreads)
+    write_current_kv(k_cur_local, v_cur_local, k_cache, v_cache, block_table, seq_lens,
+                     block_size=block_size, layout=layout, layer_kv_index=layer_kv_index)
+    out_local, _ = attention("local", q_local, k_cache, v_cache, block_table, seq_lens, **kw)
+    gated = [l for l in range(L) if layer_gated[l]]
+    if head is not None:
+        attn = out_local[gated[-1]].reshape(B, -1) if (gated and head.get("use_attn_out", 1)) else None
+        z, score = recall_head(feat_ext, attn, head["W1"], head["b1"], head["w2"], head["b2"])
+    else:
+        z, score = np.zeros(B), np.full(B, 0.5)
+    fl = flags(z, score, tau, override_flags)
+    write_current_kv(k_cur_full, v_cur_full, k_cache, v_cache, block_table, seq_lens, block_size=block_size,
+                     layout=layout, mask=fl, layer_kv_index=layer_kv_index)
+    out = out_local.copy()
+    if fl.any() and gated:
+        full, _ = attention("full", q_full if q_full is not None else q_local, k_cache, v_cache, block_table,
+                            seq_lens, request_mask=fl, **kw)
+        for l in gated:
+            for b in range(B):
+                if fl[b]:
+                    out[l, b] = full[l, b]
+    hidden = None if hidden_local is None else select_rows(hidden_local, hidden_full, fl)
+    return CommitStepResult(out, out_local, z, score, fl, hidden)

@@ -24,6 +24,7 @@ EXPORTS = [
     "oda_read_device_status", "oda_launch_count", "oda_resolved_variant", "oda_attention_grid",
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
+    "oda_write_current_kv", "oda_select_rows",
 ]
 
 
@@ -61,6 +62,10 @@ class _StepArgs(ctypes.Structure):
         ("override_flags", ctypes.c_void_p),
         ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("scores", ctypes.c_void_p),
         ("logits", ctypes.c_void_p), ("flags", ctypes.c_void_p), ("counters", ctypes.c_void_p),
+        ("k_cur_local", ctypes.c_void_p), ("v_cur_local", ctypes.c_void_p),
+        ("k_cur_full", ctypes.c_void_p), ("v_cur_full", ctypes.c_void_p),
+        ("hidden_local", ctypes.c_void_p), ("hidden_full", ctypes.c_void_p), ("hidden_out", ctypes.c_void_p),
+        ("hidden_row_bytes", ctypes.c_int64),
     ]
 
 
@@ -89,6 +94,8 @@ def load_library():
         lib.oda_local_decode_static.argtypes = [i32, i32, i32, i32, i32, i32, f32, ctypes.c_int64,
                                                 ctypes.c_int64, ctypes.c_int64, i32, vp, vp, vp, vp, vp,
                                                 vp, vp, vp]
+        lib.oda_write_current_kv.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oda_select_rows.argtypes = [vp, i32, vp, vp, vp, vp, ctypes.c_int64, vp]
         lib.oda_calibration_begin.argtypes = [vp, vp]
         lib.oda_calibration_end.argtypes = [vp, vp]
         lib.oda_calibration_spread.argtypes = [vp]
@@ -241,17 +248,31 @@ class OdaContext:
             _ptr(block_table), _ptr(seq_lens), _ptr(flags), _ptr(out), _ptr(lse),
             _stream() if stream is None else stream), "oda_full_decode_gated")
 
+    def write_current_kv(self, batch, k_cur, v_cur, mask, k_cache, v_cache, block_table, seq_lens, stream=None):
+        self._check(self.lib.oda_write_current_kv(
+            self._h, batch, _ptr(k_cur), _ptr(v_cur), _ptr(mask), _ptr(k_cache), _ptr(v_cache),
+            _ptr(block_table), _ptr(seq_lens), _stream() if stream is None else stream), "oda_write_current_kv")
+
+    def select_rows(self, batch, local, full, flags, out, stream=None):
+        self._check(self.lib.oda_select_rows(
+            self._h, batch, _ptr(local), _ptr(full), _ptr(flags), _ptr(out),
+            out[0].numel() * out.element_size(), _stream() if stream is None else stream), "oda_select_rows")
+
     @staticmethod
     def step_args(batch, q_local, k_cache, v_cache, block_table, seq_lens, out, scores, flags,
                   q_full=None, feat_ext=None, head=None, threshold=0.5, override_flags=None, lse=None,
-                  logits=None, counters=None, advance_seq_lens=False) -> _StepArgs:
+                  logits=None, counters=None, advance_seq_lens=False, k_cur_local=None, v_cur_local=None,
+                  k_cur_full=None, v_cur_full=None, hidden_local=None, hidden_full=None,
+                  hidden_out=None) -> _StepArgs:
         h = head or {}
+        row_bytes = 0 if hidden_out is None else hidden_out[0].numel() * hidden_out.element_size()
         return _StepArgs(
             batch, 1 if advance_seq_lens else 0, _ptr(q_local), _ptr(q_full), _ptr(k_cache),
             _ptr(v_cache), _ptr(block_table), _ptr(seq_lens), _ptr(feat_ext), _ptr(h.get("W1")),
             _ptr(h.get("b1")), _ptr(h.get("w2")), _ptr(h.get("b2")), float(threshold), 0,
             _ptr(override_flags), _ptr(out), _ptr(lse), _ptr(scores), _ptr(logits), _ptr(flags),
-            _ptr(counters))
+            _ptr(counters), _ptr(k_cur_local), _ptr(v_cur_local), _ptr(k_cur_full), _ptr(v_cur_full),
+            _ptr(hidden_local), _ptr(hidden_full), _ptr(hidden_out), row_bytes)
 
     def step(self, args: _StepArgs, stream=None):
         self._check(self.lib.oda_step(self._h, ctypes.byref(args), _stream() if stream is None else stream),

@@ -485,6 +485,44 @@ oda_status_t oda_recall_score(oda_ctx_t* c, int32_t batch, const float* feat_ext
     return ODA_OK;
 }
 
+oda_status_t oda_write_current_kv(oda_ctx_t* c, int32_t batch, const void* k_cur, const void* v_cur,
+                                  const uint8_t* mask, void* k_cache, void* v_cache, const int32_t* bt,
+                                  const int32_t* sl, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0) return ODA_OK;
+    if (!k_cur || !v_cur || !k_cache || !v_cache || !bt || !sl) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(k_cur) || !aligned16(v_cur) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(c, ODA_ERR_INVALID_ARG, "k_cur, v_cur and the caches must be 16-byte aligned");
+    const oda_config_t& f = c->cfg;
+    cudaError_t e = launch_write_current_kv(
+        k_cur, v_cur, mask, k_cache, v_cache, bt, sl, reinterpret_cast<const LayerInfo*>(c->ws + c->lay.layers),
+        f.num_layers, batch, f.num_kv_heads, f.head_dim, f.max_blocks_per_seq, f.kv_layer_stride, f.kv_block_stride,
+        f.kv_token_stride, f.kv_head_stride, reinterpret_cast<int32_t*>(c->ws + c->lay.status),
+        static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "commit kernel launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
+oda_status_t oda_select_rows(oda_ctx_t* c, int32_t batch, const void* local, const void* full,
+                             const uint8_t* flags, void* out, int64_t row_bytes, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (batch < 0 || row_bytes < 0 || (row_bytes % 16) != 0) return fail(c, ODA_ERR_INVALID_ARG, "bad batch or row size");
+    if (batch == 0 || row_bytes == 0) return ODA_OK;
+    if (!local || !full || !flags || !out) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(local) || !aligned16(full) || !aligned16(out))
+        return fail(c, ODA_ERR_INVALID_ARG, "rows must be 16-byte aligned");
+    cudaError_t e = launch_select_rows(local, full, flags, out, batch, (size_t)row_bytes,
+                                       static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "select kernel launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
 oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
 {
     if (!c || !a) return ODA_ERR_INVALID_ARG;
@@ -499,6 +537,15 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     const void* qf = a->q_full ? a->q_full : a->q_local;
     if (!aligned16(qf)) return fail(c, ODA_ERR_INVALID_ARG, "q_full must be 16-byte aligned");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((a->k_cur_local == nullptr) != (a->v_cur_local == nullptr) || (a->k_cur_full == nullptr) != (a->v_cur_full == nullptr))
+        return fail(c, ODA_ERR_INVALID_ARG, "K and V candidates must be given together");
+    if (a->hidden_out && (!a->hidden_local || !a->hidden_full))
+        return fail(c, ODA_ERR_INVALID_ARG, "hidden_out needs hidden_local and hidden_full");
+    if (a->k_cur_local) {  // the Local candidate of the current token, for every request
+        s = oda_write_current_kv(c, B, a->k_cur_local, a->v_cur_local, nullptr, const_cast<void*>(a->k_cache),
+                                 const_cast<void*>(a->v_cache), a->block_table, a->seq_lens, stream);
+        if (s != ODA_OK) return s;
+    }
     s = launch_attention(c, 0, 0, L, B, a->q_local, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
                          nullptr, a->out, a->lse, st);
     if (s != ODA_OK) return s;
@@ -508,9 +555,19 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     // Without a head the decision is the caller's forced flags: the Full kernel reads them
     // directly and publishes them, which saves the decision kernel's launch.
     const bool fused_decision = f.head_d_hidden == 0 && c->last_gated >= 0;
+    const uint8_t* decided = fused_decision ? a->override_flags : a->flags;  // valid once the head (if any) has run
     if (!fused_decision) {
         s = oda_recall_score(c, B, a->feat_ext, attn_last, a->W1, a->b1, a->w2, a->b2, a->threshold,
                              a->override_flags, a->scores, a->logits, a->flags, a->counters, stream);
+        if (s != ODA_OK) return s;
+    }
+    if (a->k_cur_full) {  // requests that recall keep the Full branch's candidate
+        s = oda_write_current_kv(c, B, a->k_cur_full, a->v_cur_full, decided, const_cast<void*>(a->k_cache),
+                                 const_cast<void*>(a->v_cache), a->block_table, a->seq_lens, stream);
+        if (s != ODA_OK) return s;
+    }
+    if (a->hidden_out) {
+        s = oda_select_rows(c, B, a->hidden_local, a->hidden_full, decided, a->hidden_out, a->hidden_row_bytes, stream);
         if (s != ODA_OK) return s;
     }
     bool advanced = false;
@@ -541,6 +598,8 @@ oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream,
     if (d2h_bytes) *d2h_bytes = 0;
     if (B == 0) return ODA_OK;
     if (!a->q_local || !a->out || !a->scores || !a->flags) return fail(c, ODA_ERR_INVALID_ARG, "null host pointer");
+    if (a->k_cur_local || a->v_cur_local || a->k_cur_full || a->v_cur_full || a->hidden_out)
+        return fail(c, ODA_ERR_INVALID_ARG, "the commit fields take device pointers: use oda_step");
     if (f.head_d_ext > 0 && f.head_d_hidden > 0 && !a->feat_ext) return fail(c, ODA_ERR_INVALID_ARG, "feat_ext is null");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t rows = (size_t)f.num_layers * B * f.num_q_heads;

@@ -21,6 +21,16 @@ int occupancy_splitkv_tma(int head_dim, int group);
 int tma_partial_slot_floats();
 
 
+struct LayerInfo;
+cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const uint8_t* mask, void* k_cache,
+                                    void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
+                                    const LayerInfo* layers, int num_layers, int batch, int num_kv_heads,
+                                    int head_dim, int max_blocks_per_seq, int64_t layer_stride,
+                                    int64_t block_stride, int64_t token_stride, int64_t head_stride,
+                                    int32_t* status, cudaStream_t st, bool pdl = false);
+cudaError_t launch_select_rows(const void* local, const void* full, const uint8_t* flags, void* out, int batch,
+                               size_t row_bytes, cudaStream_t st, bool pdl = false);
+
 struct HeadParams {
     const float* feat_ext;      // [B, d_ext] or nullptr
     const void* attn_out;       // [B, d_attn] fp32 or bf16, or nullptr
