@@ -349,6 +349,120 @@ int oda_oracle_select_rows(int batch, int64_t row_bytes, const uint8_t *local, c
     return 0;
 }
 
+/*
+ * The paper's recall head (appendix "Recall-head architecture"), fp64 on fp32 parameters:
+ *   towers   a, b, c = SiLU(W_i RMSNorm_i(x_i) + b_i)            x_i in R^d_model -> R^d_tower, i = 0,1,2
+ *            (x_0 = preceding selected hidden h_{t-1}, x_1 = embedding E(x_t), x_2 = Local hidden h_t^L)
+ *   u        = [a; b; c; a.b; |a-b|; a.c; |a-c|; b.c; |b-c|]      in R^(9 d_tower)
+ *   z0       = 1/2 [a + b + c + SiLU(W_f u + b_f)]
+ *   blocks   z <- z + W_down( SiLU(W_gate n) . (W_up n) ),  n = RMSNorm(z)   (n_blocks times, no biases)
+ *   q        = w . RMSNorm(z) + bias
+ * RMSNorm(x) = x / sqrt(mean(x^2) + eps) . g.  The paper does not print eps (1e-6 is used by the
+ * callers here) nor the SwiGLU operand order (SiLU on the gate projection, as in the GLU-variants
+ * paper it cites).  Parameter layout in `params`, in this order, all row-major fp32:
+ *   for i in 0..2: g_i[d_model], W_i[d_tower][d_model], b_i[d_tower];
+ *   W_f[d_tower][9 d_tower], b_f[d_tower];
+ *   for k in blocks: g_k[d_tower], W_gate[d_ff][d_tower], W_up[d_ff][d_tower], W_down[d_tower][d_ff];
+ *   g_out[d_tower], w[d_tower], bias[1].
+ * With d_model 2048, d_tower 1024, d_ff 2048 and 2 blocks this is the 28,325,889 parameters the
+ * paper states.
+ */
+int64_t oda_oracle_full_head_param_count(int d_model, int d_tower, int d_ff, int n_blocks)
+{
+    int64_t tower = (int64_t)d_model + (int64_t)d_tower * d_model + d_tower;
+    int64_t fusion = (int64_t)d_tower * 9 * d_tower + d_tower;
+    int64_t block = (int64_t)d_tower + 3ll * d_ff * d_tower;
+    return 3 * tower + fusion + n_blocks * block + 2ll * d_tower + 1;
+}
+
+static void rmsnorm64(const double *x, const float *g, int n, double eps, double *out)
+{
+    double ss = 0.0;
+    for (int i = 0; i < n; ++i) ss += x[i] * x[i];
+    double r = 1.0 / sqrt(ss / n + eps);
+    for (int i = 0; i < n; ++i) out[i] = x[i] * r * (double)g[i];
+}
+
+int oda_oracle_full_head(int batch, int d_model, int d_tower, int d_ff, int n_blocks, double eps,
+                         const float *params, const float *h_prev, const float *emb, const float *h_local,
+                         double *q_out, double *score_out)
+{
+    if (batch < 0 || d_model < 1 || d_tower < 1 || d_ff < 1 || n_blocks < 0 || !params) return -1;
+    if (!h_prev || !emb || !h_local) return -1;
+    const float *inputs[3] = {h_prev, emb, h_local};
+    const int T = d_tower;
+    double *x = (double *)malloc(sizeof(double) * (size_t)(d_model > T ? d_model : T));
+    double *n = (double *)malloc(sizeof(double) * (size_t)(d_model > T ? d_model : T));
+    double *abc = (double *)malloc(sizeof(double) * 3 * (size_t)T);
+    double *u = (double *)malloc(sizeof(double) * 9 * (size_t)T);
+    double *z = (double *)malloc(sizeof(double) * (size_t)T);
+    double *hmid = (double *)malloc(sizeof(double) * (size_t)d_ff);
+    for (int b = 0; b < batch; ++b) {
+        const float *p = params;
+        for (int i = 0; i < 3; ++i) {
+            const float *g = p, *W = p + d_model, *bias = W + (int64_t)T * d_model;
+            for (int k = 0; k < d_model; ++k) x[k] = (double)inputs[i][(int64_t)b * d_model + k];
+            rmsnorm64(x, g, d_model, eps, n);
+            for (int j = 0; j < T; ++j) {
+                double acc = (double)bias[j];
+                for (int k = 0; k < d_model; ++k) acc += (double)W[(int64_t)j * d_model + k] * n[k];
+                abc[i * T + j] = silu(acc);
+            }
+            p = bias + T;
+        }
+        const double *a = abc, *bb = abc + T, *c = abc + 2 * T;
+        for (int j = 0; j < T; ++j) {
+            u[0 * T + j] = a[j];
+            u[1 * T + j] = bb[j];
+            u[2 * T + j] = c[j];
+            u[3 * T + j] = a[j] * bb[j];
+            u[4 * T + j] = fabs(a[j] - bb[j]);
+            u[5 * T + j] = a[j] * c[j];
+            u[6 * T + j] = fabs(a[j] - c[j]);
+            u[7 * T + j] = bb[j] * c[j];
+            u[8 * T + j] = fabs(bb[j] - c[j]);
+        }
+        {
+            const float *Wf = p, *bf = Wf + (int64_t)T * 9 * T;
+            for (int j = 0; j < T; ++j) {
+                double acc = (double)bf[j];
+                for (int k = 0; k < 9 * T; ++k) acc += (double)Wf[(int64_t)j * 9 * T + k] * u[k];
+                z[j] = 0.5 * (a[j] + bb[j] + c[j] + silu(acc));
+            }
+            p = bf + T;
+        }
+        for (int blk = 0; blk < n_blocks; ++blk) {
+            const float *g = p, *Wg = g + T, *Wu = Wg + (int64_t)d_ff * T, *Wd = Wu + (int64_t)d_ff * T;
+            rmsnorm64(z, g, T, eps, n);
+            for (int m = 0; m < d_ff; ++m) {
+                double gate = 0.0, up = 0.0;
+                for (int k = 0; k < T; ++k) {
+                    gate += (double)Wg[(int64_t)m * T + k] * n[k];
+                    up += (double)Wu[(int64_t)m * T + k] * n[k];
+                }
+                hmid[m] = silu(gate) * up;
+            }
+            for (int j = 0; j < T; ++j) {
+                double acc = 0.0;
+                for (int m = 0; m < d_ff; ++m) acc += (double)Wd[(int64_t)j * d_ff + m] * hmid[m];
+                x[j] = z[j] + acc;
+            }
+            for (int j = 0; j < T; ++j) z[j] = x[j];
+            p = Wd + (int64_t)T * d_ff;
+        }
+        {
+            const float *g = p, *w = g + T, *bias = w + T;
+            rmsnorm64(z, g, T, eps, n);
+            double q = (double)bias[0];
+            for (int k = 0; k < T; ++k) q += (double)w[k] * n[k];
+            if (q_out) q_out[b] = q;
+            if (score_out) score_out[b] = 1.0 / (1.0 + exp(-q));
+        }
+    }
+    free(x); free(n); free(abc); free(u); free(z); free(hmid);
+    return 0;
+}
+
 int oda_oracle_max_threads(void)
 {
 #ifdef _OPENMP

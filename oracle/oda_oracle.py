@@ -62,6 +62,8 @@ def lib():
         _lib.oda_oracle_max_threads.restype = ctypes.c_int
         _lib.oda_oracle_write_current_kv.restype = ctypes.c_int
         _lib.oda_oracle_select_rows.restype = ctypes.c_int
+        _lib.oda_oracle_full_head.restype = ctypes.c_int
+        _lib.oda_oracle_full_head_param_count.restype = ctypes.c_int64
     return _lib
 
 
@@ -341,3 +343,26 @@ def step_with_commit(q_local, q_full, k_cache, v_cache, block_table, seq_lens, *
                     out[l, b] = full[l, b]
     hidden = None if hidden_local is None else select_rows(hidden_local, hidden_full, fl)
     return CommitStepResult(out, out_local, z, score, fl, hidden)
+
+
+def full_head_param_count(d_model: int, d_tower: int, d_ff: int, n_blocks: int) -> int:
+    return int(lib().oda_oracle_full_head_param_count(ctypes.c_int(d_model), ctypes.c_int(d_tower),
+                                                      ctypes.c_int(d_ff), ctypes.c_int(n_blocks)))
+
+
+def full_head(params: np.ndarray, h_prev: np.ndarray, emb: np.ndarray, h_local: np.ndarray, *, d_tower: int,
+              d_ff: int, n_blocks: int, eps: float = 1e-6):
+    """The paper's recall head (three towers, interaction vector, fusion, SwiGLU blocks, scalar
+    output) in fp64 on fp32 parameters.  Returns (q, sigmoid(q))."""
+    B, d_model = h_prev.shape
+    assert params.dtype == np.float32 and params.size == full_head_param_count(d_model, d_tower, d_ff, n_blocks)
+    q = np.empty(B)
+    sc = np.empty(B)
+    a = _Args()
+    rc = lib().oda_oracle_full_head(
+        ctypes.c_int(B), ctypes.c_int(d_model), ctypes.c_int(d_tower), ctypes.c_int(d_ff), ctypes.c_int(n_blocks),
+        ctypes.c_double(eps), a(params, np.float32), a(h_prev, np.float32), a(emb, np.float32),
+        a(h_local, np.float32), _out(q, np.float64), _out(sc, np.float64))
+    if rc:
+        raise ValueError(f"oda_oracle_full_head rejected its arguments ({rc})")
+    return q, sc
