@@ -149,6 +149,38 @@ oda_status_t oda_recall_score(oda_ctx_t* ctx, int32_t batch, const float* feat_e
                               uint8_t* flags, int32_t* counters, void* stream);
 
 /*
+ * The paper's own recall head (appendix "Recall-head architecture"; Eq. 2): three
+ * RMSNorm -> Linear(d_model -> d_tower) -> SiLU towers over (h_{t-1}, E(x_t), h_t^L), the interaction
+ * vector u = [a;b;c;a.b;|a-b|;a.c;|a-c|;b.c;|b-c|], z0 = (a+b+c+SiLU(W_f u + b_f))/2, n_blocks
+ * pre-RMSNorm residual SwiGLU blocks (d_tower -> d_ff -> d_tower, no biases), and
+ * q = w . RMSNorm(z) + bias; fp32 weights and arithmetic.  score = sigmoid(q); the decision rule is
+ * that of oda_recall_score (override, else nonfinite q or score > threshold; the paper's theta on q
+ * corresponds to threshold = sigmoid(theta)).  With d_model 2048, d_tower 1024, d_ff 2048 and two
+ * blocks this is the paper's 28,325,889-parameter head.
+ * params (device, 16-byte aligned, row-major fp32), in this order:
+ *   for i in 0..2: gain_i[d_model], W_i[d_tower][d_model], b_i[d_tower];
+ *   W_f[d_tower][9 d_tower], b_f[d_tower];
+ *   per block: gain[d_tower], W_gate[d_ff][d_tower], W_up[d_ff][d_tower], W_down[d_tower][d_ff];
+ *   gain_out[d_tower], w[d_tower], bias[1].
+ * h_prev, emb, h_local: [batch, d_model] fp32 device.  scratch: device, 256-byte aligned, at least
+ * oda_full_head_scratch_bytes(head, batch) bytes, used only during the call.  d_model and d_ff
+ * must be multiples of 4 and d_tower of 8 (else ODA_ERR_UNSUPPORTED).  3 + 2 n_blocks launches.
+ */
+typedef struct {
+    int32_t d_model, d_tower, d_ff, n_blocks;
+    float eps;      /* RMSNorm epsilon (the paper does not print it; 1e-6 is customary) */
+    int32_t pad;
+    const float* params;
+} oda_full_head_t;
+int64_t oda_full_head_param_count(int32_t d_model, int32_t d_tower, int32_t d_ff, int32_t n_blocks);
+size_t oda_full_head_scratch_bytes(const oda_full_head_t* head, int32_t batch);
+oda_status_t oda_recall_score_full(oda_ctx_t* ctx, int32_t batch, const oda_full_head_t* head,
+                                   const float* h_prev, const float* emb, const float* h_local,
+                                   float threshold, const uint8_t* override_flags, float* scores,
+                                   float* logits, uint8_t* flags, int32_t* counters, void* scratch,
+                                   size_t scratch_bytes, void* stream);
+
+/*
  * Gated Full pass (Eq. 1, S^F; Algorithm 1, line 4): for gated layers in [layer_begin,
  * layer_end) and requests with flags[b] != 0, recomputes attention over all t positions and
  * overwrites those rows of out/lse in place; every other row is left untouched.  The work

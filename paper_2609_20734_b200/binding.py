@@ -24,7 +24,8 @@ EXPORTS = [
     "oda_read_device_status", "oda_launch_count", "oda_resolved_variant", "oda_attention_grid",
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
-    "oda_write_current_kv", "oda_select_rows",
+    "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
+    "oda_recall_score_full",
 ]
 
 
@@ -48,6 +49,12 @@ class _Config(ctypes.Structure):
         ("head_d_ext", ctypes.c_int32), ("head_use_attn_out", ctypes.c_int32),
         ("head_d_hidden", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
+
+
+class _FullHead(ctypes.Structure):
+    _fields_ = [("d_model", ctypes.c_int32), ("d_tower", ctypes.c_int32), ("d_ff", ctypes.c_int32),
+                ("n_blocks", ctypes.c_int32), ("eps", ctypes.c_float), ("pad", ctypes.c_int32),
+                ("params", ctypes.c_void_p)]
 
 
 class _StepArgs(ctypes.Structure):
@@ -96,6 +103,12 @@ def load_library():
                                                 vp, vp, vp]
         lib.oda_write_current_kv.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_select_rows.argtypes = [vp, i32, vp, vp, vp, vp, ctypes.c_int64, vp]
+        lib.oda_full_head_param_count.argtypes = [i32, i32, i32, i32]
+        lib.oda_full_head_param_count.restype = ctypes.c_int64
+        lib.oda_full_head_scratch_bytes.argtypes = [ctypes.POINTER(_FullHead), i32]
+        lib.oda_full_head_scratch_bytes.restype = ctypes.c_size_t
+        lib.oda_recall_score_full.argtypes = [vp, i32, ctypes.POINTER(_FullHead), vp, vp, vp, f32, vp, vp, vp, vp,
+                                              vp, vp, ctypes.c_size_t, vp]
         lib.oda_calibration_begin.argtypes = [vp, vp]
         lib.oda_calibration_end.argtypes = [vp, vp]
         lib.oda_calibration_spread.argtypes = [vp]
@@ -195,9 +208,10 @@ class OdaContext:
             self.set_workspace(self.workspace.data_ptr(), self.workspace.numel())
 
     def close(self):
-        if getattr(self, "_h", None) and self._h.value:
-            self.lib.oda_destroy(self._h)
-            self._h = ctypes.c_void_p()
+        h = getattr(self, "_h", None)
+        if h is not None and h.value:
+            self.lib.oda_destroy(h)
+            self._h = None
 
     __del__ = close
 
@@ -247,6 +261,22 @@ class OdaContext:
             self._h, layer_begin, layer_end, batch, _ptr(q_full), _ptr(k_cache), _ptr(v_cache),
             _ptr(block_table), _ptr(seq_lens), _ptr(flags), _ptr(out), _ptr(lse),
             _stream() if stream is None else stream), "oda_full_decode_gated")
+
+    def recall_score_full(self, batch, params, d_tower, d_ff, n_blocks, h_prev, emb, h_local, threshold,
+                          override_flags, scores, logits, flags, counters=None, eps=1e-6, scratch=None,
+                          stream=None):
+        """The paper's full recall head; `params` is the flat fp32 parameter tensor (see oda.h)."""
+        import torch
+
+        head = _FullHead(h_prev.shape[1], d_tower, d_ff, n_blocks, eps, 0, _ptr(params))
+        need = self.lib.oda_full_head_scratch_bytes(ctypes.byref(head), batch)
+        if scratch is None:
+            scratch = torch.empty(need, dtype=torch.uint8, device=h_prev.device)
+        self._check(self.lib.oda_recall_score_full(
+            self._h, batch, ctypes.byref(head), _ptr(h_prev), _ptr(emb), _ptr(h_local), float(threshold),
+            _ptr(override_flags), _ptr(scores), _ptr(logits), _ptr(flags), _ptr(counters), _ptr(scratch),
+            scratch.numel(), _stream() if stream is None else stream), "oda_recall_score_full")
+        return scratch
 
     def write_current_kv(self, batch, k_cur, v_cur, mask, k_cache, v_cache, block_table, seq_lens, stream=None):
         self._check(self.lib.oda_write_current_kv(

@@ -523,6 +523,46 @@ oda_status_t oda_select_rows(oda_ctx_t* c, int32_t batch, const void* local, con
     return ODA_OK;
 }
 
+int64_t oda_full_head_param_count(int32_t d_model, int32_t d_tower, int32_t d_ff, int32_t n_blocks)
+{
+    if (d_model < 1 || d_tower < 1 || d_ff < 1 || n_blocks < 0) return 0;
+    return full_head_param_count(d_model, d_tower, d_ff, n_blocks);
+}
+
+size_t oda_full_head_scratch_bytes(const oda_full_head_t* h, int32_t batch)
+{
+    if (!h || batch < 1) return 0;
+    return full_head_scratch_bytes(h->d_model, h->d_tower, h->d_ff, batch);
+}
+
+oda_status_t oda_recall_score_full(oda_ctx_t* c, int32_t batch, const oda_full_head_t* h, const float* h_prev,
+                                   const float* emb, const float* h_local, float threshold,
+                                   const uint8_t* override_flags, float* scores, float* logits, uint8_t* flags,
+                                   int32_t* counters, void* scratch, size_t scratch_bytes, void* stream)
+{
+    if (!c || !h) return ODA_ERR_INVALID_ARG;
+    if (batch < 0 || batch > kMaxBatch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, 128]");
+    if (batch == 0) return ODA_OK;
+    if (h->d_model < 4 || h->d_tower < 8 || h->d_ff < 4 || h->n_blocks < 0 || !(h->eps >= 0.f))
+        return fail(c, ODA_ERR_INVALID_ARG, "bad head dimensions");
+    if ((h->d_model % 4) || (h->d_tower % 8) || (h->d_ff % 4))
+        return fail(c, ODA_ERR_UNSUPPORTED, "d_model and d_ff must be multiples of 4, d_tower of 8");
+    if (!h->params || !h_prev || !emb || !h_local || !scores || !flags || !scratch)
+        return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(h->params) || !aligned16(h_prev) || !aligned16(emb) || !aligned16(h_local) ||
+        (reinterpret_cast<uintptr_t>(scratch) % 256) != 0)
+        return fail(c, ODA_ERR_INVALID_ARG, "parameters and inputs must be 16-byte aligned, scratch 256-byte aligned");
+    if (scratch_bytes < full_head_scratch_bytes(h->d_model, h->d_tower, h->d_ff, batch))
+        return fail(c, ODA_ERR_WORKSPACE, "scratch smaller than oda_full_head_scratch_bytes()");
+    int launches = 0;
+    cudaError_t e = launch_full_head(batch, h->d_model, h->d_tower, h->d_ff, h->n_blocks, h->eps, h->params, h_prev,
+                                     emb, h_local, threshold, override_flags, scores, logits, flags, counters,
+                                     scratch, static_cast<cudaStream_t>(stream), c->use_pdl, &launches);
+    c->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(c, e, "full recall head launch");
+    return ODA_OK;
+}
+
 oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
 {
     if (!c || !a) return ODA_ERR_INVALID_ARG;

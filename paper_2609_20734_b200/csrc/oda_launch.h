@@ -21,6 +21,14 @@ int occupancy_splitkv_tma(int head_dim, int group);
 int tma_partial_slot_floats();
 
 
+long long full_head_param_count(int d_model, int d_tower, int d_ff, int n_blocks);
+size_t full_head_scratch_bytes(int d_model, int d_tower, int d_ff, int batch);
+cudaError_t launch_full_head(int batch, int d_model, int d_tower, int d_ff, int n_blocks, float eps,
+                             const float* params, const float* h_prev, const float* emb, const float* h_local,
+                             float threshold, const uint8_t* override_flags, float* scores, float* logits,
+                             uint8_t* flags, int32_t* counters, void* scratch, cudaStream_t st, bool pdl,
+                             int* launches);
+
 struct LayerInfo;
 cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const uint8_t* mask, void* k_cache,
                                     void* v_cache, const int32_t* block_table, const int32_t* seq_lens,

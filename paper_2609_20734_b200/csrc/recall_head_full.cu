@@ -1,0 +1,366 @@
+// The paper's recall head (appendix "Recall-head architecture"): three RMSNorm -> Linear -> SiLU
+// towers, the 9-way interaction vector, a fusion projection, pre-RMSNorm residual SwiGLU blocks and
+// a scalar output; fp32 weights and arithmetic as in the paper.  28.3 M parameters = 113 MB read
+// once per step, so every stage is a bandwidth-bound GEMV: one kernel template, launched once per
+// stage (towers, fusion, gate+up, down, ..., output), chained by programmatic dependent launch.
+//
+// A stage is  y[b][n] = epilogue( sum_k W[n][k] * gain[k] * x[b][k] ):  CTA (row block of 8 rows,
+// 512-wide slice of k) streams its weights with 128-bit loads, stages x of up to 16 requests in
+// shared memory (the interaction vector is formed on the fly from the towers' outputs), publishes
+// partial sums and -- where the stage input is RMS-normalised -- the slice's sum of squares; the
+// CTA that completes a row block (one atomic ticket, no waiting) adds the slices in order and
+// applies the stage's epilogue.  All sums have a fixed order: the result does not depend on
+// scheduling.
+#include <algorithm>
+
+#include "launch_ex.cuh"
+#include "oda_launch.h"
+
+namespace oda {
+
+constexpr int kFRows = 8;
+constexpr int kFThreads = kFRows * 32;
+
+enum { kStageTower = 0, kStageFusion = 1, kStageGateUp = 2, kStageDown = 3, kStageOut = 4 };
+
+struct FullStageParams {
+    int32_t stage, batch, T, F, d_model;
+    int32_t K;                   // reduction length of this stage
+    int32_t row_blocks;
+    float eps;
+    const float* W;              // towers: W of tower 0 (+ i * tower_stride); gate+up: W_gate, W_up = W + F*T
+    const float* gain;           // RMSNorm gain of the stage input (towers: + i * tower_stride), or nullptr
+    const float* bias;           // towers (+ i * tower_stride), fusion, output; or nullptr
+    long long tower_stride;
+    const float *in0, *in1, *in2;  // towers: the three inputs [B][d_model]; fusion: abc [3][B][T];
+                                   // gate+up, output: z [B][T]; down: h [B][F]
+    float* out;                  // towers: abc; fusion: z; gate+up: h; down: z (in place)
+    float* pre;                  // [k slices][rows][batch]
+    float* ssq;                  // [row blocks][k slices][batch]
+    int32_t* rb_tickets;         // [row blocks], zero between launches
+    // output stage
+    float threshold;
+    const uint8_t* override_flags;
+    float* scores;
+    float* logits;
+    uint8_t* flags;
+    int32_t* counters;
+};
+
+__device__ __forceinline__ float silu_f(float a) { return a / (1.f + expf(-a)); }
+
+// four consecutive elements k..k+3 (k % 4 == 0) of the stage input of request b
+__device__ __forceinline__ float4 stage_x4(const FullStageParams& p, int tower, int b, int k)
+{
+    if (p.stage == kStageTower) {
+        const float* in = tower == 0 ? p.in0 : (tower == 1 ? p.in1 : p.in2);
+        return __ldg(reinterpret_cast<const float4*>(in + (size_t)b * p.d_model + k));
+    }
+    if (p.stage == kStageFusion) {
+        // u = [a; b; c; a.b; |a-b|; a.c; |a-c|; b.c; |b-c|]
+        const int seg = k / p.T, j = k - seg * p.T;
+        const float* abc = p.in0;
+        const size_t row = (size_t)b * p.T + j, plane = (size_t)p.batch * p.T;
+        if (seg < 3) return *reinterpret_cast<const float4*>(abc + seg * plane + row);
+        const int pair = (seg - 3) >> 1;  // 0: (a,b)  1: (a,c)  2: (b,c)
+        const int i0 = pair == 2 ? 1 : 0, i1 = pair == 0 ? 1 : 2;
+        const float4 x = *reinterpret_cast<const float4*>(abc + i0 * plane + row);
+        const float4 y = *reinterpret_cast<const float4*>(abc + i1 * plane + row);
+        if ((seg - 3) & 1) return make_float4(fabsf(x.x - y.x), fabsf(x.y - y.y), fabsf(x.z - y.z), fabsf(x.w - y.w));
+        return make_float4(x.x * y.x, x.y * y.y, x.z * y.z, x.w * y.w);
+    }
+    return *reinterpret_cast<const float4*>(p.in0 + (size_t)b * p.K + k);  // z [B][T] or h [B][F]
+}
+
+// finishes output element (row r of the stage, request b) from the complete sums
+__device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, int b, float acc, float acc_up, float ss)
+{
+    const float rs = p.gain ? rsqrtf(ss / (float)p.K + p.eps) : 1.f;
+    if (p.stage == kStageTower) {
+        const int i = r / p.T, j = r - i * p.T;
+        p.out[((size_t)i * p.batch + b) * p.T + j] = silu_f(acc * rs + __ldg(p.bias + i * p.tower_stride + j));
+    } else if (p.stage == kStageFusion) {
+        const size_t row = (size_t)b * p.T + r, plane = (size_t)p.batch * p.T;
+        p.out[row] = 0.5f * (p.in0[row] + p.in0[plane + row] + p.in0[2 * plane + row] + silu_f(acc + __ldg(p.bias + r)));
+    } else if (p.stage == kStageGateUp) {
+        p.out[(size_t)b * p.F + r] = silu_f(acc * rs) * (acc_up * rs);
+    } else if (p.stage == kStageDown) {
+        p.out[(size_t)b * p.T + r] += acc;
+    } else {
+        const float z = acc * rs + __ldg(p.bias);
+        const float score = 1.f / (1.f + expf(-z));
+        uint8_t f;
+        if (p.override_flags)
+            f = p.override_flags[b] ? 1 : 0;
+        else
+            f = (!isfinite(z) || score > p.threshold) ? 1 : 0;
+        p.scores[b] = score;
+        if (p.logits) p.logits[b] = z;
+        p.flags[b] = f;
+        if (p.counters) {
+            p.counters[2 * b] += 1;
+            p.counters[2 * b + 1] += f;
+        }
+    }
+}
+
+// Tile shapes (requests x features of x in shared memory, 32 KiB either way): 4 x 2048 for small
+// batches -- a lane then has all 64 of its weights in flight at once and, at the paper's sizes,
+// only the fusion stage is split over k -- and 16 x 512 for larger batches.
+template <int kFBT, int kFKT>
+__global__ void __launch_bounds__(kFThreads, 2) full_head_stage_kernel(const __grid_constant__ FullStageParams p)
+{
+    constexpr int kWC = kFKT / 128;  // float4 weight loads per lane
+    constexpr int kXL = kFBT * kFKT / 4 / kFThreads;  // float4 loads of x per thread
+    __shared__ __align__(16) float s_x[kFBT][kFKT];   // x * gain
+    __shared__ float s_acc[kFRows][kFBT];
+    __shared__ float s_ss[kFRows][kFBT];
+    __shared__ int s_last;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rb = blockIdx.x, ks = blockIdx.y, n_ks = gridDim.y;
+    const int k0 = ks * kFKT;
+    // which weight row this warp streams, and which tower the row block belongs to
+    int tower = 0;
+    const float* wrow;
+    const float* gain = p.gain;
+    int n;  // row index in the stage's numbering of partial sums
+    if (p.stage == kStageTower) {
+        n = rb * kFRows + warp;
+        tower = n / p.T;
+        wrow = p.W + tower * p.tower_stride + (size_t)(n - tower * p.T) * p.K;
+        gain = p.gain + tower * p.tower_stride;
+    } else if (p.stage == kStageGateUp) {
+        const int m = rb * (kFRows / 2) + (warp & 3);  // hidden unit; warps 0-3 gate, 4-7 up
+        n = (warp < 4 ? 0 : p.F) + m;
+        wrow = p.W + (size_t)n * p.K;
+    } else {
+        n = rb * kFRows + warp;
+        wrow = p.W + (size_t)n * p.K;
+    }
+    const int n_rows = p.stage == kStageTower ? 3 * p.T : (p.stage == kStageGateUp ? 2 * p.F : (p.stage == kStageOut ? 1 : p.T));
+    const bool row_ok = p.stage == kStageGateUp ? (rb * (kFRows / 2) + (warp & 3)) < p.F : n < n_rows;
+    float4 w[kWC];
+#pragma unroll
+    for (int c = 0; c < kWC; ++c) {
+        const int k = k0 + c * 128 + lane * 4;
+        w[c] = (row_ok && k < p.K) ? __ldg(reinterpret_cast<const float4*>(wrow + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int b0 = 0; b0 < p.batch; b0 += kFBT) {
+        if (b0) __syncthreads();
+        // stage x * gain; every load of the tile is in flight together.  Thread t always stages
+        // request u = (t + i*256) / (KT/4): with KT/4 a multiple of 256 or vice versa a thread's
+        // loads belong to few requests, whose sum of squares it accumulates on the way.
+        float4 xr[kXL], gr[kXL];
+#pragma unroll
+        for (int t = 0; t < kXL; ++t) {
+            const int idx = tid + t * kFThreads;
+            const int u = idx / (kFKT / 4), q = idx - u * (kFKT / 4);
+            const bool ok = b0 + u < p.batch && k0 + q * 4 < p.K;
+            xr[t] = ok ? stage_x4(p, tower, b0 + u, k0 + q * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            gr[t] = (ok && gain) ? __ldg(reinterpret_cast<const float4*>(gain + k0 + q * 4)) : make_float4(1.f, 1.f, 1.f, 1.f);
+        }
+        if (gain) {  // sum of x^2 over this slice, per request
+#pragma unroll
+            for (int u = 0; u < kFBT; ++u) {
+                float ss = 0.f;
+#pragma unroll
+                for (int t = 0; t < kXL; ++t) {
+                    if ((tid + t * kFThreads) / (kFKT / 4) == u)
+                        ss += xr[t].x * xr[t].x + xr[t].y * xr[t].y + xr[t].z * xr[t].z + xr[t].w * xr[t].w;
+                }
+                for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                if (lane == 0) s_ss[warp][u] = ss;
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < kXL; ++t) {
+            const int idx = tid + t * kFThreads;
+            const int u = idx / (kFKT / 4), q = idx - u * (kFKT / 4);
+            reinterpret_cast<float4*>(&s_x[u][0])[q] =
+                make_float4(xr[t].x * gr[t].x, xr[t].y * gr[t].y, xr[t].z * gr[t].z, xr[t].w * gr[t].w);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < kFBT; ++u) {
+            if (b0 + u >= p.batch) break;
+            float a = 0.f;
+#pragma unroll
+            for (int c = 0; c < kWC; ++c) {
+                const float4 x = reinterpret_cast<const float4*>(&s_x[u][0])[c * 32 + lane];
+                a = fmaf(w[c].x, x.x, a);
+                a = fmaf(w[c].y, x.y, a);
+                a = fmaf(w[c].z, x.z, a);
+                a = fmaf(w[c].w, x.w, a);
+            }
+            for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            if (lane == 0) s_acc[warp][u] = a;
+        }
+        __syncthreads();
+        // ---- the tile's results: finish here when the stage is not split over k, else publish
+        const int out_rows = p.stage == kStageGateUp ? kFRows / 2 : kFRows;
+        for (int e = tid; e < out_rows * kFBT; e += kFThreads) {
+            const int r = e / kFBT, u = e - r * kFBT;
+            if (b0 + u >= p.batch) continue;
+            float ss = 0.f;
+            if (gain) {
+#pragma unroll
+                for (int wv = 0; wv < kFRows; ++wv) ss += s_ss[wv][u];  // fixed order
+            }
+            if (n_ks == 1) {
+                if (p.stage == kStageGateUp) {
+                    const int m = rb * (kFRows / 2) + r;
+                    if (m < p.F) stage_finish(p, m, b0 + u, s_acc[r][u], s_acc[r + 4][u], ss);
+                } else {
+                    const int nn = rb * kFRows + r;
+                    if (nn < n_rows) stage_finish(p, nn, b0 + u, s_acc[r][u], 0.f, ss);
+                }
+            } else {
+                if (gain && r == 0) __stcg(p.ssq + ((size_t)rb * n_ks + ks) * p.batch + b0 + u, ss);
+                for (int rr = r; rr < kFRows; rr += out_rows) {  // gate+up: both halves
+                    int nn;
+                    bool ok;
+                    if (p.stage == kStageGateUp) {
+                        const int m = rb * (kFRows / 2) + (rr & 3);
+                        nn = (rr < 4 ? 0 : p.F) + m;
+                        ok = m < p.F;
+                    } else {
+                        nn = rb * kFRows + rr;
+                        ok = nn < n_rows;
+                    }
+                    if (ok) __stcg(p.pre + ((size_t)ks * n_rows + nn) * p.batch + b0 + u, s_acc[rr][u]);
+                }
+            }
+        }
+    }
+    if (n_ks == 1) return;
+    // ---- split over k: the CTA that completes the row block adds the slices in order
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int old = atomicAdd(p.rb_tickets + rb, 1);
+        s_last = (old == n_ks - 1);
+        if (s_last) p.rb_tickets[rb] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const int out_rows = p.stage == kStageGateUp ? kFRows / 2 : kFRows;
+    for (int e = tid; e < out_rows * p.batch; e += kFThreads) {
+        const int r = e / p.batch, b = e - r * p.batch;
+        float ss = 0.f;
+        if (p.gain)
+            for (int s2 = 0; s2 < n_ks; ++s2) ss += __ldcg(p.ssq + ((size_t)rb * n_ks + s2) * p.batch + b);
+        auto acc_of = [&](int row) {
+            float a = 0.f;
+            for (int s2 = 0; s2 < n_ks; ++s2) a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
+            return a;
+        };
+        if (p.stage == kStageGateUp) {
+            const int m = rb * (kFRows / 2) + r;
+            if (m < p.F) stage_finish(p, m, b, acc_of(m), acc_of(p.F + m), ss);
+        } else {
+            const int nn = rb * kFRows + r;
+            if (nn < n_rows) stage_finish(p, nn, b, acc_of(nn), 0.f, ss);
+        }
+    }
+}
+
+long long full_head_param_count(int d_model, int T, int F, int n_blocks)
+{
+    const long long tower = (long long)d_model + (long long)T * d_model + T;
+    const long long fusion = (long long)T * 9 * T + T;
+    const long long block = (long long)T + 3ll * F * T;
+    return 3 * tower + fusion + n_blocks * block + 2ll * T + 1;
+}
+
+static int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+constexpr int kFKT = 512;  // the narrower tile: what the scratch is sized for
+
+// scratch layout (floats unless noted): abc [3][B][T] | z [B][T] | h [B][F] | pre | ssq | tickets (int32)
+struct FullScratch {
+    size_t abc, z, h, pre, ssq, tickets, total;
+};
+
+static FullScratch full_scratch_layout(int d_model, int T, int F, int batch)
+{
+    FullScratch s;
+    auto al = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t B = batch;
+    size_t off = 0;
+    s.abc = off; off = al(off + 3 * B * T * 4);
+    s.z = off; off = al(off + B * T * 4);
+    s.h = off; off = al(off + B * F * 4);
+    // pre: max over stages of k slices * rows
+    const size_t pre_rows = std::max({(size_t)ceil_div(d_model, kFKT) * 3 * T, (size_t)ceil_div(9ll * T, kFKT) * T,
+                                      (size_t)ceil_div(T, kFKT) * 2 * F, (size_t)ceil_div(F, kFKT) * T});
+    s.pre = off; off = al(off + pre_rows * B * 4);
+    const size_t ssq_rows = std::max({(size_t)ceil_div(3ll * T, kFRows) * ceil_div(d_model, kFKT),
+                                      (size_t)ceil_div(F, kFRows / 2) * ceil_div(T, kFKT), (size_t)ceil_div(T, kFKT)});
+    s.ssq = off; off = al(off + ssq_rows * B * 4);
+    const size_t max_rb = std::max({(size_t)ceil_div(3ll * T, kFRows), (size_t)ceil_div(F, kFRows / 2), (size_t)T});
+    s.tickets = off; off = al(off + max_rb * 4);
+    s.total = off;
+    return s;
+}
+
+size_t full_head_scratch_bytes(int d_model, int T, int F, int batch)
+{
+    return full_scratch_layout(d_model, T, F, batch).total;
+}
+
+cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks, float eps, const float* params,
+                             const float* h_prev, const float* emb, const float* h_local, float threshold,
+                             const uint8_t* override_flags, float* scores, float* logits, uint8_t* flags,
+                             int32_t* counters, void* scratch, cudaStream_t st, bool pdl, int* launches)
+{
+    char* sc = static_cast<char*>(scratch);
+    const FullScratch L = full_scratch_layout(d_model, T, F, batch);
+    float* abc = reinterpret_cast<float*>(sc + L.abc);
+    float* z = reinterpret_cast<float*>(sc + L.z);
+    float* h = reinterpret_cast<float*>(sc + L.h);
+    cudaError_t e = cudaMemsetAsync(sc + L.tickets, 0, L.total - L.tickets, st);
+    if (e != cudaSuccess) return e;
+    FullStageParams p = {};
+    p.batch = batch; p.T = T; p.F = F; p.d_model = d_model; p.eps = eps;
+    p.pre = reinterpret_cast<float*>(sc + L.pre);
+    p.ssq = reinterpret_cast<float*>(sc + L.ssq);
+    p.rb_tickets = reinterpret_cast<int32_t*>(sc + L.tickets);
+    auto launch = [&](bool dep) {
+        cudaError_t le = batch <= 4
+            ? launch_ex(full_head_stage_kernel<4, 2048>, dim3(p.row_blocks, ceil_div(p.K, 2048)), dim3(kFThreads), 0, st, dep, p)
+            : launch_ex(full_head_stage_kernel<16, 512>, dim3(p.row_blocks, ceil_div(p.K, 512)), dim3(kFThreads), 0, st, dep, p);
+        if (le == cudaSuccess && launches) ++*launches;
+        return le;
+    };
+    const long long tower_stride = (long long)d_model + (long long)T * d_model + T;
+    const float* cur = params;
+    // towers (one launch for the three)
+    p.stage = kStageTower; p.K = d_model; p.row_blocks = ceil_div(3ll * T, kFRows);
+    p.gain = cur; p.W = cur + d_model; p.bias = cur + d_model + (long long)T * d_model; p.tower_stride = tower_stride;
+    p.in0 = h_prev; p.in1 = emb; p.in2 = h_local; p.out = abc;
+    if ((e = launch(false)) != cudaSuccess) return e;  // follows a memset: ordinary launch
+    cur += 3 * tower_stride;
+    // fusion
+    p.stage = kStageFusion; p.K = 9 * T; p.row_blocks = ceil_div(T, kFRows);
+    p.gain = nullptr; p.W = cur; p.bias = cur + (long long)T * 9 * T; p.in0 = abc; p.in1 = p.in2 = nullptr; p.out = z;
+    if ((e = launch(pdl)) != cudaSuccess) return e;
+    cur += (long long)T * 9 * T + T;
+    for (int k = 0; k < n_blocks; ++k) {
+        p.stage = kStageGateUp; p.K = T; p.row_blocks = ceil_div(F, kFRows / 2);
+        p.gain = cur; p.W = cur + T; p.bias = nullptr; p.in0 = z; p.out = h;
+        if ((e = launch(pdl)) != cudaSuccess) return e;
+        p.stage = kStageDown; p.K = F; p.row_blocks = ceil_div(T, kFRows);
+        p.gain = nullptr; p.W = cur + T + 2ll * F * T; p.in0 = h; p.out = z;
+        if ((e = launch(pdl)) != cudaSuccess) return e;
+        cur += (long long)T + 3ll * F * T;
+    }
+    p.stage = kStageOut; p.K = T; p.row_blocks = 1;
+    p.gain = cur; p.W = cur + T; p.bias = cur + 2 * T; p.in0 = z; p.out = nullptr;
+    p.threshold = threshold; p.override_flags = override_flags; p.scores = scores; p.logits = logits;
+    p.flags = flags; p.counters = counters;
+    return launch(pdl);
+}
+
+}  // namespace oda

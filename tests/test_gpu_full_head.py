@@ -1,0 +1,82 @@
+"""GPU parity of the paper's full recall head (three towers, interaction vector, fusion, SwiGLU
+blocks) against the fp64 oracle, at toy sizes and at the paper's 28,325,889-parameter size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oda_oracle as orc
+from paper_2609_20734_b200 import binding, synth
+from tests import gpu_helpers as gh
+from tests.helpers import make_problem
+from tests.test_oracle_full_head import _layout, _pack
+
+pytestmark = pytest.mark.gpu
+
+
+def _params(seed, dm, T, F, nb):
+    parts = {}
+    for i, (n, shp) in enumerate(_layout(dm, T, F, nb)):
+        fan_in = shp[-1] if len(shp) == 2 else 1
+        std = 1.0 / np.sqrt(fan_in) if len(shp) == 2 else 0.1
+        parts[n] = synth.gauss_f32_tensor(seed, 200 + i, shp, std=std)
+        if n.startswith("g") or n.startswith("bg"):
+            parts[n] = (1.0 + parts[n]).astype(np.float32)
+    return _pack(parts, dm, T, F, nb)
+
+
+def _ctx():
+    prob = make_problem(1, 1, 1, 1, 1, 64, [20])
+    return gh.make_ctx(prob, [8], [0], [1])
+
+
+@pytest.mark.parametrize("dm,T,F,nb,B", [(64, 32, 40, 2, 5), (128, 64, 96, 1, 20), (2048, 1024, 2048, 2, 4)])
+def test_full_head_parity(dm, T, F, nb, B):
+    ctx = _ctx()
+    params = _params(3, dm, T, F, nb)
+    assert params.size == binding.load_library().oda_full_head_param_count(dm, T, F, nb)
+    if (dm, T, F, nb) == (2048, 1024, 2048, 2):
+        assert params.size == 28325889
+    x = [synth.gauss_f32_tensor(4, i, (B, dm)) for i in range(3)]
+    q, s = orc.full_head(params, *x, d_tower=T, d_ff=F, n_blocks=nb)
+    srt = np.sort(s)
+    tau = float(0.5 * (srt[B // 2 - 1] + srt[B // 2]))
+    scores = torch.zeros(B, device="cuda")
+    logits = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    counters = torch.zeros((B, 2), dtype=torch.int32, device="cuda")
+    pd = torch.from_numpy(params).cuda()
+    xd = [torch.from_numpy(v).cuda() for v in x]
+    scratch = None
+    for _ in range(2):   # twice: tickets and scratch must be reusable
+        scratch = ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], xd[2], tau, None, scores, logits, flags,
+                                        counters, scratch=scratch)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(logits.cpu().numpy(), q, rtol=0, atol=1e-4)
+    np.testing.assert_allclose(scores.cpu().numpy(), s, rtol=0, atol=2e-5)
+    decided = np.abs(s - tau) >= gh.FLAG_BAND
+    np.testing.assert_array_equal(flags.cpu().numpy()[decided], orc.flags(q, s, tau)[decided])
+    c = counters.cpu().numpy()
+    assert (c[:, 0] == 2).all() and (c[:, 1] == 2 * flags.cpu().numpy()).all()
+    # forced flags: the head still runs
+    ov = (np.arange(B) % 2).astype(np.uint8)
+    ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], xd[2], tau, torch.from_numpy(ov).cuda(), scores, None,
+                          flags, None, scratch=scratch)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(flags.cpu().numpy(), ov)
+    np.testing.assert_allclose(scores.cpu().numpy(), s, rtol=0, atol=2e-5)
+
+
+def test_full_head_nonfinite_input_selects_full_and_bad_dims_are_refused():
+    ctx = _ctx()
+    dm, T, F, nb, B = 64, 32, 40, 1, 3
+    params = torch.from_numpy(_params(5, dm, T, F, nb)).cuda()
+    x = [torch.from_numpy(synth.gauss_f32_tensor(6, i, (B, dm))).cuda() for i in range(3)]
+    x[2][1, 7] = float("nan")
+    scores = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    ctx.recall_score_full(B, params, T, F, nb, x[0], x[1], x[2], 2.0, None, scores, None, flags)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(flags.cpu().numpy(), [0, 1, 0])   # threshold 2 is never exceeded; NaN forces Full
+    with pytest.raises(binding.OdaError) as e:
+        ctx.recall_score_full(B, params, 36, F, nb, x[0], x[1], x[2], 0.5, None, scores, None, flags)
+    assert e.value.status == 2
