@@ -113,7 +113,7 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def reference_arm(args, wl):
+def reference_arm(args, wl, realised_rate=None):
     """The oracle, as it stands, timed on the host cores.  A step is a bounded sample of the
     workload: Local on `nl` layers and Full on `nf` layers of the stack, extrapolated to all
     layers and combined at the realised recall rate of the same forced-flag schedule."""
@@ -131,7 +131,7 @@ def reference_arm(args, wl):
     idx = np.arange(0, nl * lay.layer_stride, dtype=np.uint64)
     k, v = synth.gauss_bf16(kk, idx), synth.gauss_bf16(vk, idx)
     flags = [wl.override_flags(s) for s in range(args.warmup + args.steps)]
-    realised = float(np.mean([f.mean() for f in flags[args.warmup:]]))
+    realised = float(np.mean([f.mean() for f in flags[args.warmup:]])) if realised_rate is None else realised_rate
 
     def one(step, mode, n):
         q = wl.q_host(step)[:n]
@@ -432,7 +432,7 @@ def main():
             ref_args = argparse.Namespace(**vars(args))
             ref_args.steps, ref_args.warmup = 3, 1
             with contextlib.redirect_stdout(buf):
-                reference_arm(ref_args, workloads.make(args.config, recall_rate=args.recall_rate))
+                reference_arm(ref_args, workloads.make(args.config, recall_rate=args.recall_rate), realised)
             line["cpu_baseline"] = json.loads(buf.getvalue())["cpu_baseline"]
         print(json.dumps(line))
     if world > 1:
