@@ -51,6 +51,9 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--kernel-reps", type=int, default=10)
     ap.add_argument("--no-calibrate", action="store_true", help="keep the equal split of work across CTAs")
+    ap.add_argument("--paper-sweep", action="store_true",
+                    help="attention-only decode at the paper's seven prompt lengths (batch 1, w=2048+4 sinks, "
+                         "first-k-of-16 schedules); prints one JSON table and exits")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the Local and the all-flagged Full attention launches (for ncu captures)")
     return ap.parse_args()
@@ -171,9 +174,91 @@ def config_dict(wl, args, realised):
             "launch": "one CUDA graph replay per step"}
 
 
+PAPER_LENGTHS = [4139, 15918, 31400, 63852, 128852, 261696, 516788]
+
+
+def paper_sweep(args):
+    """Tokens/s of the attention path at the paper's prompt lengths: native Full alone, Local
+    alone, and ODA steps with Full on the first 2 / 4 / 8 of every 16 steps (12.5 / 25 / 50 %)."""
+    import torch
+
+    from paper_2609_20734_b200 import binding, workloads
+
+    torch.cuda.set_device(0)
+    flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+    rows = []
+    for n in PAPER_LENGTHS:
+        wl = workloads.make("paper", seq_lens0=np.array([n], np.int32), steps=40)
+        st = workloads.materialize(wl)
+        ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks, variant=args.variant))
+        B, L = wl.B, wl.L
+        shape = (L, B, wl.Hq, wl.D)
+        q = workloads.q_device(wl, 0)
+        out = torch.zeros(shape, device="cuda")
+        scores = torch.zeros(B, device="cuda")
+        flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+        ov = torch.zeros(B, dtype=torch.uint8, device="cuda")
+        ones = torch.ones(B, dtype=torch.uint8, device="cuda")
+        seq0 = st.seq_lens.clone()
+        if not args.no_calibrate:
+            ctx.calibration_begin()
+            ctx.full_decode_gated(0, L, B, q, st.k_cache, st.v_cache, st.block_table, st.seq_lens, ones, out, None)
+            ctx.calibration_end()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+
+        def capture(fn):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    fn(side.cuda_stream)
+            return g
+
+        g_step = capture(lambda s_: ctx.step(ctx.step_args(B, q, st.k_cache, st.v_cache, st.block_table, st.seq_lens,
+                                                             out, scores, flags, override_flags=ov,
+                                                             advance_seq_lens=True), stream=s_))
+        g_full = capture(lambda s_: ctx.full_decode_gated(0, L, B, q, st.k_cache, st.v_cache, st.block_table,
+                                                            st.seq_lens, ones, out, None, stream=s_))
+        g_local = capture(lambda s_: ctx.local_decode(0, L, B, q, st.k_cache, st.v_cache, st.block_table,
+                                                        st.seq_lens, out, None, stream=s_))
+        torch.cuda.synchronize()
+
+        def timed(graph, steps, first_k=None):
+            st.seq_lens.copy_(seq0)
+            tot = 0.0
+            for s_ in range(steps + 2):
+                if first_k is not None:
+                    ov.fill_(1 if (s_ % 16) < first_k else 0)
+                flush.fill_(s_ & 0xFF)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                graph.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                if s_ >= 2:
+                    tot += e0.elapsed_time(e1)
+            return B * steps / (tot * 1e-3)
+
+        row = {"input_tokens": n, "full_only_tok_s": timed(g_full, 8), "local_only_tok_s": timed(g_local, 8)}
+        for k, name in ((2, "oda_12.5"), (4, "oda_25"), (8, "oda_50")):
+            # 32 timed steps after 2 warm-ups: two whole 16-step periods, phase shifted by 2
+            row[name + "_tok_s"] = timed(g_step, 32, first_k=k)
+        for name in ("local_only", "oda_12.5", "oda_25", "oda_50"):
+            row[name + "_speedup_vs_full"] = row[name + "_tok_s"] / row["full_only_tok_s"]
+        rows.append(row)
+        del st, ctx, g_step, g_full, g_local
+        torch.cuda.empty_cache()
+    print(json.dumps({"paper_sweep": rows, "shape": "28 layers, 16q/8kv heads, head_dim 128, batch 1, window 2048 + 4 sinks",
+                      "note": "attention path only; the paper's table times the whole model in vLLM on A100s"}))
+
+
 def main():
     args = parse()
     from paper_2609_20734_b200 import workloads
+
+    if args.paper_sweep:
+        paper_sweep(args)
+        return
 
     ov = {"recall_rate": args.recall_rate}
     wl = workloads.make(args.config, **ov)

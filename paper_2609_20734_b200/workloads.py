@@ -162,6 +162,14 @@ def make(name: str, **ov) -> Workload:
         wl = Workload("hybrid", L, 4, 32, 8, 128, windows, sinks, gated,
                       np.full(4, 262144, np.int32), 8, kv_index=kv_index, head=(0, 1, 256),
                       recall_rate=0.15)
+    elif name == "paper":
+        # The paper's timing workload: batch 1, s=4 sinks + w=2048 window, one prompt per length
+        # (4,139 ... 516,788 tokens) and a prescribed first-k-of-16 schedule.  The attention shape
+        # is Qwen3-1.7B's public configuration (28 layers, 16 query / 8 KV heads, head_dim 128);
+        # the paper itself only states the hidden size.
+        w, s, g = _uniform(28, 2048, 4)
+        wl = Workload("paper", 28, 1, 16, 8, 128, w, s, g, np.array([128852], np.int32), 16,
+                      schedule="periodic", recall_rate=0.125)
     else:
         raise KeyError(name)
     return replace(wl, **ov) if ov else wl
