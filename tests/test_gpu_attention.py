@@ -201,3 +201,37 @@ def test_calibrated_split_gives_the_same_result():
         gh.assert_close(full[l].cpu().numpy(), reff[l], gh.ATOL_OUT, f"calibrated full layer {l}")
         np.testing.assert_allclose(full[l].cpu().numpy(), before[l].cpu().numpy(), rtol=0, atol=1e-5)
     assert ctx.read_device_status() == 0
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_maximum_batch_many_layers_tiny_sequences(variant):
+    """128 requests (the batch limit) of 1..200 tokens on 40 layers with three layer classes:
+    many tiny units per span, most spans crossing many unit boundaries."""
+    B, L = 128, 40
+    rng = np.random.RandomState(5)
+    seq = rng.randint(1, 201, size=B).tolist()
+    seq[0], seq[1], seq[2] = 1, 16, 17
+    prob = make_problem(31, L, B, 4, 2, 64, seq, layout="nhd")
+    windows = [32 if l % 3 == 0 else (48 if l % 3 == 1 else 300) for l in range(L)]
+    sinks = [4 if l % 3 == 0 else (0 if l % 3 == 1 else 2) for l in range(L)]
+    gated = [1 if l % 3 != 1 else 0 for l in range(L)]
+    ctx = gh.make_ctx(prob, windows, sinks, gated, variant=variant)
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8)
+    gh.assert_close(out, ref, gh.ATOL_OUT, "max-batch local")
+    gh.assert_close(lse, rlse, gh.ATOL_LSE, "max-batch lse")
+    flags_h = (rng.rand(B) < 0.3).astype(np.uint8)
+    full, _ = gh.new_out(prob, fill=-3.0)
+    ctx.full_decode_gated(0, L, B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
+                          torch.from_numpy(flags_h).cuda(), full, None)
+    torch.cuda.synchronize()
+    reff, _ = oracle_attention(prob, "full", windows, sinks, nthreads=8)
+    full = full.cpu().numpy()
+    for l in range(L):
+        for b in range(B):
+            if gated[l] and flags_h[b]:
+                gh.assert_close(full[l, b], reff[l, b], gh.ATOL_OUT, f"max-batch full l{l} b{b}")
+            else:
+                assert (full[l, b] == -3.0).all()
+    assert ctx.read_device_status() == 0
