@@ -107,8 +107,11 @@ __device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, in
 // Tile shapes (requests x features of x in shared memory, 32 KiB either way): 4 x 2048 for small
 // batches -- a lane then has all 64 of its weights in flight at once and, at the paper's sizes,
 // only the fusion stage is split over k -- and 16 x 512 for larger batches.
+// Grid: x = CTAs that share the row blocks of one (k slice, tower) round-robin, y = k slice,
+// z = tower (tower stage only).  A CTA stages its x tile once and then walks its row blocks with
+// the next block's weights already in flight.
 template <int kFBT, int kFKT>
-__global__ void __launch_bounds__(kFThreads, 2) full_head_stage_kernel(const __grid_constant__ FullStageParams p)
+__global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_stage_kernel(const __grid_constant__ FullStageParams p)
 {
     constexpr int kWC = kFKT / 128;  // float4 weight loads per lane
     constexpr int kXL = kFBT * kFKT / 4 / kFThreads;  // float4 loads of x per thread
@@ -119,150 +122,174 @@ __global__ void __launch_bounds__(kFThreads, 2) full_head_stage_kernel(const __g
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int rb = blockIdx.x, ks = blockIdx.y, n_ks = gridDim.y;
+    const int ks = blockIdx.y, n_ks = gridDim.y;
+    const int tower = p.stage == kStageTower ? (int)blockIdx.z : 0;
     const int k0 = ks * kFKT;
-    // which weight row this warp streams, and which tower the row block belongs to
-    int tower = 0;
-    const float* wrow;
-    const float* gain = p.gain;
-    int n;  // row index in the stage's numbering of partial sums
-    if (p.stage == kStageTower) {
-        n = rb * kFRows + warp;
-        tower = n / p.T;
-        wrow = p.W + tower * p.tower_stride + (size_t)(n - tower * p.T) * p.K;
-        gain = p.gain + tower * p.tower_stride;
-    } else if (p.stage == kStageGateUp) {
-        const int m = rb * (kFRows / 2) + (warp & 3);  // hidden unit; warps 0-3 gate, 4-7 up
-        n = (warp < 4 ? 0 : p.F) + m;
-        wrow = p.W + (size_t)n * p.K;
-    } else {
-        n = rb * kFRows + warp;
-        wrow = p.W + (size_t)n * p.K;
-    }
     const int n_rows = p.stage == kStageTower ? 3 * p.T : (p.stage == kStageGateUp ? 2 * p.F : (p.stage == kStageOut ? 1 : p.T));
-    const bool row_ok = p.stage == kStageGateUp ? (rb * (kFRows / 2) + (warp & 3)) < p.F : n < n_rows;
-    float4 w[kWC];
+    const int out_rows = p.stage == kStageGateUp ? kFRows / 2 : kFRows;
+    // row blocks this CTA's group covers, and the group's offset in the stage's row numbering
+    const int group_rbs = p.stage == kStageTower ? (p.T + kFRows - 1) / kFRows
+                        : (p.stage == kStageGateUp ? (p.F + out_rows - 1) / out_rows
+                        : (p.stage == kStageOut ? 1 : (p.T + kFRows - 1) / kFRows));
+    const int group_row0 = tower * p.T;
+    const float* gain = p.gain ? p.gain + tower * p.tower_stride : nullptr;
+    const float* wbase = p.W + tower * p.tower_stride;
+    // (row in the stage's numbering, is it a real row) of this warp for row block rb
+    auto row_of = [&](int rb, bool& ok) {
+        if (p.stage == kStageGateUp) {
+            const int m = rb * out_rows + (warp & 3);  // hidden unit; warps 0-3 gate, 4-7 up
+            ok = m < p.F;
+            return (warp < 4 ? 0 : p.F) + m;
+        }
+        const int local = rb * kFRows + warp;
+        ok = local < (p.stage == kStageTower ? p.T : n_rows);
+        return group_row0 + local;
+    };
+    auto load_w = [&](float4 (&w)[kWC], int rb) {
+        bool ok;
+        const int n = row_of(rb, ok);
+        const float* wrow = wbase + (size_t)(n - group_row0) * p.K;
 #pragma unroll
-    for (int c = 0; c < kWC; ++c) {
-        const int k = k0 + c * 128 + lane * 4;
-        w[c] = (row_ok && k < p.K) ? __ldg(reinterpret_cast<const float4*>(wrow + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+        for (int c = 0; c < kWC; ++c) {
+            const int k = k0 + c * 128 + lane * 4;
+            w[c] = (ok && k < p.K) ? __ldg(reinterpret_cast<const float4*>(wrow + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
     for (int b0 = 0; b0 < p.batch; b0 += kFBT) {
+        const bool last_tile = b0 + kFBT >= p.batch;
+        float4 w_cur[kWC], w_nxt[kWC];
+        int rb = blockIdx.x;
+        if (rb < group_rbs) load_w(w_cur, rb);
         if (b0) __syncthreads();
-        // stage x * gain; every load of the tile is in flight together.  Thread t always stages
-        // request u = (t + i*256) / (KT/4): with KT/4 a multiple of 256 or vice versa a thread's
-        // loads belong to few requests, whose sum of squares it accumulates on the way.
-        float4 xr[kXL], gr[kXL];
+        {   // stage x * gain; every load of the tile is in flight together; the sum of squares of
+            // the raw x is accumulated on the way
+            float4 xr[kXL], gr[kXL];
 #pragma unroll
-        for (int t = 0; t < kXL; ++t) {
-            const int idx = tid + t * kFThreads;
-            const int u = idx / (kFKT / 4), q = idx - u * (kFKT / 4);
-            const bool ok = b0 + u < p.batch && k0 + q * 4 < p.K;
-            xr[t] = ok ? stage_x4(p, tower, b0 + u, k0 + q * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            gr[t] = (ok && gain) ? __ldg(reinterpret_cast<const float4*>(gain + k0 + q * 4)) : make_float4(1.f, 1.f, 1.f, 1.f);
-        }
-        if (gain) {  // sum of x^2 over this slice, per request
-#pragma unroll
-            for (int u = 0; u < kFBT; ++u) {
-                float ss = 0.f;
-#pragma unroll
-                for (int t = 0; t < kXL; ++t) {
-                    if ((tid + t * kFThreads) / (kFKT / 4) == u)
-                        ss += xr[t].x * xr[t].x + xr[t].y * xr[t].y + xr[t].z * xr[t].z + xr[t].w * xr[t].w;
-                }
-                for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-                if (lane == 0) s_ss[warp][u] = ss;
+            for (int t = 0; t < kXL; ++t) {
+                const int idx = tid + t * kFThreads;
+                const int u = idx / (kFKT / 4), q = idx - u * (kFKT / 4);
+                const bool ok = b0 + u < p.batch && k0 + q * 4 < p.K;
+                xr[t] = ok ? stage_x4(p, tower, b0 + u, k0 + q * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                gr[t] = (ok && gain) ? __ldg(reinterpret_cast<const float4*>(gain + k0 + q * 4)) : make_float4(1.f, 1.f, 1.f, 1.f);
             }
-        }
-#pragma unroll
-        for (int t = 0; t < kXL; ++t) {
-            const int idx = tid + t * kFThreads;
-            const int u = idx / (kFKT / 4), q = idx - u * (kFKT / 4);
-            reinterpret_cast<float4*>(&s_x[u][0])[q] =
-                make_float4(xr[t].x * gr[t].x, xr[t].y * gr[t].y, xr[t].z * gr[t].z, xr[t].w * gr[t].w);
-        }
-        __syncthreads();
-#pragma unroll
-        for (int u = 0; u < kFBT; ++u) {
-            if (b0 + u >= p.batch) break;
-            float a = 0.f;
-#pragma unroll
-            for (int c = 0; c < kWC; ++c) {
-                const float4 x = reinterpret_cast<const float4*>(&s_x[u][0])[c * 32 + lane];
-                a = fmaf(w[c].x, x.x, a);
-                a = fmaf(w[c].y, x.y, a);
-                a = fmaf(w[c].z, x.z, a);
-                a = fmaf(w[c].w, x.w, a);
-            }
-            for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-            if (lane == 0) s_acc[warp][u] = a;
-        }
-        __syncthreads();
-        // ---- the tile's results: finish here when the stage is not split over k, else publish
-        const int out_rows = p.stage == kStageGateUp ? kFRows / 2 : kFRows;
-        for (int e = tid; e < out_rows * kFBT; e += kFThreads) {
-            const int r = e / kFBT, u = e - r * kFBT;
-            if (b0 + u >= p.batch) continue;
-            float ss = 0.f;
             if (gain) {
 #pragma unroll
-                for (int wv = 0; wv < kFRows; ++wv) ss += s_ss[wv][u];  // fixed order
-            }
-            if (n_ks == 1) {
-                if (p.stage == kStageGateUp) {
-                    const int m = rb * (kFRows / 2) + r;
-                    if (m < p.F) stage_finish(p, m, b0 + u, s_acc[r][u], s_acc[r + 4][u], ss);
-                } else {
-                    const int nn = rb * kFRows + r;
-                    if (nn < n_rows) stage_finish(p, nn, b0 + u, s_acc[r][u], 0.f, ss);
-                }
-            } else {
-                if (gain && r == 0) __stcg(p.ssq + ((size_t)rb * n_ks + ks) * p.batch + b0 + u, ss);
-                for (int rr = r; rr < kFRows; rr += out_rows) {  // gate+up: both halves
-                    int nn;
-                    bool ok;
-                    if (p.stage == kStageGateUp) {
-                        const int m = rb * (kFRows / 2) + (rr & 3);
-                        nn = (rr < 4 ? 0 : p.F) + m;
-                        ok = m < p.F;
-                    } else {
-                        nn = rb * kFRows + rr;
-                        ok = nn < n_rows;
+                for (int u = 0; u < kFBT; ++u) {
+                    float ss = 0.f;
+#pragma unroll
+                    for (int t = 0; t < kXL; ++t) {
+                        if ((tid + t * kFThreads) / (kFKT / 4) == u)
+                            ss += xr[t].x * xr[t].x + xr[t].y * xr[t].y + xr[t].z * xr[t].z + xr[t].w * xr[t].w;
                     }
-                    if (ok) __stcg(p.pre + ((size_t)ks * n_rows + nn) * p.batch + b0 + u, s_acc[rr][u]);
+                    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    if (lane == 0) s_ss[warp][u] = ss;
                 }
+            }
+#pragma unroll
+            for (int t = 0; t < kXL; ++t) {
+                const int idx = tid + t * kFThreads;
+                const int u = idx / (kFKT / 4), q = idx - u * (kFKT / 4);
+                reinterpret_cast<float4*>(&s_x[u][0])[q] =
+                    make_float4(xr[t].x * gr[t].x, xr[t].y * gr[t].y, xr[t].z * gr[t].z, xr[t].w * gr[t].w);
             }
         }
-    }
-    if (n_ks == 1) return;
-    // ---- split over k: the CTA that completes the row block adds the slices in order
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int old = atomicAdd(p.rb_tickets + rb, 1);
-        s_last = (old == n_ks - 1);
-        if (s_last) p.rb_tickets[rb] = 0;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const int out_rows = p.stage == kStageGateUp ? kFRows / 2 : kFRows;
-    for (int e = tid; e < out_rows * p.batch; e += kFThreads) {
-        const int r = e / p.batch, b = e - r * p.batch;
-        float ss = 0.f;
-        if (p.gain)
-            for (int s2 = 0; s2 < n_ks; ++s2) ss += __ldcg(p.ssq + ((size_t)rb * n_ks + s2) * p.batch + b);
-        auto acc_of = [&](int row) {
-            float a = 0.f;
-            for (int s2 = 0; s2 < n_ks; ++s2) a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
-            return a;
-        };
-        if (p.stage == kStageGateUp) {
-            const int m = rb * (kFRows / 2) + r;
-            if (m < p.F) stage_finish(p, m, b, acc_of(m), acc_of(p.F + m), ss);
-        } else {
-            const int nn = rb * kFRows + r;
-            if (nn < n_rows) stage_finish(p, nn, b, acc_of(nn), 0.f, ss);
+        __syncthreads();
+        for (; rb < group_rbs; rb += gridDim.x) {
+            const bool more = rb + (int)gridDim.x < group_rbs;
+            if (more) load_w(w_nxt, rb + gridDim.x);  // in flight while this block is computed
+#pragma unroll
+            for (int u = 0; u < kFBT; ++u) {
+                if (b0 + u >= p.batch) break;
+                float a = 0.f;
+#pragma unroll
+                for (int c = 0; c < kWC; ++c) {
+                    const float4 x = reinterpret_cast<const float4*>(&s_x[u][0])[c * 32 + lane];
+                    a = fmaf(w_cur[c].x, x.x, a);
+                    a = fmaf(w_cur[c].y, x.y, a);
+                    a = fmaf(w_cur[c].z, x.z, a);
+                    a = fmaf(w_cur[c].w, x.w, a);
+                }
+                for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+                if (lane == 0) s_acc[warp][u] = a;
+            }
+            __syncthreads();
+            // ---- the block's results for this tile of requests: finish here when the stage is not
+            //      split over k, else publish
+            const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb;  // row block id in the scratch
+            for (int e = tid; e < out_rows * kFBT; e += kFThreads) {
+                const int r = e / kFBT, u = e - r * kFBT;
+                if (b0 + u >= p.batch) continue;
+                float ss = 0.f;
+                if (gain) {
+#pragma unroll
+                    for (int wv = 0; wv < kFRows; ++wv) ss += s_ss[wv][u];  // fixed order
+                }
+                if (n_ks == 1) {
+                    if (p.stage == kStageGateUp) {
+                        const int m = rb * out_rows + r;
+                        if (m < p.F) stage_finish(p, m, b0 + u, s_acc[r][u], s_acc[r + 4][u], ss);
+                    } else {
+                        const int local = rb * kFRows + r;
+                        if (local < (p.stage == kStageTower ? p.T : n_rows)) stage_finish(p, group_row0 + local, b0 + u, s_acc[r][u], 0.f, ss);
+                    }
+                } else {
+                    if (gain && r == 0) __stcg(p.ssq + ((size_t)grb * n_ks + ks) * p.batch + b0 + u, ss);
+                    for (int rr = r; rr < kFRows; rr += out_rows) {  // gate+up: both halves
+                        int nn;
+                        bool ok;
+                        if (p.stage == kStageGateUp) {
+                            const int m = rb * out_rows + (rr & 3);
+                            nn = (rr < 4 ? 0 : p.F) + m;
+                            ok = m < p.F;
+                        } else {
+                            const int local = rb * kFRows + rr;
+                            nn = group_row0 + local;
+                            ok = local < (p.stage == kStageTower ? p.T : n_rows);
+                        }
+                        if (ok) __stcg(p.pre + ((size_t)ks * n_rows + nn) * p.batch + b0 + u, s_acc[rr][u]);
+                    }
+                }
+            }
+            __syncthreads();  // s_acc and s_last are reused by the next row block
+#pragma unroll
+            for (int c = 0; c < kWC; ++c) w_cur[c] = w_nxt[c];
+        }
+        if (n_ks > 1 && last_tile) {
+            // ---- split over k: one fence for everything this CTA published, then one ticket per
+            //      row block it worked on; the CTA that completes a row block adds the slices in order
+            __threadfence();
+            __syncthreads();
+            for (int rb2 = blockIdx.x; rb2 < group_rbs; rb2 += gridDim.x) {
+                const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb2;
+                if (tid == 0) {
+                    const int old = atomicAdd(p.rb_tickets + grb, 1);
+                    s_last = (old == n_ks - 1);
+                    if (s_last) p.rb_tickets[grb] = 0;
+                }
+                __syncthreads();
+                if (s_last) {
+                    __threadfence();
+                    for (int e = tid; e < out_rows * p.batch; e += kFThreads) {
+                        const int r = e / p.batch, b = e - r * p.batch;
+                        float ss = 0.f;
+                        if (gain)
+                            for (int s2 = 0; s2 < n_ks; ++s2) ss += __ldcg(p.ssq + ((size_t)grb * n_ks + s2) * p.batch + b);
+                        auto acc_of = [&](int row) {
+                            float a = 0.f;
+                            for (int s2 = 0; s2 < n_ks; ++s2) a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
+                            return a;
+                        };
+                        if (p.stage == kStageGateUp) {
+                            const int m = rb2 * out_rows + r;
+                            if (m < p.F) stage_finish(p, m, b, acc_of(m), acc_of(p.F + m), ss);
+                        } else {
+                            const int local = rb2 * kFRows + r;
+                            if (local < (p.stage == kStageTower ? p.T : n_rows)) stage_finish(p, group_row0 + local, b, acc_of(group_row0 + local), 0.f, ss);
+                        }
+                    }
+                }
+                __syncthreads();
+            }
         }
     }
 }
@@ -317,6 +344,9 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
 {
     char* sc = static_cast<char*>(scratch);
     const FullScratch L = full_scratch_layout(d_model, T, F, batch);
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        sms = 148;
     float* abc = reinterpret_cast<float*>(sc + L.abc);
     float* z = reinterpret_cast<float*>(sc + L.z);
     float* h = reinterpret_cast<float*>(sc + L.h);
@@ -328,9 +358,17 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
     p.ssq = reinterpret_cast<float*>(sc + L.ssq);
     p.rb_tickets = reinterpret_cast<int32_t*>(sc + L.tickets);
     auto launch = [&](bool dep) {
-        cudaError_t le = batch <= 4
-            ? launch_ex(full_head_stage_kernel<4, 2048>, dim3(p.row_blocks, ceil_div(p.K, 2048)), dim3(kFThreads), 0, st, dep, p)
-            : launch_ex(full_head_stage_kernel<16, 512>, dim3(p.row_blocks, ceil_div(p.K, 512)), dim3(kFThreads), 0, st, dep, p);
+        const int kt = batch <= 4 ? 2048 : 512;
+        const int n_ks = ceil_div(p.K, kt);
+        const int groups = p.stage == kStageTower ? 3 : 1;
+        const int group_rbs = p.stage == kStageTower ? ceil_div(T, kFRows) : p.row_blocks;
+        // small batches: about one CTA per SM in total, each walking several row blocks; large
+        // batches (narrow tiles, many k slices): one row block per CTA
+        int gx = batch <= 4 ? sms / (n_ks * groups) : group_rbs;
+        gx = std::max(1, std::min(gx, group_rbs));
+        const dim3 grid(gx, n_ks, groups);
+        cudaError_t le = batch <= 4 ? launch_ex(full_head_stage_kernel<4, 2048>, grid, dim3(kFThreads), 0, st, dep, p)
+                                    : launch_ex(full_head_stage_kernel<16, 512>, grid, dim3(kFThreads), 0, st, dep, p);
         if (le == cudaSuccess && launches) ++*launches;
         return le;
     };
