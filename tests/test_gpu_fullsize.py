@@ -149,3 +149,19 @@ def test_hybrid_shape_fixed_and_gated_layers():
     check_units(wl, st, 0, seq, out, lse, flags, units)
     assert np.isfinite(scores).all()
     assert ctx.read_device_status() == 0
+
+
+def test_longest_paper_context_one_layer():
+    """The paper's longest prompt (516,788 tokens, s=4, w=2048, 16q/8kv heads, D=128) on one layer:
+    32,300 pages per unit, every span a partial of some unit; Full and Local units sampled."""
+    wl = workloads.make("paper", L=1, windows=[2048], sinks=[4], gated=[1],
+                        seq_lens0=np.array([516788], np.int32), steps=2)
+    st = workloads.materialize(wl)
+    ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks))
+    seq = np.asarray(wl.seq_lens0)
+    out1, lse1, _, fl1, _ = run_graph_step(wl, st, ctx, 0, [1])
+    check_units(wl, st, 0, seq, out1, lse1, fl1, [(0, 0, 5)])
+    out0, lse0, _, fl0, _ = run_graph_step(wl, st, ctx, 0, [0])
+    check_units(wl, st, 0, seq, out0, lse0, fl0, [(0, 0, 0), (0, 0, 7)])
+    assert (lse1 >= lse0 - 1e-4).all()
+    assert ctx.read_device_status() == 0
