@@ -46,6 +46,9 @@ def parse():
                     help="alias the layers onto this many physical cache slices (bounds memory for the large "
                          "configs); -1 = one slice per layer")
     ap.add_argument("--context", type=int, default=0, help="override every request's context length")
+    ap.add_argument("--reuse-local", action="store_true",
+                    help="variant: the gated pass reads only the positions Local did not and merges with the "
+                         "Local result (exact here because the synthetic stack uses the same queries for both)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -171,7 +174,8 @@ def config_dict(wl, args, realised):
             "recall_rate_target": wl.recall_rate, "recall_rate_realised": realised,
             "global_batch": wl.B * args.gpus, "parallelism": f"dp{args.gpus} (requests sharded, no collective)",
             "l2": "flushed between timed steps (256 MiB write, untimed)",
-            "launch": "one CUDA graph replay per step"}
+            "launch": "one CUDA graph replay per step",
+            "gated_pass": "remainder S^F minus S^L merged with Local" if getattr(wl, "reuse_local", False) else "recomputes all of S^F"}
 
 
 PAPER_LENGTHS = [4139, 15918, 31400, 63852, 128852, 261696, 516788]
@@ -271,6 +275,7 @@ def main():
         wl.kv_index = None
     if args.context > 0:
         wl.seq_lens0 = np.full(wl.B, args.context, np.int32)
+    wl.reuse_local = bool(args.reuse_local)
     if args.impl == "reference":
         reference_arm(args, wl)
         return

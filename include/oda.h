@@ -91,8 +91,17 @@ typedef struct {
     int32_t head_d_ext;
     int32_t head_use_attn_out;
     int32_t head_d_hidden;
-    int32_t reserved;           /* 0; 1 = launch every kernel fully serialised (no programmatic
-                                 * dependent launch between the kernels of a step) */
+    int32_t options;            /* bit 0: launch every kernel fully serialised (no programmatic
+                                 * dependent launch between the kernels of a step).
+                                 * bit 1: the gated pass reads only the positions Local did not,
+                                 * S^F \ S^L = [min(s,t), t-w), and merges them with the Local result
+                                 * already in out/lse by log-sum-exp.  That is exact only when the
+                                 * Full branch's queries are the Local branch's (an attention-only
+                                 * stack, or the first layer of a model): q_full must equal q_local,
+                                 * out/lse must hold the Local pass of the same step, lse must not be
+                                 * NULL in oda_full_decode_gated.  The paper's runtime recomputes Full
+                                 * from scratch; this variant makes a recalled step cost exactly one
+                                 * Full pass in bytes.  TMA variant only. */
 } oda_config_t;
 
 /* Lifetime.  oda_create validates and copies the config (host only, no device work).

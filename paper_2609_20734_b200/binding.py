@@ -47,7 +47,7 @@ class _Config(ctypes.Structure):
         ("kv_layer_stride", ctypes.c_int64), ("kv_block_stride", ctypes.c_int64),
         ("kv_token_stride", ctypes.c_int64), ("kv_head_stride", ctypes.c_int64),
         ("head_d_ext", ctypes.c_int32), ("head_use_attn_out", ctypes.c_int32),
-        ("head_d_hidden", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("head_d_hidden", ctypes.c_int32), ("options", ctypes.c_int32),
     ]
 
 
@@ -151,6 +151,7 @@ class OdaConfig:
     head_use_attn_out: int = 1
     head_d_hidden: int = 0
     serialize_launches: int = 0   # 1 = no programmatic dependent launch between the kernels of a step
+    reuse_local: int = 0          # 1 = the gated pass reads only S^F \ S^L and merges with Local (q_full == q_local)
     _keep: list = field(default_factory=list, repr=False)
 
     def to_c(self) -> _Config:
@@ -167,7 +168,8 @@ class OdaConfig:
             arr(self.layer_window, np.int32), arr(self.layer_sinks, np.int32),
             arr(self.layer_gated, np.uint8), arr(self.layer_kv_index, np.int32),
             self.kv_layer_stride, self.kv_block_stride, self.kv_token_stride, self.kv_head_stride,
-            self.head_d_ext, self.head_use_attn_out, self.head_d_hidden, self.serialize_launches)
+            self.head_d_ext, self.head_use_attn_out, self.head_d_hidden,
+            (1 if self.serialize_launches else 0) | (2 if self.reuse_local else 0))
 
 
 def _ptr(t) -> Optional[int]:

@@ -23,7 +23,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct WsLayout {
     size_t status, layers, tickets, head_partial, head_pre, head_rb_tickets, sm_claims, sm_bytes, cum_share, partials;
-    size_t st_q_local, st_q_full, st_feat, st_override, st_out, st_lse, st_scores, st_logits, st_flags;
+    size_t st_q_local, st_q_full, st_feat, st_override, st_out, st_lse, st_scores, st_logits, st_flags, own_lse;
     size_t total;
 };
 
@@ -58,6 +58,7 @@ struct oda_ctx {
     int64_t blocks_bound = 1;
     int64_t launches = 0;
     bool use_pdl = true;  // programmatic dependent launch between the kernels of a step
+    bool reuse_local = false;  // the gated pass reads only S^F \ S^L and merges with the Local result
     std::string err;
 };
 
@@ -105,6 +106,7 @@ void compute_layout(oda_ctx* c)
     w.st_scores = take(B * 4);
     w.st_logits = take(B * 4);
     w.st_flags = take(B);
+    w.own_lse = take(L * B * Hq * 4);  // lse of the step when the caller keeps none (remainder mode needs it)
     w.total = off;
 }
 
@@ -170,7 +172,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
         int n = 0;
         for (int l = lb; l < le; ++l) n += (c->layers[l].cls == i);
         p.cls_layers_in_call[i] = n;
-        if (n && (mode == 0 || c->cls_gated[i])) any = true;
+        if (n && (mode == 0 || c->cls_gated[i])) any = true;  // modes 1 and 2 touch gated layers only
     }
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
     p.advance_seq_lens = advance;
@@ -313,8 +315,17 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         delete c;
         return ODA_ERR_UNSUPPORTED;  // layer stride is not a whole number of blocks
     }
-    c->use_pdl = cfg->reserved == 0;  // reserved = 1 turns programmatic dependent launch off
+    if (cfg->options < 0 || cfg->options > 3) {
+        delete c;
+        return ODA_ERR_INVALID_ARG;
+    }
+    c->use_pdl = (cfg->options & 1) == 0;
+    c->reuse_local = (cfg->options & 2) != 0;
     c->variant = cfg->variant == ODA_VARIANT_AUTO ? (tma_ok ? ODA_VARIANT_TMA_MMA : ODA_VARIANT_SIMT) : cfg->variant;
+    if (c->reuse_local && c->variant != ODA_VARIANT_TMA_MMA) {
+        delete c;
+        return ODA_ERR_UNSUPPORTED;  // the remainder-only gated pass exists in the TMA variant only
+    }
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
@@ -433,7 +444,8 @@ oda_status_t oda_full_decode_gated(oda_ctx_t* c, int32_t lb, int32_t le, int32_t
     oda_status_t s = check_attn_args(c, lb, le, batch, q, k, v, bt, sl, out);
     if (s != ODA_OK || batch == 0 || lb == le) return s;
     if (!flags) return fail(c, ODA_ERR_INVALID_ARG, "flags is null");
-    return launch_attention(c, 1, lb, le, batch, q, k, v, bt, sl, flags, out, lse,
+    if (c->reuse_local && !lse) return fail(c, ODA_ERR_INVALID_ARG, "the remainder-only gated pass needs the Local pass's lse");
+    return launch_attention(c, c->reuse_local ? 2 : 1, lb, le, batch, q, k, v, bt, sl, flags, out, lse,
                             static_cast<cudaStream_t>(stream));
 }
 
@@ -586,8 +598,10 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
                                  const_cast<void*>(a->v_cache), a->block_table, a->seq_lens, stream);
         if (s != ODA_OK) return s;
     }
+    float* step_lse = a->lse;
+    if (!step_lse && c->reuse_local) step_lse = reinterpret_cast<float*>(c->ws + c->lay.own_lse);
     s = launch_attention(c, 0, 0, L, B, a->q_local, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
-                         nullptr, a->out, a->lse, st);
+                         nullptr, a->out, step_lse, st);
     if (s != ODA_OK) return s;
     const char* attn_last = nullptr;
     if (c->last_gated >= 0 && f.head_use_attn_out)
@@ -613,8 +627,8 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     bool advanced = false;
     if (c->last_gated >= 0) {
         // the Full kernel is the last reader of seq_lens in the step: it also advances them
-        s = launch_attention(c, 1, 0, L, B, qf, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
-                             fused_decision ? a->override_flags : a->flags, a->out, a->lse, st,
+        s = launch_attention(c, c->reuse_local ? 2 : 1, 0, L, B, qf, a->k_cache, a->v_cache, a->block_table, a->seq_lens,
+                             fused_decision ? a->override_flags : a->flags, a->out, step_lse, st,
                              a->advance_seq_lens ? a->seq_lens : nullptr, &advanced, fused_decision ? a : nullptr);
         if (s != ODA_OK) return s;
     }

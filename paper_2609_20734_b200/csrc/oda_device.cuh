@@ -38,7 +38,8 @@ struct AttnParams {
     int64_t kv_layer_stride, kv_block_stride, kv_token_stride, kv_head_stride;
     int32_t layer_begin, layer_end, batch, max_batch;
     int32_t num_q_heads, num_kv_heads, max_blocks_per_seq, out_bf16;
-    int32_t mode;          // 0 = Local (Eq. 1 S^L), 1 = gated Full (S^F)
+    int32_t mode;          // 0 = Local (Eq. 1 S^L), 1 = gated Full (S^F), 2 = gated remainder S^F \ S^L,
+                           //     merged into the Local result that out/lse already hold
     int32_t ncls;
     int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
     int32_t max_items;
@@ -112,7 +113,8 @@ struct Item {
 };
 
 // Eq. 1 in 0-based form.  Local: sinks [0, min(s,t)), window [max(0,t-w), t); when they touch
-// or overlap the set is the single range [0, t).  Full: [0, t).
+// or overlap the set is the single range [0, t).  Full: [0, t).  Remainder (mode 2): the gap
+// [min(s,t), max(0,t-w)) between sinks and window, empty when Local already covers everything.
 struct Ranges {
     int32_t lo, hi;       // window (or whole) segment
     int32_t sink_hi;      // 0 if there is no separate sink segment
@@ -126,6 +128,14 @@ __device__ __forceinline__ Ranges eq1_ranges(int mode, int t, int w, int s)
     r.sink_hi = 0;
     if (mode == 1) {
         r.lo = 0;
+    } else if (mode == 2) {
+        const int s_eff = s < t ? s : t;
+        const int lo = t - w > 0 ? t - w : 0;
+        r.lo = s_eff;
+        r.hi = lo > s_eff ? lo : s_eff;  // empty when the window reaches the sinks
+        r.pg0 = r.lo / kPage;
+        r.pg1 = r.hi > r.lo ? (r.hi + kPage - 1) / kPage : r.pg0;
+        return r;
     } else {
         int s_eff = s < t ? s : t;
         int lo = t - w > 0 ? t - w : 0;
@@ -164,7 +174,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     // issue every global load of the plan before using any of them: one memory latency, not three
     const bool has_b = tid < B;  // blockDim.x >= kMaxBatch
     const int t_raw = has_b ? p.seq_lens[tid] : 1;
-    const int fl_raw = (has_b && p.mode == 1) ? p.flags[tid] : 1;
+    const int fl_raw = (has_b && p.mode != 0) ? p.flags[tid] : 1;
     LayerInfo li0, li1;
     li0.cls = li0.kv_index = li1.cls = li1.kv_index = 0;
     if (tid < nl) li0 = p.layers[p.layer_begin + tid];
@@ -191,7 +201,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         for (int b0 = 0; b0 < B; b0 += 32) {
             const int b = b0 + lane;
             int np = 0;
-            if (b < B && p.cls_layers_in_call[c] > 0 && (p.mode == 0 || (p.cls_gated[c] && pl.active[b]))) {
+            if (b < B && p.cls_layers_in_call[c] > 0 && (p.mode == 0 || (p.cls_gated[c] && pl.active[b]))) {  // modes 1 and 2 are gated
                 const int t = pl.seq[b];
                 if (t < 1) {
                     atomicOr(p.status, kStatusBadSeqLen);

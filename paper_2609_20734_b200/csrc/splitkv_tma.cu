@@ -338,31 +338,55 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         const int hrow = lane >> 2, qc = (lane & 3) * 2;
         const float kLn2 = 0.6931471805599453f;
         auto store_final = [&](const Item& it, const float (&o)[D / 16][4], const float4& ml) {
+            // remainder mode: the Local lse is read by every lane of a head before any lane replaces it
+            float l_old2[2] = {0.f, 0.f};
+            if (p.mode == 2) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (qc + e < G)
+                        l_old2[e] = p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + it.g * G + qc + e] * 1.4426950408889634f;
+            }
+            __syncwarp();
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int hg = qc + e;
                 if (hg >= G) continue;
-                const float mm = e ? ml.z : ml.x, ll = e ? ml.w : ml.y;
-                const float inv = 1.f / ll;
+                float mm = e ? ml.z : ml.x, ll = e ? ml.w : ml.y;
                 const int h = it.g * G + hg;
                 const size_t idx = (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h) * D + hrow;
+                const size_t lidx = ((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h;
+                // remainder mode: out/lse hold the Local result of the same queries; fold it in as
+                // one more partial of weight e^lse (value out, already normalised)
+                float wa = 0.f, wb = 1.f;
+                if (p.mode == 2) {
+                    const float l_old = l_old2[e];  // log2 units
+                    const float mu = fmaxf(l_old, mm);
+                    wa = ex2(l_old - mu);
+                    wb = ex2(mm - mu);
+                    ll = wa + wb * ll;
+                    mm = mu;
+                }
+                const float inv = 1.f / ll;
                 if (p.out_bf16) {
                     __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.out) + idx;
 #pragma unroll
                     for (int n = 0; n < D / 16; ++n) {
-                        ob[n * 16] = __float2bfloat16_rn(o[n][e] * inv);
-                        ob[n * 16 + 8] = __float2bfloat16_rn(o[n][2 + e] * inv);
+                        const float a0 = p.mode == 2 ? wa * __bfloat162float(ob[n * 16]) : 0.f;
+                        const float a1 = p.mode == 2 ? wa * __bfloat162float(ob[n * 16 + 8]) : 0.f;
+                        ob[n * 16] = __float2bfloat16_rn((a0 + wb * o[n][e]) * inv);
+                        ob[n * 16 + 8] = __float2bfloat16_rn((a1 + wb * o[n][2 + e]) * inv);
                     }
                 } else {
                     float* of = reinterpret_cast<float*>(p.out) + idx;
 #pragma unroll
                     for (int n = 0; n < D / 16; ++n) {
-                        of[n * 16] = o[n][e] * inv;
-                        of[n * 16 + 8] = o[n][2 + e] * inv;
+                        const float a0 = p.mode == 2 ? wa * of[n * 16] : 0.f;
+                        const float a1 = p.mode == 2 ? wa * of[n * 16 + 8] : 0.f;
+                        of[n * 16] = (a0 + wb * o[n][e]) * inv;
+                        of[n * 16 + 8] = (a1 + wb * o[n][2 + e]) * inv;
                     }
                 }
-                if (p.lse && hrow == 0)
-                    p.lse[((size_t)it.layer * p.batch + it.b) * p.num_q_heads + h] = (mm + log2f(ll)) * kLn2;
+                if (p.lse && hrow == 0) p.lse[lidx] = (mm + log2f(ll)) * kLn2;
             }
         };
         for (uint32_t k = 0;; ++k) {

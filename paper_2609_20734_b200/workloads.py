@@ -38,6 +38,7 @@ class Workload:
     schedule: str = "bernoulli"      # "bernoulli" | "periodic" | "head"
     seed: int = BASE_SEED
     threshold: float = 0.5
+    reuse_local: bool = False        # gated pass reads only S^F \ S^L (valid here: q_full == q_local)
 
     @property
     def G(self):
@@ -78,8 +79,8 @@ class Workload:
         plus the whole history for flagged requests on gated layers."""
         kb = self.kv_token_bytes
         local = sum(self.local_tokens(l, int(t)) for l in range(self.L) for t in seq_lens) * kb
-        full = sum(int(t) for l in range(self.L) if self.gated[l]
-                   for t, f in zip(seq_lens, flags) if f) * kb
+        full = sum(int(t) - (self.local_tokens(l, int(t)) if self.reuse_local else 0)
+                   for l in range(self.L) if self.gated[l] for t, f in zip(seq_lens, flags) if f) * kb
         return local, full
 
     def override_flags(self, step):
@@ -227,4 +228,5 @@ def oda_config(wl: Workload, num_blocks: int, **kw):
         max_blocks_per_seq=wl.max_blocks_per_seq, layer_window=wl.windows, layer_sinks=wl.sinks,
         layer_gated=wl.gated, layer_kv_index=wl.kv_index, kv_layer_stride=st["layer"],
         kv_block_stride=st["block"], kv_token_stride=st["token"], kv_head_stride=st["head"],
-        head_d_ext=d_ext, head_use_attn_out=use_attn, head_d_hidden=d_h, **kw)
+        head_d_ext=d_ext, head_use_attn_out=use_attn, head_d_hidden=d_h,
+        **{"reuse_local": int(wl.reuse_local), **kw})

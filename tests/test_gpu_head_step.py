@@ -231,3 +231,38 @@ def test_step_flag_invariants_on_device():
     torch.cuda.synchronize()
     for l in range(wl.L):
         assert torch.equal(res["ones"][l], full[l] if wl.gated[l] else loc[l])  # all flags 1 => Full on gated layers
+
+
+def test_remainder_only_gated_pass_equals_full():
+    """Option 'reuse_local': the gated pass reads only S^F \\ S^L and merges with the Local result.
+    With q_full == q_local that is Full attention: same oracle bar, and within rounding of the
+    recompute-from-scratch path; requests whose window already covers everything are left alone."""
+    L = 4
+    wl = workloads.make("batched", L=L, B=6, windows=[64, 32, 64, 32], sinks=[4, 0, 4, 0], gated=[1, 0, 1, 0],
+                        seq_lens0=np.array([100, 900, 33, 2500, 68, 69], np.int32), steps=2, head=(0, 1, 16))
+    st = workloads.materialize(wl)
+    head = wl.head_host()
+    B, shape = wl.B, (wl.L, wl.B, wl.Hq, wl.D)
+    ov_h = np.array([1, 1, 1, 0, 1, 1], np.uint8)
+    ov = torch.from_numpy(ov_h).cuda()
+    q = workloads.q_device(wl, 0)
+    outs = {}
+    for reuse in (0, 1):
+        cfg = workloads.oda_config(wl, st.num_blocks, reuse_local=reuse)
+        ctx = binding.OdaContext(cfg)
+        out = torch.zeros(shape, device="cuda")
+        lse = torch.zeros(shape[:3], device="cuda")
+        scores = torch.zeros(B, device="cuda")
+        flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+        for keep_lse in (True, False):   # the step keeps its own lse when the caller passes none
+            ctx.step(ctx.step_args(B, q, st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, scores, flags,
+                                   head=st.head, override_flags=ov, lse=lse if keep_lse else None))
+            torch.cuda.synchronize()
+            outs[(reuse, keep_lse)] = (out.cpu().numpy().copy(), lse.cpu().numpy().copy())
+        assert ctx.read_device_status() == 0
+    ref = _oracle_step(wl, st.table_host, st.num_blocks, np.asarray(wl.seq_lens0), 0, head, 0.5, ov_h)
+    for key, (o, l) in outs.items():
+        gh.assert_close(o, ref.out, gh.ATOL_OUT, f"reuse={key}")
+    gh.assert_close(outs[(1, True)][1], ref.lse, gh.ATOL_LSE, "merged lse")
+    np.testing.assert_allclose(outs[(1, True)][0], outs[(0, True)][0], rtol=0, atol=1e-5)
+    np.testing.assert_array_equal(outs[(1, False)][0], outs[(1, True)][0])
