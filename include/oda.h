@@ -158,6 +158,28 @@ oda_status_t oda_recall_score(oda_ctx_t* ctx, int32_t batch, const float* feat_e
                               uint8_t* flags, int32_t* counters, void* stream);
 
 /*
+ * The same head split for KV-head tensor parallelism (the paper runs on one GPU; this is how its
+ * Algorithm 1 shards when every rank owns num_kv_heads of the model's KV heads, the query heads
+ * of their groups, and the matching columns of W1).  A context is created with the RANK's head
+ * counts; head_d_ext is non-zero only on the rank that owns the external features.
+ *   oda_recall_preact:   pre_out[b][j] = sum over this rank's input columns of W1[j][col] x[b][col]
+ *     (no bias).  W1_cols points at the rank's first column inside row 0 of the full matrix and
+ *     w1_row_stride is the full row length in floats.  pre_out [batch, d_hidden] fp32 device.
+ *   -- the caller sums pre_out over the ranks (one all-reduce of batch x d_hidden floats) --
+ *   oda_recall_finalize: z = w2 . SiLU(pre_sum + b1) + b2 and the decision rule of
+ *     oda_recall_score; every rank that holds the same pre_sum writes the same flags.
+ * Summation order differs from oda_recall_score, so scores agree to fp32 rounding, not bitwise.
+ * One launch each; neither synchronises.
+ */
+oda_status_t oda_recall_preact(oda_ctx_t* ctx, int32_t batch, const float* feat_ext,
+                               const void* attn_out_last, const float* W1_cols, int64_t w1_row_stride,
+                               float* pre_out, void* stream);
+oda_status_t oda_recall_finalize(oda_ctx_t* ctx, int32_t batch, const float* pre_sum, const float* b1,
+                                 const float* w2, const float* b2, float threshold,
+                                 const uint8_t* override_flags, float* scores, float* logits,
+                                 uint8_t* flags, int32_t* counters, void* stream);
+
+/*
  * The paper's own recall head (appendix "Recall-head architecture"; Eq. 2): three
  * RMSNorm -> Linear(d_model -> d_tower) -> SiLU towers over (h_{t-1}, E(x_t), h_t^L), the interaction
  * vector u = [a;b;c;a.b;|a-b|;a.c;|a-c|;b.c;|b-c|], z0 = (a+b+c+SiLU(W_f u + b_f))/2, n_blocks

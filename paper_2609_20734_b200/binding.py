@@ -25,7 +25,7 @@ EXPORTS = [
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
-    "oda_recall_score_full",
+    "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize",
 ]
 
 
@@ -94,6 +94,10 @@ def load_library():
         lib.oda_set_workspace.argtypes = [vp, vp, ctypes.c_size_t, vp]
         lib.oda_local_decode.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_recall_score.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp]
+        lib.oda_recall_preact.argtypes = [vp, i32, vp, vp, vp, ctypes.c_int64, vp, vp]
+        lib.oda_recall_preact.restype = i32
+        lib.oda_recall_finalize.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp]
+        lib.oda_recall_finalize.restype = i32
         lib.oda_full_decode_gated.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
         lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
@@ -256,6 +260,20 @@ class OdaContext:
             self._h, batch, _ptr(feat_ext), _ptr(attn_out_last), _ptr(W1), _ptr(b1), _ptr(w2), _ptr(b2),
             float(threshold), _ptr(override_flags), _ptr(scores), _ptr(logits), _ptr(flags),
             _ptr(counters), _stream() if stream is None else stream), "oda_recall_score")
+
+    def recall_preact(self, batch, feat_ext, attn_out_last, W1_cols, w1_row_stride, pre_out, stream=None):
+        """This rank's share of W1 x; W1_cols is a device address (int) or a tensor."""
+        w = W1_cols if isinstance(W1_cols, int) else _ptr(W1_cols)
+        self._check(self.lib.oda_recall_preact(
+            self._h, batch, _ptr(feat_ext), _ptr(attn_out_last), w, int(w1_row_stride), _ptr(pre_out),
+            _stream() if stream is None else stream), "oda_recall_preact")
+
+    def recall_finalize(self, batch, pre_sum, b1, w2, b2, threshold, override_flags, scores, logits, flags,
+                        counters=None, stream=None):
+        self._check(self.lib.oda_recall_finalize(
+            self._h, batch, _ptr(pre_sum), _ptr(b1), _ptr(w2), _ptr(b2), float(threshold),
+            _ptr(override_flags), _ptr(scores), _ptr(logits), _ptr(flags), _ptr(counters),
+            _stream() if stream is None else stream), "oda_recall_finalize")
 
     def full_decode_gated(self, layer_begin, layer_end, batch, q_full, k_cache, v_cache, block_table,
                           seq_lens, flags, out, lse=None, stream=None):

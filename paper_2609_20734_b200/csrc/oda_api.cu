@@ -489,10 +489,74 @@ oda_status_t oda_recall_score(oda_ctx_t* c, int32_t batch, const float* feat_ext
     p.attn_bf16 = f.out_dtype;
     p.max_batch = f.max_batch;
     p.threshold = threshold;
+    p.w1_stride = p.d_ext + p.d_attn;
     p.vec4 = (p.d_ext % 4 == 0) && (p.d_attn % 4 == 0) && aligned16(W1) && aligned16(feat_ext) &&
              aligned16(attn_out_last);
     cudaError_t e = launch_recall_head(p, static_cast<cudaStream_t>(stream), c->use_pdl);
     if (e != cudaSuccess) return cuda_fail(c, e, "recall head launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
+oda_status_t oda_recall_preact(oda_ctx_t* c, int32_t batch, const float* feat_ext, const void* attn_out_last,
+                               const float* W1_cols, int64_t w1_row_stride, float* pre_out, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0) return ODA_OK;
+    const oda_config_t& f = c->cfg;
+    if (f.head_d_hidden <= 0) return fail(c, ODA_ERR_INVALID_ARG, "no recall head configured");
+    HeadParams p;
+    std::memset(&p, 0, sizeof p);
+    p.d_hidden = f.head_d_hidden;
+    p.d_ext = f.head_d_ext;
+    p.d_attn = f.head_use_attn_out ? f.num_q_heads * f.head_dim : 0;
+    if (!W1_cols || !pre_out) return fail(c, ODA_ERR_INVALID_ARG, "W1_cols or pre_out is null");
+    if (p.d_ext > 0 && !feat_ext) return fail(c, ODA_ERR_INVALID_ARG, "feat_ext is null but head_d_ext > 0");
+    if (p.d_attn > 0 && !attn_out_last) return fail(c, ODA_ERR_INVALID_ARG, "attn_out_last is null but head_use_attn_out is set");
+    if (p.d_ext + p.d_attn < 1) return fail(c, ODA_ERR_INVALID_ARG, "the head has no input on this rank");
+    if (w1_row_stride < p.d_ext + p.d_attn) return fail(c, ODA_ERR_INVALID_ARG, "w1_row_stride is smaller than this rank's column count");
+    p.feat_ext = feat_ext;
+    p.attn_out = attn_out_last;
+    p.W1 = W1_cols;
+    p.w1_stride = w1_row_stride;
+    p.pre_out = pre_out;
+    p.pre = reinterpret_cast<float*>(c->ws + c->lay.head_pre);
+    p.rb_tickets = reinterpret_cast<int32_t*>(c->ws + c->lay.head_rb_tickets);
+    p.batch = batch;
+    p.attn_bf16 = f.out_dtype;
+    p.max_batch = f.max_batch;
+    p.vec4 = (p.d_ext % 4 == 0) && (p.d_attn % 4 == 0) && (w1_row_stride % 4 == 0) && aligned16(W1_cols) &&
+             aligned16(feat_ext) && aligned16(attn_out_last);
+    cudaError_t e = launch_recall_head(p, static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "recall head (first layer) launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
+oda_status_t oda_recall_finalize(oda_ctx_t* c, int32_t batch, const float* pre_sum, const float* b1,
+                                 const float* w2, const float* b2, float threshold, const uint8_t* override_flags,
+                                 float* scores, float* logits, uint8_t* flags, int32_t* counters, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0) return ODA_OK;
+    if (c->cfg.head_d_hidden <= 0) return fail(c, ODA_ERR_INVALID_ARG, "no recall head configured");
+    if (!pre_sum || !b1 || !w2 || !b2 || !scores || !flags) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    HeadParams p;
+    std::memset(&p, 0, sizeof p);
+    p.d_hidden = c->cfg.head_d_hidden;
+    p.b1 = b1; p.w2 = w2; p.b2 = b2;
+    p.override_flags = override_flags;
+    p.scores = scores;
+    p.logits = logits;
+    p.flags = flags;
+    p.counters = counters;
+    p.batch = batch;
+    p.threshold = threshold;
+    cudaError_t e = launch_recall_finalize(p, pre_sum, static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "recall head (second layer) launch");
     c->launches += 1;
     return ODA_OK;
 }

@@ -52,6 +52,8 @@ struct HeadParams {
     float* pre;                 // [K slices][d_hidden][max_batch] partial pre-activations
     int32_t* ticket;            // one int, zero between launches
     int32_t* rb_tickets;        // [row blocks], zero between launches
+    float* pre_out;             // non-null: stop after W1 x and write [batch][d_hidden] sums (no bias)
+    int64_t w1_stride;          // floats between rows of W1 (d_ext + d_attn unless W1 is a column slice)
     int32_t batch, d_ext, d_attn, d_hidden, attn_bf16, max_batch;
     int32_t vec4;               // 128-bit loads are legal: widths multiples of 4, pointers 16-byte aligned
     float threshold;
@@ -62,6 +64,8 @@ constexpr int kMaxHeadBatch = 128;
 int recall_head_grid(int d_hidden);
 int recall_head_ksplits(int d_in);
 cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl = false);
+// z = b2 + w2 . SiLU(pre_sum + b1) and the decision, from summed first-layer products [batch][d_hidden]
+cudaError_t launch_recall_finalize(const HeadParams& p, const float* pre_sum, cudaStream_t st, bool pdl = false);
 cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st, bool pdl = false);
 
 }  // namespace oda

@@ -61,12 +61,12 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
     for (int c = 0; c < 4; ++c) {
         const int i = k0 + c * 128 + lane * 4;
         if (j < p.d_hidden && p.vec4 && i < d_in) {
-            const float4 v = __ldg(reinterpret_cast<const float4*>(p.W1 + (size_t)j * d_in + i));
+            const float4 v = __ldg(reinterpret_cast<const float4*>(p.W1 + (size_t)j * p.w1_stride + i));
             w[c][0] = v.x; w[c][1] = v.y; w[c][2] = v.z; w[c][3] = v.w;
         } else {
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                w[c][e] = (j < p.d_hidden && i + e < d_in) ? __ldg(p.W1 + (size_t)j * d_in + i + e) : 0.f;
+                w[c][e] = (j < p.d_hidden && i + e < d_in) ? __ldg(p.W1 + (size_t)j * p.w1_stride + i + e) : 0.f;
         }
     }
     for (int b0 = 0; b0 < p.batch; b0 += kHeadBT) {
@@ -121,6 +121,16 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    if (p.pre_out) {  // column-split head: this rank's share of W1 x, K slices added in order
+        for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
+            const int b = e / kHeadRows, jj = rb * kHeadRows + (e - b * kHeadRows);
+            if (jj >= p.d_hidden) continue;
+            float a = 0.f;
+            for (int s = 0; s < n_ks; ++s) a += __ldcg(p.pre + ((size_t)s * p.d_hidden + jj) * p.max_batch + b);
+            p.pre_out[(size_t)b * p.d_hidden + jj] = a;
+        }
+        return;
+    }
     for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
         const int r = e / p.batch, b = e - r * p.batch;
         const int jj = rb * kHeadRows + r;
@@ -174,6 +184,41 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
     }
 }
 
+// Second half of a column-split head: pre_sum[b][j] holds W1 x summed over the ranks.  One warp
+// per request; lanes take hidden units 32 apart and a fixed shuffle tree adds them, so every
+// rank that holds the same pre_sum takes the same decision.
+__global__ void __launch_bounds__(kHeadThreads) recall_finalize_kernel(const __grid_constant__ HeadParams p,
+                                                                       const float* __restrict__ pre_sum)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * kHeadRows + warp;
+    if (b >= p.batch) return;
+    float zp = 0.f;
+    for (int j = lane; j < p.d_hidden; j += 32) {
+        const float a = pre_sum[(size_t)b * p.d_hidden + j] + __ldg(p.b1 + j);
+        zp += __ldg(p.w2 + j) * (a / (1.f + expf(-a)));
+    }
+    for (int o = 16; o; o >>= 1) zp += __shfl_xor_sync(0xffffffffu, zp, o);
+    if (lane == 0) {
+        const float z = __ldg(p.b2) + zp;
+        const float score = 1.f / (1.f + expf(-z));
+        uint8_t f;
+        if (p.override_flags)
+            f = p.override_flags[b] ? 1 : 0;
+        else
+            f = (!isfinite(z) || score > p.threshold) ? 1 : 0;
+        p.scores[b] = score;
+        if (p.logits) p.logits[b] = z;
+        p.flags[b] = f;
+        if (p.counters) {
+            p.counters[2 * b] += 1;
+            p.counters[2 * b + 1] += f;
+        }
+    }
+}
+
 // no head configured: flags are the override
 __global__ void copy_flags_kernel(const uint8_t* __restrict__ ov, uint8_t* __restrict__ flags,
                                   float* scores, float* logits, int32_t* counters, int batch)
@@ -209,6 +254,12 @@ cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl)
                          p.logits, p.counters, p.batch);
     return launch_ex(recall_head_kernel, dim3(recall_head_grid(p.d_hidden), recall_head_ksplits(p.d_ext + p.d_attn)),
                      dim3(kHeadThreads), 0, st, pdl, p);
+}
+
+cudaError_t launch_recall_finalize(const HeadParams& p, const float* pre_sum, cudaStream_t st, bool pdl)
+{
+    return launch_ex(recall_finalize_kernel, dim3((p.batch + kHeadRows - 1) / kHeadRows), dim3(kHeadThreads), 0, st,
+                     pdl, p, pre_sum);
 }
 
 cudaError_t launch_advance_seq_lens(int32_t* seq_lens, int batch, cudaStream_t st, bool pdl)

@@ -1,0 +1,93 @@
+"""KV-head tensor parallelism for one decode step (Algorithm 1 sharded over attention heads).
+
+Rank r of n owns KV heads [r*Hkv/n, (r+1)*Hkv/n), the query heads of their groups and the matching
+columns of the recall head's first layer.  Attention needs no exchange: heads are independent.
+The decision needs one: every rank multiplies its columns of W1 by its slice of the head input,
+the [batch, d_hidden] products are summed over the ranks (the step's only collective), and every
+rank applies bias, SiLU, the second layer and the decision rule to the same sums, so all ranks
+gate the same requests.  Argument marshalling only: the arithmetic runs in the library's kernels
+and the collective in torch.distributed.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+
+@dataclass(frozen=True)
+class HeadShard:
+    """What one rank owns."""
+    rank: int
+    world: int
+    kv_heads: int          # KV heads on this rank
+    q_heads: int           # query heads on this rank
+    kv_head_begin: int     # first global KV head
+    q_head_begin: int      # first global query head
+    d_ext: int             # external head features this rank multiplies (rank 0 owns them all)
+    col_begin: int         # first column of W1 this rank multiplies
+    col_count: int         # number of columns
+    d_in: int              # full row length of W1
+
+
+def head_shard(rank: int, world: int, num_q_heads: int, num_kv_heads: int, head_dim: int,
+               d_ext: int = 0, use_attn_out: bool = True) -> HeadShard:
+    """Contiguous split of the KV heads; the head input is [feat_ext ; attention heads in order]."""
+    if world < 1 or not 0 <= rank < world:
+        raise ValueError("rank outside [0, world)")
+    if num_kv_heads % world or num_q_heads % num_kv_heads:
+        raise ValueError("KV heads must divide evenly over the ranks, and query heads over KV heads")
+    kv = num_kv_heads // world
+    g = num_q_heads // num_kv_heads
+    q = kv * g
+    d_attn = num_q_heads * head_dim if use_attn_out else 0
+    own_ext = d_ext if rank == 0 else 0
+    attn_cols = q * head_dim if use_attn_out else 0
+    col_begin = 0 if rank == 0 else d_ext + rank * attn_cols
+    return HeadShard(rank, world, kv, q, rank * kv, rank * q, own_ext, col_begin, own_ext + attn_cols,
+                     d_ext + d_attn)
+
+
+def sum_over_ranks(t, group=None):
+    """The step's one collective: element-wise sum of a small fp32 tensor over the ranks."""
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    return t
+
+
+def tp_local_and_preact(ctx, shard: HeadShard, batch, q_local, k_cache, v_cache, block_table, seq_lens, out,
+                        *, W1, pre, feat_ext=None, lse=None):
+    """Before the exchange: the Local pass over the rank's heads, then the rank's share of W1 x."""
+    L = ctx.cfg.num_layers
+    ctx.local_decode(0, L, batch, q_local, k_cache, v_cache, block_table, seq_lens, out, lse)
+    gated = [l for l in range(L) if ctx.cfg.layer_gated[l]]
+    # the head reads the Local output of the last gated layer, as the single-GPU step does
+    attn_last = out[gated[-1]] if (ctx.cfg.head_use_attn_out and gated) else None
+    ctx.recall_preact(batch, feat_ext if shard.d_ext else None, attn_last,
+                      W1.data_ptr() + 4 * shard.col_begin, shard.d_in, pre)
+
+
+def tp_decide_and_recompute(ctx, batch, q_full, k_cache, v_cache, block_table, seq_lens, out, *, pre_sum,
+                            b1, w2, b2, threshold, scores, flags, logits=None, lse=None,
+                            override_flags=None, counters=None):
+    """After the exchange: the decision from the summed products, then the gated Full pass."""
+    ctx.recall_finalize(batch, pre_sum, b1, w2, b2, threshold, override_flags, scores, logits, flags, counters)
+    ctx.full_decode_gated(0, ctx.cfg.num_layers, batch, q_full, k_cache, v_cache, block_table, seq_lens,
+                          flags, out, lse)
+
+
+def tp_step(ctx, shard: HeadShard, batch, q_local, k_cache, v_cache, block_table, seq_lens, out, *,
+            W1, b1, w2, b2, threshold, pre, scores, flags, feat_ext=None, q_full=None, logits=None,
+            lse=None, override_flags=None, counters=None, all_reduce=sum_over_ranks):
+    """One decode step on one rank.  `ctx` was created with the rank's head counts (and head_d_ext =
+    shard.d_ext); caches, q and out hold the rank's heads only; W1 is the full [d_hidden, d_in]
+    matrix (each rank reads only its columns).  `pre` is a [batch, d_hidden] fp32 device buffer.
+    """
+    tp_local_and_preact(ctx, shard, batch, q_local, k_cache, v_cache, block_table, seq_lens, out,
+                        W1=W1, pre=pre, feat_ext=feat_ext, lse=lse)
+    all_reduce(pre)
+    tp_decide_and_recompute(ctx, batch, q_local if q_full is None else q_full, k_cache, v_cache, block_table,
+                            seq_lens, out, pre_sum=pre, b1=b1, w2=w2, b2=b2, threshold=threshold,
+                            scores=scores, flags=flags, logits=logits, lse=lse,
+                            override_flags=override_flags, counters=counters)
+    return flags

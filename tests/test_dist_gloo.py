@@ -62,3 +62,89 @@ def test_request_shard_covers_everything_once():
             assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
             sizes = [hi - lo for lo, hi in spans]
             assert max(sizes) - min(sizes) <= 1
+
+
+def _tp_problem():
+    from tests.helpers import make_problem
+    from paper_2609_20734_b200 import synth
+
+    L, B, Hq, Hkv, D, d_ext, d_h = 2, 3, 8, 4, 16, 5, 12
+    prob = make_problem(8, L, B, Hq, Hkv, D, [40, 7, 130])
+    head = dict(W1=synth.gauss_f32_tensor(3, synth.STREAM_W1, (d_h, d_ext + Hq * D), std=0.1),
+                b1=synth.gauss_f32_tensor(3, synth.STREAM_B1, (d_h,), std=0.1),
+                w2=synth.gauss_f32_tensor(3, synth.STREAM_W2, (d_h,), std=0.1),
+                b2=synth.gauss_f32_tensor(3, synth.STREAM_B2, (1,), std=0.1))
+    fe = synth.gauss_f32_tensor(3, synth.STREAM_FEAT, (B, d_ext))
+    return prob, head, fe, d_ext, d_h
+
+
+def _tp_worker(rank, world, port, ret):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import oda_oracle as orc
+    from paper_2609_20734_b200 import tensor_parallel as tp
+
+    prob, head, fe, d_ext, d_h = _tp_problem()
+    L, B, Hq, Hkv, D, lay = prob["L"], prob["B"], prob["Hq"], prob["Hkv"], prob["D"], prob["layout"]
+    sh = tp.head_shard(rank, world, Hq, Hkv, D, d_ext, True)
+    # the rank's heads: a slice of q, and the caches entered at its first KV head
+    q = np.ascontiguousarray(prob["q"][:, :, sh.q_head_begin:sh.q_head_begin + sh.q_heads])
+    off = sh.kv_head_begin * lay.head_stride
+    out, _ = orc.attention("local", q, prob["k"][off:], prob["v"][off:], prob["table"], prob["seq_lens"],
+                           num_kv_heads=sh.kv_heads, block_size=16, layout=lay, layer_window=[16, 16],
+                           layer_sinks=[2, 2])
+    x = out[L - 1].reshape(B, -1)
+    if sh.d_ext:
+        x = np.concatenate([fe.astype(np.float64), x], axis=1)
+    assert x.shape[1] == sh.col_count
+    W = head["W1"][:, sh.col_begin:sh.col_begin + sh.col_count].astype(np.float64)
+    pre = torch.from_numpy(x @ W.T)
+    tp.sum_over_ranks(pre)                           # the step's one collective
+    a = pre.numpy() + head["b1"].astype(np.float64)
+    z = (a / (1.0 + np.exp(-a))) @ head["w2"].astype(np.float64) + float(head["b2"][0])
+    ret[rank] = (sh, out, z)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_kv_head_tensor_parallel_two_ranks_gloo():
+    """Ranks own disjoint KV heads and W1 columns; after one all-reduce of the first-layer
+    products every rank holds the logits of the unsharded head, and the heads' outputs tile
+    the unsharded attention output."""
+    world = 2
+    with mp.Manager() as m:
+        ret = m.dict()
+        mp.spawn(_tp_worker, args=(world, 29613, ret), nprocs=world, join=True)
+        res = dict(ret)
+    from oracle import oda_oracle as orc
+    from tests.helpers import oracle_attention
+
+    prob, head, fe, d_ext, d_h = _tp_problem()
+    whole, _ = oracle_attention(prob, "local", [16, 16], [2, 2])
+    z, _ = orc.recall_head(fe, whole[prob["L"] - 1], head["W1"], head["b1"], head["w2"], head["b2"])
+    cols = []
+    for r in range(world):
+        sh, out, zr = res[r]
+        np.testing.assert_array_equal(out, whole[:, :, sh.q_head_begin:sh.q_head_begin + sh.q_heads])
+        np.testing.assert_allclose(zr, z, rtol=0, atol=1e-12)
+        np.testing.assert_array_equal(zr, res[0][2])     # identical on every rank
+        cols += list(range(sh.col_begin, sh.col_begin + sh.col_count))
+    assert cols == list(range(d_ext + prob["Hq"] * prob["D"]))
+
+
+def test_head_shard_arithmetic():
+    from paper_2609_20734_b200 import tensor_parallel as tp
+    import pytest
+
+    for world in (1, 2, 4, 8):
+        shards = [tp.head_shard(r, world, 32, 8, 128, 24, True) for r in range(world)]
+        assert sum(s.kv_heads for s in shards) == 8 and sum(s.q_heads for s in shards) == 32
+        assert sum(s.col_count for s in shards) == shards[0].d_in == 24 + 32 * 128
+        assert all(a.col_begin + a.col_count == b.col_begin for a, b in zip(shards, shards[1:]))
+        assert all(s.q_head_begin == s.kv_head_begin * 4 for s in shards)
+        assert [s.d_ext for s in shards] == [24] + [0] * (world - 1)
+    with pytest.raises(ValueError):
+        tp.head_shard(0, 3, 32, 8, 128)
+    with pytest.raises(ValueError):
+        tp.head_shard(2, 2, 32, 8, 128)

@@ -1,0 +1,100 @@
+"""KV-head tensor-parallel step: the ranks of a 2- and 4-way split run one after another on one
+GPU (their kernels never wait on each other; the exchange between the two phases is a plain sum
+here), and the assembled result is compared with the unsharded oracle step."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oda_oracle as orc
+from paper_2609_20734_b200 import synth
+from paper_2609_20734_b200 import tensor_parallel as tp
+from tests import gpu_helpers as gh
+from tests.helpers import make_problem
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("world,layout,d_ext", [(2, "hnd", 32), (4, "nhd", 0), (1, "hnd", 6)])
+def test_tensor_parallel_step_matches_unsharded_oracle(world, layout, d_ext):
+    L, B, Hq, Hkv, D, d_h = 3, 5, 8, 4, 128, 40
+    windows, sinks, gated = [64, 32, 64], [4, 0, 4], [1, 1, 0]
+    prob = make_problem(31, L, B, Hq, Hkv, D, [100, 900, 33, 2500, 64], layout=layout)
+    lay = prob["layout"]
+    d_in = d_ext + Hq * D
+    head = dict(W1=synth.gauss_f32_tensor(9, synth.STREAM_W1, (d_h, d_in), std=0.05),
+                b1=synth.gauss_f32_tensor(9, synth.STREAM_B1, (d_h,), std=0.05),
+                w2=synth.gauss_f32_tensor(9, synth.STREAM_W2, (d_h,), std=0.05),
+                b2=synth.gauss_f32_tensor(9, synth.STREAM_B2, (1,), std=0.05), use_attn_out=1)
+    fe = synth.gauss_f32_tensor(9, synth.STREAM_FEAT, (B, d_ext)) if d_ext else None
+    kw = dict(num_kv_heads=Hkv, block_size=16, layout=lay, layer_window=windows, layer_sinks=sinks,
+              layer_gated=gated, head=head, feat_ext=fe, nthreads=4)
+    sc = np.sort(orc.step(prob["q"], None, prob["k"], prob["v"], prob["table"], prob["seq_lens"], tau=0.5, **kw).score)
+    tau = float(0.5 * (sc[2] + sc[3]))              # two of the five requests recall
+    assert sc[3] - tau > 2 * gh.FLAG_BAND and tau - sc[2] > 2 * gh.FLAG_BAND
+    ref = orc.step(prob["q"], None, prob["k"], prob["v"], prob["table"], prob["seq_lens"], tau=tau, **kw)
+    assert ref.flags.sum() == 2
+
+    dev = gh.upload(prob)
+    hd = gh.head_to_device(head)
+    fe_d = None if fe is None else torch.from_numpy(fe).cuda()
+    q_all = dev["q"].view(L, B, Hq, D)
+    ranks = []
+    for r in range(world):
+        sh = tp.head_shard(r, world, Hq, Hkv, D, d_ext, True)
+        rp = dict(prob, Hq=sh.q_heads, Hkv=sh.kv_heads)
+        ctx = gh.make_ctx(rp, windows, sinks, gated, head=(sh.d_ext, 1, d_h))
+        off = sh.kv_head_begin * lay.head_stride      # the rank's heads inside the shared test cache
+        st = dict(sh=sh, ctx=ctx, k=dev["k"][off:], v=dev["v"][off:],
+                  q=q_all[:, :, sh.q_head_begin:sh.q_head_begin + sh.q_heads].contiguous(),
+                  out=torch.full((L, B, sh.q_heads, D), float("nan"), device="cuda"),
+                  lse=torch.full((L, B, sh.q_heads), float("nan"), device="cuda"),
+                  pre=torch.full((B, d_h), float("nan"), device="cuda"),
+                  scores=torch.zeros(B, device="cuda"), logits=torch.zeros(B, device="cuda"),
+                  flags=torch.zeros(B, dtype=torch.uint8, device="cuda"))
+        ranks.append(st)
+    for st in ranks:
+        tp.tp_local_and_preact(st["ctx"], st["sh"], B, st["q"], st["k"], st["v"], dev["table"], dev["seq_lens"],
+                               st["out"], W1=hd["W1"], pre=st["pre"], feat_ext=fe_d, lse=st["lse"])
+    pre_sum = torch.stack([st["pre"] for st in ranks]).sum(0)     # stands in for the all-reduce
+    for st in ranks:
+        tp.tp_decide_and_recompute(st["ctx"], B, st["q"], st["k"], st["v"], dev["table"], dev["seq_lens"],
+                                   st["out"], pre_sum=pre_sum.clone(), b1=hd["b1"], w2=hd["w2"], b2=hd["b2"],
+                                   threshold=tau, scores=st["scores"], flags=st["flags"], logits=st["logits"],
+                                   lse=st["lse"])
+    torch.cuda.synchronize()
+    for st in ranks:
+        assert st["ctx"].read_device_status() == 0
+        np.testing.assert_array_equal(st["flags"].cpu().numpy(), ref.flags)
+        np.testing.assert_allclose(st["scores"].cpu().numpy(), ref.score, rtol=0, atol=gh.ATOL_SCORE)
+        # every rank holds the same sums, so the decisions are bitwise the same
+        assert torch.equal(st["scores"], ranks[0]["scores"]) and torch.equal(st["logits"], ranks[0]["logits"])
+    out = torch.cat([st["out"] for st in ranks], dim=2).cpu().numpy()
+    lse = torch.cat([st["lse"] for st in ranks], dim=2).cpu().numpy()
+    gh.assert_close(out, ref.out, gh.ATOL_OUT, "assembled out")
+    gh.assert_close(lse, ref.lse, gh.ATOL_LSE, "assembled lse")
+
+
+def test_preact_plus_finalize_equals_fused_head():
+    """world = 1: the two-call head agrees with the fused one to fp32 rounding, odd widths included."""
+    B, d_ext, Hq, D, d_h = 7, 7, 2, 64, 19
+    prob = make_problem(1, 1, B, Hq, Hq, D, [20] * B)
+    ctx = gh.make_ctx(prob, [8], [0], [1], head=(d_ext, 1, d_h))
+    d_in = d_ext + Hq * D
+    hd = {k: torch.from_numpy(v).cuda() for k, v in dict(
+        W1=synth.gauss_f32_tensor(5, synth.STREAM_W1, (d_h, d_in), std=0.05),
+        b1=synth.gauss_f32_tensor(5, synth.STREAM_B1, (d_h,), std=0.05),
+        w2=synth.gauss_f32_tensor(5, synth.STREAM_W2, (d_h,), std=0.05),
+        b2=synth.gauss_f32_tensor(5, synth.STREAM_B2, (1,), std=0.05)).items()}
+    fe = torch.from_numpy(synth.gauss_f32_tensor(5, synth.STREAM_FEAT, (B, d_ext))).cuda()
+    attn = torch.from_numpy(synth.gauss_f32_tensor(6, synth.STREAM_FEAT, (B, Hq, D))).cuda()
+    s1, z1, s2, z2 = (torch.zeros(B, device="cuda") for _ in range(4))
+    f1, f2 = (torch.zeros(B, dtype=torch.uint8, device="cuda") for _ in range(2))
+    pre = torch.zeros((B, d_h), device="cuda")
+    ctx.recall_score(B, fe, attn, hd["W1"], hd["b1"], hd["w2"], hd["b2"], 0.5, None, s1, z1, f1)
+    ctx.recall_preact(B, fe, attn, hd["W1"], d_in, pre)
+    ctx.recall_finalize(B, pre, hd["b1"], hd["w2"], hd["b2"], 0.5, None, s2, z2, f2)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(s2.cpu().numpy(), s1.cpu().numpy(), rtol=0, atol=1e-6)
+    np.testing.assert_allclose(z2.cpu().numpy(), z1.cpu().numpy(), rtol=0, atol=1e-5)
+    x = torch.cat([fe, attn.reshape(B, -1)], dim=1).double()
+    np.testing.assert_allclose(pre.cpu().numpy(), (x @ hd["W1"].double().T).cpu().numpy(), rtol=0, atol=1e-5)
