@@ -101,7 +101,11 @@ typedef struct {
                                  * out/lse must hold the Local pass of the same step, lse must not be
                                  * NULL in oda_full_decode_gated.  The paper's runtime recomputes Full
                                  * from scratch; this variant makes a recalled step cost exactly one
-                                 * Full pass in bytes.  TMA variant only. */
+                                 * Full pass in bytes.  TMA variant only.
+                                 * bit 2: oda_full_decode_gated skips a flagged request whose seq_len is
+                                 * 0 (its rows stay untouched) instead of setting the device status:
+                                 * for a rank of a sequence-sharded pass that holds none of a short
+                                 * request (see oda_merge_partials). */
 } oda_config_t;
 
 /* Lifetime.  oda_create validates and copies the config (host only, no device work).
@@ -178,6 +182,26 @@ oda_status_t oda_recall_finalize(oda_ctx_t* ctx, int32_t batch, const float* pre
                                  const float* w2, const float* b2, float threshold,
                                  const uint8_t* override_flags, float* scores, float* logits,
                                  uint8_t* flags, int32_t* counters, void* stream);
+
+/*
+ * Sequence sharding of the gated Full pass (the paper runs on one GPU; this is how the history of
+ * Eq. 1's S^F splits over ranks that each hold a range of positions).  Every rank runs
+ * oda_full_decode_gated over its own slice (its block table and lengths) and gets, per row,
+ * softmax attention over that slice as (out_r, lse_r); the rows of all ranks are gathered into
+ * parts_out [n_parts][L, batch, q_heads, D] fp32 and parts_lse [n_parts][L, batch, q_heads] fp32
+ * (natural-log lse), and this call combines them for gated layers in [layer_begin, layer_end) and
+ * requests with flags[b] != 0 (all requests if flags == NULL):
+ *   lse = M + ln sum_r e^{lse_r - M},  out = sum_r e^{lse_r - lse} out_r,  parts in index order.
+ * part_tokens [n_parts][batch] i32 (nullable) gives the number of positions each rank holds of each
+ * request: a part with 0 positions, or whose lse is -inf, contributes nothing (its rows are never
+ * read as numbers that matter, so they may be uninitialised); if no part contributes, out = 0 and
+ * lse = -inf.  Other rows of out/lse are not touched.  lse may be NULL.
+ * fp32 contexts only (ODA_ERR_UNSUPPORTED otherwise).  One launch; does not synchronise.
+ */
+oda_status_t oda_merge_partials(oda_ctx_t* ctx, int32_t n_parts, int32_t layer_begin, int32_t layer_end,
+                                int32_t batch, const float* parts_out, const float* parts_lse,
+                                const int32_t* part_tokens, const uint8_t* flags, void* out, float* lse,
+                                void* stream);
 
 /*
  * The paper's own recall head (appendix "Recall-head architecture"; Eq. 2): three

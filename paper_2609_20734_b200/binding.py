@@ -25,7 +25,7 @@ EXPORTS = [
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
-    "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize",
+    "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
 ]
 
 
@@ -98,6 +98,8 @@ def load_library():
         lib.oda_recall_preact.restype = i32
         lib.oda_recall_finalize.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, vp, vp, vp, vp, vp]
         lib.oda_recall_finalize.restype = i32
+        lib.oda_merge_partials.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        lib.oda_merge_partials.restype = i32
         lib.oda_full_decode_gated.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
         lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
@@ -155,6 +157,7 @@ class OdaConfig:
     head_use_attn_out: int = 1
     head_d_hidden: int = 0
     serialize_launches: int = 0   # 1 = no programmatic dependent launch between the kernels of a step
+    allow_empty: int = 0          # 1 = gated passes skip flagged requests of length 0 (sequence-sharded ranks)
     reuse_local: int = 0          # 1 = the gated pass reads only S^F \ S^L and merges with Local (q_full == q_local)
     _keep: list = field(default_factory=list, repr=False)
 
@@ -173,7 +176,7 @@ class OdaConfig:
             arr(self.layer_gated, np.uint8), arr(self.layer_kv_index, np.int32),
             self.kv_layer_stride, self.kv_block_stride, self.kv_token_stride, self.kv_head_stride,
             self.head_d_ext, self.head_use_attn_out, self.head_d_hidden,
-            (1 if self.serialize_launches else 0) | (2 if self.reuse_local else 0))
+            (1 if self.serialize_launches else 0) | (2 if self.reuse_local else 0) | (4 if self.allow_empty else 0))
 
 
 def _ptr(t) -> Optional[int]:
@@ -274,6 +277,12 @@ class OdaContext:
             self._h, batch, _ptr(pre_sum), _ptr(b1), _ptr(w2), _ptr(b2), float(threshold),
             _ptr(override_flags), _ptr(scores), _ptr(logits), _ptr(flags), _ptr(counters),
             _stream() if stream is None else stream), "oda_recall_finalize")
+
+    def merge_partials(self, n_parts, layer_begin, layer_end, batch, parts_out, parts_lse, flags, out, lse=None,
+                       part_tokens=None, stream=None):
+        self._check(self.lib.oda_merge_partials(
+            self._h, n_parts, layer_begin, layer_end, batch, _ptr(parts_out), _ptr(parts_lse), _ptr(part_tokens),
+            _ptr(flags), _ptr(out), _ptr(lse), _stream() if stream is None else stream), "oda_merge_partials")
 
     def full_decode_gated(self, layer_begin, layer_end, batch, q_full, k_cache, v_cache, block_table,
                           seq_lens, flags, out, lse=None, stream=None):

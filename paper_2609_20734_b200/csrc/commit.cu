@@ -56,6 +56,80 @@ select_rows_kernel(const uint4* __restrict__ local, const uint4* __restrict__ fu
     }
 }
 
+// Sequence-sharded Full pass: part r holds softmax attention over rank r's slice of the history
+// as (normalised out_r, lse_r).  The whole-history result is the log-sum-exp combination
+//   lse = M + ln sum_r e^{lse_r - M},  out = sum_r e^{lse_r - lse} out_r,  M = max_r lse_r,
+// parts added in rank order.  A part with part_tokens[r][b] == 0 or lse = -inf (the rank held
+// none of the request) adds nothing.  One warp per (layer, request, query head) row; V floats per lane.
+template <int V>
+__global__ void __launch_bounds__(256)
+merge_partials_kernel(const float* __restrict__ parts_out, const float* __restrict__ parts_lse,
+                      const int32_t* __restrict__ part_tokens, const uint8_t* __restrict__ flags,
+                      const LayerInfo* __restrict__ layers, float* __restrict__ out,
+                      float* __restrict__ lse, int n_parts, int layer_begin, int layer_end, int batch, int q_heads,
+                      int num_layers, int max_batch_rows)
+{
+    griddep_wait();
+    griddep_launch_dependents();
+    constexpr int D = V * 32;
+    const int lane = threadIdx.x & 31;
+    const long long rows = (long long)(layer_end - layer_begin) * batch * q_heads;
+    const long long part_rows = (long long)num_layers * max_batch_rows * q_heads;
+    for (long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < rows;
+         w += ((long long)gridDim.x * blockDim.x) >> 5) {
+        const int h = (int)(w % q_heads);
+        const int b = (int)((w / q_heads) % batch);
+        const int l = layer_begin + (int)(w / ((long long)q_heads * batch));
+        if (!layers[l].gated || (flags && !flags[b])) continue;
+        const long long row = ((long long)l * max_batch_rows + b) * q_heads + h;
+        float m = -INFINITY;
+        unsigned long long have = 0;  // parts that hold some of this request (n_parts <= 64)
+        for (int r = 0; r < n_parts; ++r) {
+            if (part_tokens && part_tokens[r * batch + b] <= 0) continue;
+            const float lr = parts_lse[r * part_rows + row];
+            if (lr == -INFINITY) continue;
+            have |= 1ull << r;
+            m = fmaxf(m, lr);
+        }
+        float acc[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+        float sum = 0.f;
+        if (have) {
+            for (int r = 0; r < n_parts; ++r) {
+                if (!((have >> r) & 1)) continue;
+                const float lr = parts_lse[r * part_rows + row];
+                const float wgt = expf(lr - m);
+                sum += wgt;
+                const float* src = parts_out + (r * part_rows + row) * D + lane * V;
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = fmaf(wgt, src[e], acc[e]);
+            }
+        }
+        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        float* dst = out + row * D + lane * V;
+#pragma unroll
+        for (int e = 0; e < V; ++e) dst[e] = acc[e] * inv;
+        if (lse && lane == 0) lse[row] = sum > 0.f ? m + logf(sum) : -INFINITY;
+    }
+}
+
+cudaError_t launch_merge_partials(const float* parts_out, const float* parts_lse, const int32_t* part_tokens,
+                                  const uint8_t* flags, const LayerInfo* layers, float* out, float* lse, int n_parts, int layer_begin,
+                                  int layer_end, int batch, int q_heads, int head_dim, int num_layers,
+                                  cudaStream_t st, bool pdl)
+{
+    const long long rows = (long long)(layer_end - layer_begin) * batch * q_heads;
+    int grid = (int)((rows + 7) / 8);
+    if (grid > 1184) grid = 1184;
+    if (grid < 1) grid = 1;
+    if (head_dim == 128)
+        return launch_ex(merge_partials_kernel<4>, dim3(grid), dim3(256), 0, st, pdl, parts_out, parts_lse, part_tokens,
+                         flags, layers, out, lse, n_parts, layer_begin, layer_end, batch, q_heads, num_layers, batch);
+    return launch_ex(merge_partials_kernel<2>, dim3(grid), dim3(256), 0, st, pdl, parts_out, parts_lse, part_tokens, flags, layers,
+                     out, lse, n_parts, layer_begin, layer_end, batch, q_heads, num_layers, batch);
+}
+
 cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const uint8_t* mask, void* k_cache,
                                     void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
                                     const LayerInfo* layers, int num_layers, int batch, int num_kv_heads,

@@ -58,6 +58,7 @@ struct oda_ctx {
     int64_t blocks_bound = 1;
     int64_t launches = 0;
     bool use_pdl = true;  // programmatic dependent launch between the kernels of a step
+    bool allow_empty = false;  // gated passes skip requests of length 0 instead of reporting them
     bool reuse_local = false;  // the gated pass reads only S^F \ S^L and merges with the Local result
     std::string err;
 };
@@ -176,6 +177,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     }
     if (!any) return ODA_OK;  // e.g. a Full call over fixed-window layers only
     p.advance_seq_lens = advance;
+    p.allow_empty = c->allow_empty ? 1 : 0;
     if (publish) {
         p.flags_out = publish->flags;
         p.scores_out = publish->scores;
@@ -315,12 +317,13 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         delete c;
         return ODA_ERR_UNSUPPORTED;  // layer stride is not a whole number of blocks
     }
-    if (cfg->options < 0 || cfg->options > 3) {
+    if (cfg->options < 0 || cfg->options > 7) {
         delete c;
         return ODA_ERR_INVALID_ARG;
     }
     c->use_pdl = (cfg->options & 1) == 0;
     c->reuse_local = (cfg->options & 2) != 0;
+    c->allow_empty = (cfg->options & 4) != 0;
     c->variant = cfg->variant == ODA_VARIANT_AUTO ? (tma_ok ? ODA_VARIANT_TMA_MMA : ODA_VARIANT_SIMT) : cfg->variant;
     if (c->reuse_local && c->variant != ODA_VARIANT_TMA_MMA) {
         delete c;
@@ -579,6 +582,29 @@ oda_status_t oda_write_current_kv(oda_ctx_t* c, int32_t batch, const void* k_cur
         f.kv_token_stride, f.kv_head_stride, reinterpret_cast<int32_t*>(c->ws + c->lay.status),
         static_cast<cudaStream_t>(stream), c->use_pdl);
     if (e != cudaSuccess) return cuda_fail(c, e, "commit kernel launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
+oda_status_t oda_merge_partials(oda_ctx_t* c, int32_t n_parts, int32_t lb, int32_t le, int32_t batch,
+                                const float* parts_out, const float* parts_lse, const int32_t* part_tokens,
+                                const uint8_t* flags, void* out, float* lse, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    const oda_config_t& f = c->cfg;
+    if (n_parts < 1 || n_parts > 64) return fail(c, ODA_ERR_INVALID_ARG, "n_parts outside [1, 64]");
+    if (lb < 0 || le > f.num_layers || lb > le) return fail(c, ODA_ERR_INVALID_ARG, "bad layer range");
+    if (batch < 0 || batch > f.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0 || lb == le) return ODA_OK;
+    if (f.out_dtype != 0) return fail(c, ODA_ERR_UNSUPPORTED, "parts are merged in fp32: create the context with out_dtype 0");
+    if (!parts_out || !parts_lse || !out) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(parts_out) || !aligned16(out)) return fail(c, ODA_ERR_INVALID_ARG, "parts_out and out must be 16-byte aligned");
+    cudaError_t e = launch_merge_partials(parts_out, parts_lse, part_tokens, flags,
+                                          reinterpret_cast<const LayerInfo*>(c->ws + c->lay.layers),
+                                          static_cast<float*>(out), lse, n_parts, lb, le, batch, f.num_q_heads,
+                                          f.head_dim, f.num_layers, static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "partial merge launch");
     c->launches += 1;
     return ODA_OK;
 }

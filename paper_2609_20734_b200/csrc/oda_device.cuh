@@ -46,6 +46,7 @@ struct AttnParams {
     float scale_log2e;     // sm_scale * log2(e)
     int32_t cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
     int32_t cls_layers_in_call[kMaxClasses];
+    int32_t allow_empty;   // gated passes: a request with seq_len 0 is skipped silently (a rank that holds none of it)
     int32_t* advance_seq_lens;  // nullable: seq_lens to increment once every CTA has read them
     int32_t* done_counter;      // zero between launches
     // Full pass of a step without a recall head: `flags` are the caller's forced flags, and the
@@ -204,7 +205,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             if (b < B && p.cls_layers_in_call[c] > 0 && (p.mode == 0 || (p.cls_gated[c] && pl.active[b]))) {  // modes 1 and 2 are gated
                 const int t = pl.seq[b];
                 if (t < 1) {
-                    atomicOr(p.status, kStatusBadSeqLen);
+                    if (!(t == 0 && p.allow_empty && p.mode != 0)) atomicOr(p.status, kStatusBadSeqLen);
                 } else {
                     Ranges r = eq1_ranges(p.mode, t, p.cls_window[c], p.cls_sinks[c]);
                     np = r.pg1 - r.pg0;

@@ -39,6 +39,11 @@ cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const 
 cudaError_t launch_select_rows(const void* local, const void* full, const uint8_t* flags, void* out, int batch,
                                size_t row_bytes, cudaStream_t st, bool pdl = false);
 
+cudaError_t launch_merge_partials(const float* parts_out, const float* parts_lse, const int32_t* part_tokens,
+                                  const uint8_t* flags, const LayerInfo* layers, float* out, float* lse, int n_parts, int layer_begin,
+                                  int layer_end, int batch, int q_heads, int head_dim, int num_layers,
+                                  cudaStream_t st, bool pdl = false);
+
 struct HeadParams {
     const float* feat_ext;      // [B, d_ext] or nullptr
     const void* attn_out;       // [B, d_attn] fp32 or bf16, or nullptr

@@ -91,3 +91,43 @@ def tp_step(ctx, shard: HeadShard, batch, q_local, k_cache, v_cache, block_table
                             scores=scores, flags=flags, logits=logits, lse=lse,
                             override_flags=override_flags, counters=counters)
     return flags
+
+
+# ---- sequence sharding of the gated Full pass ------------------------------------------------
+def sequence_shard(rank: int, world: int, seq_len: int, page: int = 16):
+    """Contiguous split of a request's ceil(seq_len / page) pages over the ranks, as even as whole
+    pages allow.  Returns (first page, end page, positions held); short requests leave the last
+    ranks empty."""
+    if world < 1 or not 0 <= rank < world:
+        raise ValueError("rank outside [0, world)")
+    pages = (int(seq_len) + page - 1) // page
+    lo = (rank * pages + world - 1) // world
+    hi = ((rank + 1) * pages + world - 1) // world
+    held = max(0, min(int(seq_len), hi * page) - lo * page)
+    return lo, hi, held
+
+
+def gather_over_ranks(dst, src, group=None):
+    """All-gather of equally shaped tensors into dst[rank] (dst has a leading world axis)."""
+    import torch.distributed as dist
+
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_gather(list(dst.unbind(0)), src, group=group)   # dst[r] are contiguous views
+    else:
+        dst.copy_(src.reshape(dst.shape))
+    return dst
+
+
+def sp_full_step(ctx, world, batch, q_full, k_cache, v_cache, block_table_local, seq_lens_local, part_tokens,
+                 flags, part_out, part_lse, parts_out, parts_lse, out, lse=None, gather=gather_over_ranks):
+    """Gated Full pass of one rank of a sequence-sharded cache, then the exchange and the merge.
+    The context is created with allow_empty = 1; block_table_local / seq_lens_local describe the
+    positions this rank holds; part_tokens [world, batch] i32 holds every rank's counts; part_out /
+    part_lse are this rank's [L, batch, Hq, D] / [L, batch, Hq] results and parts_* their gathered
+    [world, ...] forms.  out / lse receive the whole-history rows of flagged requests."""
+    L = ctx.cfg.num_layers
+    ctx.full_decode_gated(0, L, batch, q_full, k_cache, v_cache, block_table_local, seq_lens_local, flags,
+                          part_out, part_lse)
+    gather(parts_out, part_out)
+    gather(parts_lse, part_lse)
+    ctx.merge_partials(world, 0, L, batch, parts_out, parts_lse, flags, out, lse, part_tokens=part_tokens)

@@ -148,3 +148,68 @@ def test_head_shard_arithmetic():
         tp.head_shard(0, 3, 32, 8, 128)
     with pytest.raises(ValueError):
         tp.head_shard(2, 2, 32, 8, 128)
+
+
+_SP_SEQ = [40, 7, 130, 65, 18]
+
+
+def _sp_worker(rank, world, port, ret):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import oda_oracle as orc
+    from paper_2609_20734_b200 import tensor_parallel as tp
+    from tests.helpers import make_problem
+
+    prob = make_problem(6, 2, len(_SP_SEQ), 4, 2, 16, _SP_SEQ)
+    B, width = len(_SP_SEQ), prob["table"].shape[1]
+    table = np.zeros((B, width), np.int32)
+    held = np.zeros(B, np.int32)
+    for b, t in enumerate(_SP_SEQ):
+        lo, hi, held[b] = tp.sequence_shard(rank, world, t)
+        table[b, :hi - lo] = prob["table"][b, lo:hi]
+    out, lse = orc.attention("full", prob["q"], prob["k"], prob["v"], table, np.maximum(held, 1),
+                             num_kv_heads=2, block_size=16, layout=prob["layout"], layer_window=[16, 16],
+                             layer_sinks=[2, 2], request_mask=(held > 0).astype(np.uint8))
+    out = torch.from_numpy(np.nan_to_num(out))
+    lse = torch.from_numpy(np.where(np.isnan(lse), -np.inf, lse))
+    outs = torch.empty((world,) + tuple(out.shape), dtype=out.dtype)
+    lses = torch.empty((world,) + tuple(lse.shape), dtype=lse.dtype)
+    tp.gather_over_ranks(outs, out)
+    tp.gather_over_ranks(lses, lse)
+    m = lses.max(0).values
+    wgt = torch.exp(lses - m)
+    merged = (wgt[..., None] * outs).sum(0) / wgt.sum(0)[..., None]
+    ret[rank] = (held.copy(), merged.numpy(), (m + torch.log(wgt.sum(0))).numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sequence_sharded_full_two_ranks_gloo():
+    """Ranks hold page ranges of every request; their (out, lse) pairs, gathered and combined by
+    log-sum-exp, are Full attention over the whole history on every rank."""
+    world = 2
+    with mp.Manager() as m:
+        ret = m.dict()
+        mp.spawn(_sp_worker, args=(world, 29615, ret), nprocs=world, join=True)
+        res = dict(ret)
+    from tests.helpers import make_problem, oracle_attention
+
+    prob = make_problem(6, 2, len(_SP_SEQ), 4, 2, 16, _SP_SEQ)
+    whole, whole_lse = oracle_attention(prob, "full", [16, 16], [2, 2])
+    assert (sum(res[r][0] for r in range(world)) == np.array(_SP_SEQ)).all()
+    assert (res[1][0] == 0).any()                    # the 7-token request fits one rank
+    for r in range(world):
+        np.testing.assert_allclose(res[r][1], whole, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(res[r][2], whole_lse, rtol=0, atol=1e-12)
+
+
+def test_sequence_shard_covers_every_position_once():
+    from paper_2609_20734_b200 import tensor_parallel as tp
+
+    for t in (1, 15, 16, 17, 100, 2500):
+        for world in (1, 2, 3, 8):
+            parts = [tp.sequence_shard(r, world, t) for r in range(world)]
+            assert parts[0][0] == 0 and parts[-1][1] == (t + 15) // 16
+            assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
+            assert sum(p[2] for p in parts) == t

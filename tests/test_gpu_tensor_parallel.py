@@ -98,3 +98,53 @@ def test_preact_plus_finalize_equals_fused_head():
     np.testing.assert_allclose(z2.cpu().numpy(), z1.cpu().numpy(), rtol=0, atol=1e-5)
     x = torch.cat([fe, attn.reshape(B, -1)], dim=1).double()
     np.testing.assert_allclose(pre.cpu().numpy(), (x @ hd["W1"].double().T).cpu().numpy(), rtol=0, atol=1e-5)
+
+
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_sequence_sharded_full_pass_matches_oracle(world):
+    """Each 'rank' runs the gated Full pass over its page range of every request (ranks run one
+    after another on this GPU); the merged rows equal the oracle's Full attention over the whole
+    history, short requests that leave ranks empty included."""
+    L, B, Hq, Hkv, D = 3, 6, 8, 2, 128
+    windows, sinks, gated = [64, 32, 64], [4, 0, 4], [1, 0, 1]
+    seq = [100, 900, 5, 2500, 64, 17]
+    prob = make_problem(41, L, B, Hq, Hkv, D, seq)
+    flags_h = np.array([1, 1, 1, 1, 0, 1], np.uint8)
+    want, want_lse = orc.attention("full", prob["q"], prob["k"], prob["v"], prob["table"], prob["seq_lens"],
+                                   num_kv_heads=Hkv, block_size=16, layout=prob["layout"], layer_window=windows,
+                                   layer_sinks=sinks, request_mask=flags_h, nthreads=4)
+    dev = gh.upload(prob)
+    flags = torch.from_numpy(flags_h).cuda()
+    lay = prob["layout"]
+    cfg = dict(num_layers=L, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=B,
+               max_blocks_per_seq=prob["table"].shape[1], layer_window=windows, layer_sinks=sinks,
+               layer_gated=gated, kv_layer_stride=lay.layer_stride, kv_block_stride=lay.block_stride,
+               kv_token_stride=lay.token_stride, kv_head_stride=lay.head_stride, allow_empty=1)
+    from paper_2609_20734_b200 import binding
+    ctx = binding.OdaContext(binding.OdaConfig(**cfg))
+    width = prob["table"].shape[1]
+    parts_out = torch.full((world, L, B, Hq, D), float("nan"), device="cuda")
+    parts_lse = torch.full((world, L, B, Hq), float("nan"), device="cuda")
+    tokens = np.zeros((world, B), np.int32)
+    for r in range(world):
+        table_r = np.zeros((B, width), np.int32)
+        for b, t in enumerate(seq):
+            lo, hi, held = tp.sequence_shard(r, world, t)
+            table_r[b, :hi - lo] = prob["table"][b, lo:hi]
+            tokens[r, b] = held
+        ctx.full_decode_gated(0, L, B, dev["q"], dev["k"], dev["v"], torch.from_numpy(table_r).cuda(),
+                              torch.from_numpy(tokens[r]).cuda(), flags, parts_out[r], parts_lse[r])
+    assert (tokens.sum(0) == np.array(seq)).all() and (world == 1 or (tokens == 0).any())
+    out = torch.full((L, B, Hq, D), 7.0, device="cuda")
+    lse = torch.full((L, B, Hq), 7.0, device="cuda")
+    ctx.merge_partials(world, 0, L, B, parts_out, parts_lse, flags, out, lse, part_tokens=torch.from_numpy(tokens).cuda())
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() == 0
+    o, ls = out.cpu().numpy(), lse.cpu().numpy()
+    for l in range(L):
+        for b in range(B):
+            if gated[l] and flags_h[b]:
+                gh.assert_close(o[l, b], want[l, b], gh.ATOL_OUT, f"layer {l} request {b} out")
+                gh.assert_close(ls[l, b], want_lse[l, b], gh.ATOL_LSE, f"layer {l} request {b} lse")
+            else:
+                assert (o[l, b] == 7.0).all() and (ls[l, b] == 7.0).all()   # untouched
