@@ -49,6 +49,8 @@ def parse():
     ap.add_argument("--reuse-local", action="store_true",
                     help="variant: the gated pass reads only the positions Local did not and merges with the "
                          "Local result (exact here because the synthetic stack uses the same queries for both)")
+    ap.add_argument("--shuffled", type=int, default=-1,
+                    help="1: physical blocks in a seeded random order, 0: in logical order (default: the config's own)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -170,7 +172,8 @@ def reference_arm(args, wl, realised_rate=None):
 def config_dict(wl, args, realised):
     return {"workload": f"{wl.name}: L={wl.L} B={wl.B} Hq={wl.Hq} Hkv={wl.Hkv} D={wl.D} "
                         f"context={int(np.max(wl.seq_lens0))} window={wl.windows[0]} sinks={wl.sinks[0]} block=16 "
-                        f"bf16 KV ~N(0,1), {wl.schedule} flags",
+                        f"bf16 KV ~N(0,1), {wl.schedule} flags, "
+                        f"{'shuffled' if wl.shuffled else 'in-order'} block tables",
             "recall_rate_target": wl.recall_rate, "recall_rate_realised": realised,
             "global_batch": wl.B * args.gpus, "parallelism": f"dp{args.gpus} (requests sharded, no collective)",
             "l2": "flushed between timed steps (256 MiB write, untimed)",
@@ -265,6 +268,8 @@ def main():
         return
 
     ov = {"recall_rate": args.recall_rate}
+    if args.shuffled >= 0:
+        ov["shuffled"] = bool(args.shuffled)
     wl = workloads.make(args.config, **ov)
     if args.sinks is not None:
         wl.sinks = [args.sinks if g else s for g, s in zip(wl.gated, wl.sinks)]
