@@ -219,12 +219,19 @@ oda_status_t oda_merge_partials(oda_ctx_t* ctx, int32_t n_parts, int32_t layer_b
  *   gain_out[d_tower], w[d_tower], bias[1].
  * h_prev, emb, h_local: [batch, d_model] fp32 device.  scratch: device, 256-byte aligned, at least
  * oda_full_head_scratch_bytes(head, batch) bytes, used only during the call.  d_model and d_ff
- * must be multiples of 4 and d_tower of 8 (else ODA_ERR_UNSUPPORTED).  3 + 2 n_blocks launches.
+ * must be multiples of 4 and d_tower of 8 (else ODA_ERR_UNSUPPORTED).
+ * variant 0 or 1: 3 + 2 n_blocks stage launches after one memset, chained by programmatic dependent
+ * launch.  variant 2 (batch <= 4 and stage inputs that fit shared memory, else ODA_ERR_UNSUPPORTED):
+ * one persistent kernel after one 256-byte memset: a cooperative launch of one CTA per SM that
+ * streams all weights through a shared-memory ring and synchronises the stages with bounded grid
+ * barriers (a barrier that times out after ~1 s sets bit 2 of the device status word and the kernel
+ * returns).  It is kept as the measured alternative: on a B200 it is slower than the stage launches
+ * (80 vs 70 us at batch 1).  Both are deterministic; they differ in summation order only.
  */
 typedef struct {
     int32_t d_model, d_tower, d_ff, n_blocks;
     float eps;      /* RMSNorm epsilon (the paper does not print it; 1e-6 is customary) */
-    int32_t pad;
+    int32_t variant; /* 0 = auto (= 1), 1 = one launch per stage, 2 = one persistent kernel (batch <= 4) */
     const float* params;
 } oda_full_head_t;
 int64_t oda_full_head_param_count(int32_t d_model, int32_t d_tower, int32_t d_ff, int32_t n_blocks);

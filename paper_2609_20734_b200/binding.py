@@ -53,7 +53,7 @@ class _Config(ctypes.Structure):
 
 class _FullHead(ctypes.Structure):
     _fields_ = [("d_model", ctypes.c_int32), ("d_tower", ctypes.c_int32), ("d_ff", ctypes.c_int32),
-                ("n_blocks", ctypes.c_int32), ("eps", ctypes.c_float), ("pad", ctypes.c_int32),
+                ("n_blocks", ctypes.c_int32), ("eps", ctypes.c_float), ("variant", ctypes.c_int32),
                 ("params", ctypes.c_void_p)]
 
 
@@ -293,11 +293,11 @@ class OdaContext:
 
     def recall_score_full(self, batch, params, d_tower, d_ff, n_blocks, h_prev, emb, h_local, threshold,
                           override_flags, scores, logits, flags, counters=None, eps=1e-6, scratch=None,
-                          stream=None):
+                          stream=None, variant=0):
         """The paper's full recall head; `params` is the flat fp32 parameter tensor (see oda.h)."""
         import torch
 
-        head = _FullHead(h_prev.shape[1], d_tower, d_ff, n_blocks, eps, 0, _ptr(params))
+        head = _FullHead(h_prev.shape[1], d_tower, d_ff, n_blocks, eps, int(variant), _ptr(params))
         need = self.lib.oda_full_head_scratch_bytes(ctypes.byref(head), batch)
         if scratch is None:
             scratch = torch.empty(need, dtype=torch.uint8, device=h_prev.device)

@@ -651,6 +651,7 @@ oda_status_t oda_recall_score_full(oda_ctx_t* c, int32_t batch, const oda_full_h
         return fail(c, ODA_ERR_UNSUPPORTED, "d_model and d_ff must be multiples of 4, d_tower of 8");
     if (!h->params || !h_prev || !emb || !h_local || !scores || !flags || !scratch)
         return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (h->variant < 0 || h->variant > 2) return fail(c, ODA_ERR_INVALID_ARG, "head variant outside 0..2");
     if (!aligned16(h->params) || !aligned16(h_prev) || !aligned16(emb) || !aligned16(h_local) ||
         (reinterpret_cast<uintptr_t>(scratch) % 256) != 0)
         return fail(c, ODA_ERR_INVALID_ARG, "parameters and inputs must be 16-byte aligned, scratch 256-byte aligned");
@@ -659,8 +660,13 @@ oda_status_t oda_recall_score_full(oda_ctx_t* c, int32_t batch, const oda_full_h
     int launches = 0;
     cudaError_t e = launch_full_head(batch, h->d_model, h->d_tower, h->d_ff, h->n_blocks, h->eps, h->params, h_prev,
                                      emb, h_local, threshold, override_flags, scores, logits, flags, counters,
-                                     scratch, static_cast<cudaStream_t>(stream), c->use_pdl, &launches);
+                                     scratch, static_cast<cudaStream_t>(stream), c->use_pdl, &launches, h->variant,
+                                     c->ws ? reinterpret_cast<int32_t*>(c->ws + c->lay.status) : nullptr);
     c->launches += launches;
+    if (e == cudaErrorNotSupported) {
+        (void)cudaGetLastError();
+        return fail(c, ODA_ERR_UNSUPPORTED, "the fused head needs batch <= 4 and a device that can hold one CTA per SM cooperatively");
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "full recall head launch");
     return ODA_OK;
 }

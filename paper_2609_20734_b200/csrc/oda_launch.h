@@ -27,7 +27,17 @@ cudaError_t launch_full_head(int batch, int d_model, int d_tower, int d_ff, int 
                              const float* params, const float* h_prev, const float* emb, const float* h_local,
                              float threshold, const uint8_t* override_flags, float* scores, float* logits,
                              uint8_t* flags, int32_t* counters, void* scratch, cudaStream_t st, bool pdl,
-                             int* launches);
+                             int* launches, int variant, int32_t* status);
+// the same head as one persistent cooperative kernel (batch <= kFullHeadFusedMaxBatch)
+constexpr int kFullHeadFusedMaxBatch = 4;
+constexpr int kFullHeadFusedSmem = 230400;    // dynamic shared memory of the fused head (stage input + ring + control)
+long long full_head_fused_x_floats(int batch, int d_model, int T, int F);
+int full_head_fused_grid();
+cudaError_t launch_full_head_fused(int grid, int batch, int d_model, int T, int F, int n_blocks, float eps,
+                                   const float* params, const float* h_prev, const float* emb, const float* h_local,
+                                   float threshold, const uint8_t* override_flags, float* scores, float* logits,
+                                   uint8_t* flags, int32_t* counters, float* abc, float* z, float* h, int32_t* sync,
+                                   int32_t* status, cudaStream_t st);
 
 struct LayerInfo;
 cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const uint8_t* mask, void* k_cache,

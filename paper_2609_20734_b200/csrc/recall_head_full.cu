@@ -340,10 +340,28 @@ size_t full_head_scratch_bytes(int d_model, int T, int F, int batch)
 cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks, float eps, const float* params,
                              const float* h_prev, const float* emb, const float* h_local, float threshold,
                              const uint8_t* override_flags, float* scores, float* logits, uint8_t* flags,
-                             int32_t* counters, void* scratch, cudaStream_t st, bool pdl, int* launches)
+                             int32_t* counters, void* scratch, cudaStream_t st, bool pdl, int* launches, int variant,
+                             int32_t* status)
 {
     char* sc = static_cast<char*>(scratch);
     const FullScratch L = full_scratch_layout(d_model, T, F, batch);
+    // variant 2: the whole chain as one persistent kernel (measured slower than the stage launches, so
+    // 0 = auto picks the stage launches; see recall_head_fused.cu)
+    const long long x_floats = full_head_fused_x_floats(batch, d_model, T, F);
+    const int fused_grid = (variant == 2 && batch <= kFullHeadFusedMaxBatch && x_floats * 4 + 1024 + 8 * 4096 <= kFullHeadFusedSmem)
+                               ? full_head_fused_grid() : 0;
+    if (variant == 2 && fused_grid == 0) return cudaErrorNotSupported;
+    if (fused_grid > 0) {
+        cudaError_t fe = cudaMemsetAsync(sc + L.tickets, 0, 256, st);  // arrival counter and abort flag
+        if (fe != cudaSuccess) return fe;
+        fe = launch_full_head_fused(fused_grid, batch, d_model, T, F, n_blocks, eps, params, h_prev, emb, h_local,
+                                    threshold, override_flags, scores, logits, flags, counters,
+                                    reinterpret_cast<float*>(sc + L.abc), reinterpret_cast<float*>(sc + L.z),
+                                    reinterpret_cast<float*>(sc + L.h), reinterpret_cast<int32_t*>(sc + L.tickets),
+                                    status, st);
+        if (fe == cudaSuccess && launches) ++*launches;
+        return fe;
+    }
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
         sms = 148;

@@ -17,11 +17,11 @@
 
 #include "oda_device.cuh"
 #include "launch_ex.cuh"
+#include "mbar.cuh"
 #include "oda_launch.h"
 
 namespace oda {
 
-constexpr int kStatusWaitTimeout = 4;
 
 #ifdef ODA_TIMELINE
 __device__ unsigned long long g_timeline[1024 * 8];
@@ -64,57 +64,7 @@ struct TmaCfg {
     static_assert(kStages <= kMaxStages, "ring deeper than the control block");
 };
 
-// ------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t globaltimer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: gives up after ~2 s, records it in the status word and raises the CTA's abort
-// flag, so a lost completion can never hang the GPU.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 1023u) == 0) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > 2000000000ull) {
-                *abort_flag = 1;
-                atomicOr(status, kStatusWaitTimeout);
-                return false;
-            }
-        }
-    }
-    return true;
-}
-
+// ------------------------------------------------------------------ PTX helpers (mbarriers: mbar.cuh)
 __device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* map, uint32_t bar, int head,
                                               int block, uint64_t policy)
 {
@@ -123,12 +73,6 @@ __device__ __forceinline__ void tma_load_page(uint32_t dst, const CUtensorMap* m
         " [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;"
         ::"r"(dst), "l"(map), "r"(0), "r"(0), "r"(0), "r"(head), "r"(block), "r"(bar), "l"(policy)
         : "memory");
-}
-
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)

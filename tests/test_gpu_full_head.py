@@ -29,8 +29,12 @@ def _ctx():
     return gh.make_ctx(prob, [8], [0], [1])
 
 
-@pytest.mark.parametrize("dm,T,F,nb,B", [(64, 32, 40, 2, 5), (128, 64, 96, 1, 20), (2048, 1024, 2048, 2, 4)])
-def test_full_head_parity(dm, T, F, nb, B):
+@pytest.mark.parametrize("dm,T,F,nb,B,variant", [
+    (64, 32, 40, 2, 5, 0), (128, 64, 96, 1, 20, 0), (2048, 1024, 2048, 2, 4, 1),   # one launch per stage
+    (2048, 1024, 2048, 2, 4, 2), (2048, 1024, 2048, 2, 1, 2),                      # persistent kernel, paper size
+    (64, 32, 40, 2, 3, 2), (128, 64, 96, 0, 1, 2),                                 # fewer rows than CTAs, no blocks
+    (4104, 24, 2052, 1, 2, 2)])                                                    # k longer than a ring slot, ragged
+def test_full_head_parity(dm, T, F, nb, B, variant):
     ctx = _ctx()
     params = _params(3, dm, T, F, nb)
     assert params.size == binding.load_library().oda_full_head_param_count(dm, T, F, nb)
@@ -39,7 +43,7 @@ def test_full_head_parity(dm, T, F, nb, B):
     x = [synth.gauss_f32_tensor(4, i, (B, dm)) for i in range(3)]
     q, s = orc.full_head(params, *x, d_tower=T, d_ff=F, n_blocks=nb)
     srt = np.sort(s)
-    tau = float(0.5 * (srt[B // 2 - 1] + srt[B // 2]))
+    tau = float(0.5 * (srt[B // 2 - 1] + srt[B // 2])) if B > 1 else 0.5
     scores = torch.zeros(B, device="cuda")
     logits = torch.zeros(B, device="cuda")
     flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
@@ -49,7 +53,7 @@ def test_full_head_parity(dm, T, F, nb, B):
     scratch = None
     for _ in range(2):   # twice: tickets and scratch must be reusable
         scratch = ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], xd[2], tau, None, scores, logits, flags,
-                                        counters, scratch=scratch)
+                                        counters, scratch=scratch, variant=variant)
     torch.cuda.synchronize()
     np.testing.assert_allclose(logits.cpu().numpy(), q, rtol=0, atol=1e-4)
     np.testing.assert_allclose(scores.cpu().numpy(), s, rtol=0, atol=2e-5)
@@ -60,7 +64,7 @@ def test_full_head_parity(dm, T, F, nb, B):
     # forced flags: the head still runs
     ov = (np.arange(B) % 2).astype(np.uint8)
     ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], xd[2], tau, torch.from_numpy(ov).cuda(), scores, None,
-                          flags, None, scratch=scratch)
+                          flags, None, scratch=scratch, variant=variant)
     torch.cuda.synchronize()
     np.testing.assert_array_equal(flags.cpu().numpy(), ov)
     np.testing.assert_allclose(scores.cpu().numpy(), s, rtol=0, atol=2e-5)
@@ -79,4 +83,36 @@ def test_full_head_nonfinite_input_selects_full_and_bad_dims_are_refused():
     np.testing.assert_array_equal(flags.cpu().numpy(), [0, 1, 0])   # threshold 2 is never exceeded; NaN forces Full
     with pytest.raises(binding.OdaError) as e:
         ctx.recall_score_full(B, params, 36, F, nb, x[0], x[1], x[2], 0.5, None, scores, None, flags)
+    assert e.value.status == 2
+
+
+def test_fused_head_graph_replay_is_bitwise_stable_and_forced_variant_limits():
+    """The persistent kernel is captured in a CUDA graph (cooperative launch node) and replayed: the
+    same bits every time, equal to the eager call.  Batch > 4 with the fused variant forced is refused."""
+    ctx = _ctx()
+    dm, T, F, nb, B = 2048, 1024, 2048, 2, 2
+    pd = torch.from_numpy(_params(3, dm, T, F, nb)).cuda()
+    xd = [torch.from_numpy(synth.gauss_f32_tensor(4, i, (B, dm))).cuda() for i in range(3)]
+    scores = torch.zeros(B, device="cuda")
+    logits = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    scratch = ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], xd[2], 0.5, None, scores, logits, flags, variant=2)
+    torch.cuda.synchronize()
+    eager = logits.clone()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], xd[2], 0.5, None, scores, logits, flags,
+                                  scratch=scratch, variant=2)
+    for _ in range(3):
+        logits.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(logits, eager)
+    assert ctx.read_device_status() == 0
+    x5 = [torch.zeros((5, dm), device="cuda") for _ in range(3)]
+    with pytest.raises(binding.OdaError) as e:
+        ctx.recall_score_full(5, pd, T, F, nb, x5[0], x5[1], x5[2], 0.5, None, torch.zeros(5, device="cuda"), None,
+                              torch.zeros(5, dtype=torch.uint8, device="cuda"), variant=2)
     assert e.value.status == 2
