@@ -79,7 +79,8 @@ typedef struct {
     /* host arrays [num_layers], copied at create.  Eq. 1: window w >= 1 (includes the
      * current token), sinks s >= 0.  gated: 1 = ODA layer (Local, Full on recall),
      * 0 = fixed-window layer (always Local).  kv_index (nullable => identity): which
-     * layer slice of the cache holds this layer's K/V. */
+     * layer slice of the cache holds this layer's K/V.  A context takes at most four distinct
+     * (window, sinks, gated) combinations over its layers (ODA_ERR_UNSUPPORTED beyond that). */
     const int32_t* layer_window;
     const int32_t* layer_sinks;
     const uint8_t* layer_gated;
