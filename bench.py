@@ -311,7 +311,9 @@ def main():
     nsteps = args.warmup + args.steps
     qs = [workloads.q_device(wl, s) for s in range(nsteps)]
     flags_h = [wl.override_flags(s) for s in range(nsteps)]
-    ovs = [torch.from_numpy(f).cuda() for f in flags_h]
+    head_decides = flags_h[0] is None        # flags come from the recall head (no forced schedule)
+    ovs = None if head_decides else [torch.from_numpy(f).cuda() for f in flags_h]
+    flags_log = torch.zeros((nsteps, B), dtype=torch.uint8, device="cuda")
     feats = [None if wl.feat_host(s) is None else torch.from_numpy(wl.feat_host(s)).cuda() for s in range(nsteps)]
     q_s = torch.empty_like(qs[0])
     ov_s = torch.zeros(B, dtype=torch.uint8, device="cuda")
@@ -326,7 +328,8 @@ def main():
 
     step_args = ctx.step_args(B, q_s, st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, scores,
                               flags, feat_ext=fe_s, head=st.head, threshold=wl.threshold,
-                              override_flags=ov_s, lse=lse, counters=counters, advance_seq_lens=True)
+                              override_flags=None if head_decides else ov_s, lse=lse, counters=counters,
+                              advance_seq_lens=True)
     calib = 0.0
     if not args.no_calibrate:  # set-up, once: per-SM streaming rates measured on two all-flagged Full passes
         ctx.calibration_begin()
@@ -348,7 +351,8 @@ def main():
 
     def set_inputs(s):
         q_s.copy_(qs[s])
-        ov_s.copy_(ovs[s])
+        if ovs is not None:
+            ov_s.copy_(ovs[s])
         if fe_s is not None:
             fe_s.copy_(feats[s])
 
@@ -361,6 +365,7 @@ def main():
             e0.record()
             graph.replay()
             e1.record()
+            flags_log[s].copy_(flags)     # the step's decisions, for the byte count (after the timed region)
             evs.append((e0, e1))
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in evs] if timed else None
@@ -387,6 +392,9 @@ def main():
         t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
+    if head_decides:
+        flags_h = list(flags_log.cpu().numpy())
+        args.no_sweep = True                  # the sweep forces rates; this configuration decides by itself
     realised = float(np.mean([f.mean() for f in flags_h[args.warmup:]]))
     assert ctx.read_device_status() == 0, "device status word set during the timed region"
     assert int(counters[0, 0].item()) == args.warmup + args.steps, "the recall kernel did not run once per step"
@@ -407,6 +415,39 @@ def main():
             "attention_grid": ctx.attention_grid,
             "sm_bandwidth_calibration": {"applied": calib > 0, "slowest_over_fastest_sm": calib},
             "wall_s_timed_region_incl_flush": t_wall}
+
+    # ---- end to end: host buffers through oda_step_host, copies inside the timed region; every rank
+    #      runs it at the same time, the slowest rank's time counts ----
+    e2e = None
+    if not args.no_e2e and not args.kernels_only:
+        q_hs = [q.cpu().pin_memory() for q in qs]
+        ov_hs = [None if head_decides else torch.from_numpy(f).pin_memory() for f in flags_h]
+        fe_hs = [None if f is None else f.cpu().pin_memory() for f in feats]
+        out_h = torch.zeros(shape).pin_memory()
+        sc_h = torch.zeros(B).pin_memory()
+        fl_h = torch.zeros(B, dtype=torch.uint8).pin_memory()
+        st.seq_lens.copy_(seq0)
+        barrier()
+        tot, up, down = 0.0, 0, 0
+        for s in range(nsteps):
+            a = ctx.step_args(B, q_hs[s], st.k_cache, st.v_cache, st.block_table, st.seq_lens, out_h,
+                              sc_h, fl_h, feat_ext=fe_hs[s], head=st.head, threshold=wl.threshold,
+                              override_flags=ov_hs[s], counters=counters, advance_seq_lens=True)
+            flush.fill_(s & 0xFF)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            up, down = ctx.step_host(a)
+            dt = time.perf_counter() - t0
+            if s >= args.warmup:
+                tot += dt
+        if world > 1:
+            t = torch.tensor([tot], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            tot = float(t.item())
+        e2e = {"value": world * B * args.steps / tot, "unit": UNIT, "h2d_bytes_per_step": up,
+               "d2h_bytes_per_step": down, "ms_per_step": tot / args.steps * 1e3,
+               "note": "oda_step_host: pinned host q/flags in, out/scores/flags back, stream "
+                       "sync inside; KV cache, block table and head weights are device-resident state"}
 
     if rank == 0:
         peak, peak_src = peaks()
@@ -440,13 +481,26 @@ def main():
                 torch.cuda.synchronize()
                 if r >= 2:
                     kt[name].append(e0.elapsed_time(e1))
+        # the same two launches back to back without the flush: what the 126 MB L2 keeps of the
+        # previous pass (nothing of a 4 GB Full pass, most of a 137 MB Local pass)
+        kt_warm = {"local": [], "full": []}
+        for name in ("local", "full"):
+            for r in range(reps + 2):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                kgraphs[name].replay()
+                e1.record()
+                torch.cuda.synchronize()
+                if r >= 2:
+                    kt_warm[name].append(e0.elapsed_time(e1))
         lb, fb = wl.algorithmic_bytes(np.asarray(wl.seq_lens0), np.ones(B))
         kernels = {}
         for name, nbytes in (("local", lb), ("full", fb)):
             t = float(np.mean(kt[name])) * 1e-3
             kernels[name] = {"bound": "hbm", "achieved": nbytes / t / 1e9, "peak": peak, "unit": "GB/s",
                              "frac": nbytes / t / 1e9 / peak, "traffic": None,
-                             "algorithmic_bytes": nbytes, "us": t * 1e6, "frac_of_8000_nominal": nbytes / t / 8e12}
+                             "algorithmic_bytes": nbytes, "us": t * 1e6, "frac_of_8000_nominal": nbytes / t / 8e12,
+                             "us_l2_warm": float(np.mean(kt_warm[name])) * 1e3}
         dominant = "full" if realised * kernels["full"]["us"] > kernels["local"]["us"] else "local"
         line["roofline"] = dict(kernels[dominant], kernel=f"splitkv ({dominant} pass)", peak_source=peak_src)
         line["roofline_other"] = dict(kernels["local" if dominant == "full" else "full"],
@@ -490,32 +544,8 @@ def main():
             line["sweep"] = sweep
             line["affine_fit"] = {"slope_ms": float(coef[0]), "intercept_ms": float(coef[1]), "r2": r2}
 
-        # ---- end to end: host buffers through oda_step_host, copies inside the timed region ----
-        if not args.no_e2e:
-            q_hs = [q.cpu().pin_memory() for q in qs]
-            ov_hs = [torch.from_numpy(f).pin_memory() for f in flags_h]
-            fe_hs = [None if f is None else f.cpu().pin_memory() for f in feats]
-            out_h = torch.zeros(shape).pin_memory()
-            sc_h = torch.zeros(B).pin_memory()
-            fl_h = torch.zeros(B, dtype=torch.uint8).pin_memory()
-            st.seq_lens.copy_(seq0)
-            torch.cuda.synchronize()
-            tot, up, down = 0.0, 0, 0
-            for s in range(nsteps):
-                a = ctx.step_args(B, q_hs[s], st.k_cache, st.v_cache, st.block_table, st.seq_lens, out_h,
-                                  sc_h, fl_h, feat_ext=fe_hs[s], head=st.head, threshold=wl.threshold,
-                                  override_flags=ov_hs[s], counters=counters, advance_seq_lens=True)
-                flush.fill_(s & 0xFF)
-                torch.cuda.synchronize()
-                t0 = time.perf_counter()
-                up, down = ctx.step_host(a)
-                dt = time.perf_counter() - t0
-                if s >= args.warmup:
-                    tot += dt
-            line["e2e"] = {"value": world * B * args.steps / tot, "unit": UNIT, "h2d_bytes_per_step": up,
-                           "d2h_bytes_per_step": down, "ms_per_step": tot / args.steps * 1e3,
-                           "note": "oda_step_host: pinned host q/flags in, out/scores/flags back, stream "
-                                   "sync inside; KV cache, block table and head weights are device-resident state"}
+        if e2e is not None:
+            line["e2e"] = e2e
         line["clocks"] = sampler.stop()
 
         # ---- the oracle on the host cores, bounded sample ----
