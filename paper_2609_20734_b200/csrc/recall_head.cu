@@ -48,7 +48,6 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
     __shared__ __align__(16) float s_x[kHeadBT][kHeadKT];
     __shared__ float s_h[kHeadRows][kMaxHeadBatch];
     __shared__ int s_last;
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // the Local output it reads comes from the previous kernel
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rb = blockIdx.x, ks = blockIdx.y, n_rb = gridDim.x, n_ks = gridDim.y;
@@ -69,6 +68,9 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
                 w[c][e] = (j < p.d_hidden && i + e < d_in) ? __ldg(p.W1 + (size_t)j * p.w1_stride + i + e) : 0.f;
         }
     }
+    // the weights above are parameters and are already in flight; the Local output read below comes
+    // from the previous kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int b0 = 0; b0 < p.batch; b0 += kHeadBT) {
         if (b0) __syncthreads();
         // stage x[b0 .. b0+16)[k0 .. k0+512): every load of the tile is in flight together

@@ -119,7 +119,6 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
     __shared__ float s_acc[kFRows][kFBT];
     __shared__ float s_ss[kFRows][kFBT];
     __shared__ int s_last;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ks = blockIdx.y, n_ks = gridDim.y;
@@ -160,6 +159,9 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
         float4 w_cur[kWC], w_nxt[kWC];
         int rb = blockIdx.x;
         if (rb < group_rbs) load_w(w_cur, rb);
+        // weights are parameters: the first block's loads are in flight before this kernel waits for
+        // the stage that produces its input
+        if (b0 == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (b0) __syncthreads();
         {   // stage x * gain; every load of the tile is in flight together; the sum of squares of
             // the raw x is accumulated on the way
@@ -380,9 +382,9 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
         const int n_ks = ceil_div(p.K, kt);
         const int groups = p.stage == kStageTower ? 3 : 1;
         const int group_rbs = p.stage == kStageTower ? ceil_div(T, kFRows) : p.row_blocks;
-        // small batches: about one CTA per SM in total, each walking several row blocks; large
-        // batches (narrow tiles, many k slices): one row block per CTA
-        int gx = batch <= 4 ? sms / (n_ks * groups) : group_rbs;
+        // about one CTA per SM in total for small batches and two for large ones (narrow tiles, two
+        // CTAs fit an SM), each staging its x tile once and walking several row blocks
+        int gx = (batch <= 4 ? sms : 2 * sms) / (n_ks * groups);
         gx = std::max(1, std::min(gx, group_rbs));
         const dim3 grid(gx, n_ks, groups);
         cudaError_t le = batch <= 4 ? launch_ex(full_head_stage_kernel<4, 2048>, grid, dim3(kFThreads), 0, st, dep, p)
