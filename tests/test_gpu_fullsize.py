@@ -165,3 +165,83 @@ def test_longest_paper_context_one_layer():
     check_units(wl, st, 0, seq, out0, lse0, fl0, [(0, 0, 0), (0, 0, 7)])
     assert (lse1 >= lse0 - 1e-4).all()
     assert ctx.read_device_status() == 0
+
+
+def test_batched_full_size_offsets_beyond_32_bits():
+    """Configuration 3 at its full size: 32 layers, batch 16, lengths uniform in [8192, 65536],
+    shuffled block tables, 38 G bf16 elements per cache tensor (77 GB in all), so page addresses
+    need 64-bit arithmetic everywhere.  One graph-replayed step with a mixed gate pattern; sampled
+    units across the whole address range against the oracle."""
+    free, _ = torch.cuda.mem_get_info()
+    wl = workloads.make("batched", steps=2)
+    need = 2 * wl.phys_layers * int(wl.blocks_needed.sum()) * wl.Hkv * 16 * wl.D * 2
+    if free < need + (6 << 30):
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of device memory")
+    st = workloads.materialize(wl)
+    assert st.k_cache.numel() > 2**32
+    ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks))
+    seq = np.asarray(wl.seq_lens0)
+    ov = (np.arange(wl.B) % 3 == 0).astype(np.uint8)
+    out, lse, scores, flags, _ = run_graph_step(wl, st, ctx, 0, ov)
+    np.testing.assert_array_equal(flags, ov)
+    longest, shortest = int(np.argmax(seq)), int(np.argmin(seq))
+    # units whose pages lie in the first, a middle and the last layer slice; flagged and not
+    units = [(0, 0, 0), (31, 15, 7), (31, longest, 3), (16, shortest, 5), (30, 3, 1), (17, 4, 6), (31, 1, 0)]
+    check_units(wl, st, 0, seq, out, lse, flags, units)
+    assert np.isfinite(out).all()
+    assert ctx.read_device_status() == 0
+    del st, ctx
+    torch.cuda.empty_cache()
+
+
+def _fits(wl, slack=6 << 30):
+    free, _ = torch.cuda.mem_get_info()
+    need = 2 * wl.phys_layers * int(wl.blocks_needed.sum()) * wl.Hkv * 16 * wl.D * 2
+    return free >= need + slack, need
+
+
+def test_70b_full_size_eighty_layers():
+    """Configuration 4 at its full shape: 80 layers, 64q/8kv (G = 8), batch 4, context 131072,
+    window 2048 + 4 sinks; the 80 layers read 16 physical cache slices (the whole cache would be
+    160 GiB).  One request recalls: only its pages may be read by the gated pass."""
+    wl = workloads.make("70b", steps=2)
+    ok, need = _fits(wl)
+    if not ok:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of device memory")
+    st = workloads.materialize(wl)
+    ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks))
+    seq = np.asarray(wl.seq_lens0)
+    ov = np.array([0, 0, 1, 0], np.uint8)
+    out, lse, _, flags, _ = run_graph_step(wl, st, ctx, 0, ov)
+    np.testing.assert_array_equal(flags, ov)
+    check_units(wl, st, 0, seq, out, lse, flags, [(79, 2, 7), (0, 2, 0), (40, 0, 3), (79, 3, 1), (17, 1, 5)])
+    assert np.isfinite(out).all()
+    assert ctx.read_device_status() == 0
+    del st, ctx
+    torch.cuda.empty_cache()
+
+
+def test_hybrid_full_size_forty_eight_layers():
+    """Configuration 5 at its full shape: 48 layers (36 fixed-window 512 without sinks on 3 shared
+    slices, 12 gated 1024 + 4 sinks with a slice each), batch 4, context 262144."""
+    wl = workloads.make("hybrid", steps=2)
+    ok, need = _fits(wl)
+    if not ok:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of device memory")
+    st = workloads.materialize(wl)
+    ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks))
+    seq = np.asarray(wl.seq_lens0)
+    # the flags come from this configuration's head; the threshold is set between its scores
+    _, _, sc, _, _ = run_graph_step(wl, st, ctx, 0, np.zeros(wl.B, np.uint8))
+    srt = np.sort(sc)
+    wl.threshold = float(0.5 * (srt[2] + srt[3]))          # one of the four requests recalls
+    assert srt[3] - wl.threshold > 2 * gh.FLAG_BAND and wl.threshold - srt[2] > 2 * gh.FLAG_BAND
+    out, lse, scores, flags, _ = run_graph_step(wl, st, ctx, 0, None)
+    assert flags.sum() == 1
+    b1 = int(np.argmax(flags))
+    b0 = (b1 + 1) % wl.B
+    check_units(wl, st, 0, seq, out, lse, flags, [(47, b1, 7), (3, b1, 0), (47, b0, 2), (46, b1, 4), (0, b0, 6)])
+    assert np.isfinite(out).all()
+    assert ctx.read_device_status() == 0
+    del st, ctx
+    torch.cuda.empty_cache()
