@@ -35,6 +35,12 @@
  * Algorithm 1, line 8 (commit of the selected candidate) is oda_oracle_write_current_kv +
  * oda_oracle_select_rows, composed into a step by step_with_commit() of the wrapper.
  *
+ * The paper's own recall head (appendix "Recall-head architecture", Eq. 2) is
+ * oda_oracle_full_head: three RMSNorm -> Linear -> SiLU towers, the 9-way
+ * interaction vector, the fusion projection, pre-norm residual SwiGLU blocks and a
+ * normalised scalar output, in the paper's order; its parameter count is pinned to
+ * the 28,325,889 the paper states.
+ *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py
  * (brute force over literal 1-based sets in extended precision, an independent
  * masked-attention library routine, closed forms, set identities quoted from
