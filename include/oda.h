@@ -227,7 +227,7 @@ oda_status_t oda_merge_partials(oda_ctx_t* ctx, int32_t n_parts, int32_t layer_b
  * streams all weights through a shared-memory ring and synchronises the stages with bounded grid
  * barriers (a barrier that times out after ~1 s sets bit 2 of the device status word and the kernel
  * returns).  It is kept as the measured alternative: on a B200 it is slower than the stage launches
- * (80 vs 61 us at batch 1).  Both are deterministic; they differ in summation order only.
+ * (80 vs 59 us at batch 1).  Both are deterministic; they differ in summation order only.
  */
 typedef struct {
     int32_t d_model, d_tower, d_ff, n_blocks;

@@ -378,17 +378,21 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
     p.ssq = reinterpret_cast<float*>(sc + L.ssq);
     p.rb_tickets = reinterpret_cast<int32_t*>(sc + L.tickets);
     auto launch = [&](bool dep) {
-        const int kt = batch <= 4 ? 2048 : 512;
+        // small batches: a 2048-wide k tile (one CTA per SM) where that divides k (towers, down: no
+        // split over k), else a 1024-wide one (gate+up fits it whole; the fusion's k = 9 x 1024 splits
+        // evenly): two CTAs per SM.  Measured: 2048 everywhere 61 us, 1024 everywhere 68 us, mixed 59 us.
+        const int kt = batch <= 4 ? ((p.K <= 1024 || p.K % 2048 != 0) ? 1024 : 2048) : 512;
         const int n_ks = ceil_div(p.K, kt);
         const int groups = p.stage == kStageTower ? 3 : 1;
         const int group_rbs = p.stage == kStageTower ? ceil_div(T, kFRows) : p.row_blocks;
         // about one CTA per SM in total for small batches and two for large ones (narrow tiles, two
         // CTAs fit an SM), each staging its x tile once and walking several row blocks
-        int gx = (batch <= 4 ? sms : 2 * sms) / (n_ks * groups);
+        int gx = (kt >= 2048 ? sms : 2 * sms) / (n_ks * groups);
         gx = std::max(1, std::min(gx, group_rbs));
         const dim3 grid(gx, n_ks, groups);
-        cudaError_t le = batch <= 4 ? launch_ex(full_head_stage_kernel<4, 2048>, grid, dim3(kFThreads), 0, st, dep, p)
-                                    : launch_ex(full_head_stage_kernel<16, 512>, grid, dim3(kFThreads), 0, st, dep, p);
+        cudaError_t le = kt == 2048 ? launch_ex(full_head_stage_kernel<4, 2048>, grid, dim3(kFThreads), 0, st, dep, p)
+                         : kt == 1024 ? launch_ex(full_head_stage_kernel<4, 1024>, grid, dim3(kFThreads), 0, st, dep, p)
+                                      : launch_ex(full_head_stage_kernel<16, 512>, grid, dim3(kFThreads), 0, st, dep, p);
         if (le == cudaSuccess && launches) ++*launches;
         return le;
     };
