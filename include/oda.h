@@ -302,6 +302,15 @@ typedef struct {
     const void *hidden_local, *hidden_full;
     void* hidden_out;
     int64_t hidden_row_bytes;
+    /* Optional: decide with the paper's own recall head (see oda_recall_score_full) instead of the
+     * two-layer one.  full_head (HOST pointer) non-NULL => head_h_prev, head_emb, head_h_local
+     * ([B, d_model] fp32: h_{t-1}, E(x_t) and the Local branch's h_t^L, which the caller's backbone
+     * produces) and head_scratch (>= oda_full_head_scratch_bytes) are required; W1, b1, w2, b2 and
+     * feat_ext are ignored; override_flags still only replaces the decision.  oda_step only. */
+    const oda_full_head_t* full_head;
+    const float *head_h_prev, *head_emb, *head_h_local;
+    void* head_scratch;
+    size_t head_scratch_bytes;
 } oda_step_args_t;
 
 /* One whole step (Algorithm 1, lines 1-7, and line 8 when the commit fields are given): Local on

@@ -73,6 +73,9 @@ class _StepArgs(ctypes.Structure):
         ("k_cur_full", ctypes.c_void_p), ("v_cur_full", ctypes.c_void_p),
         ("hidden_local", ctypes.c_void_p), ("hidden_full", ctypes.c_void_p), ("hidden_out", ctypes.c_void_p),
         ("hidden_row_bytes", ctypes.c_int64),
+        ("full_head", ctypes.c_void_p), ("head_h_prev", ctypes.c_void_p), ("head_emb", ctypes.c_void_p),
+        ("head_h_local", ctypes.c_void_p), ("head_scratch", ctypes.c_void_p),
+        ("head_scratch_bytes", ctypes.c_size_t),
     ]
 
 
@@ -307,6 +310,14 @@ class OdaContext:
             scratch.numel(), _stream() if stream is None else stream), "oda_recall_score_full")
         return scratch
 
+    def full_head_scratch(self, batch, d_model, d_tower, d_ff, n_blocks, device="cuda"):
+        """A scratch tensor large enough for the paper's head at this batch."""
+        import torch
+
+        head = _FullHead(d_model, d_tower, d_ff, n_blocks, 1e-6, 0, None)
+        return torch.empty(self.lib.oda_full_head_scratch_bytes(ctypes.byref(head), batch), dtype=torch.uint8,
+                           device=device)
+
     def write_current_kv(self, batch, k_cur, v_cur, mask, k_cache, v_cache, block_table, seq_lens, stream=None):
         self._check(self.lib.oda_write_current_kv(
             self._h, batch, _ptr(k_cur), _ptr(v_cur), _ptr(mask), _ptr(k_cache), _ptr(v_cache),
@@ -322,16 +333,29 @@ class OdaContext:
                   q_full=None, feat_ext=None, head=None, threshold=0.5, override_flags=None, lse=None,
                   logits=None, counters=None, advance_seq_lens=False, k_cur_local=None, v_cur_local=None,
                   k_cur_full=None, v_cur_full=None, hidden_local=None, hidden_full=None,
-                  hidden_out=None) -> _StepArgs:
+                  hidden_out=None, full_head=None) -> _StepArgs:
+        """full_head: dict(params, d_tower, d_ff, n_blocks, h_prev, emb, h_local, scratch[, eps, variant])
+        to decide with the paper's own recall head."""
         h = head or {}
         row_bytes = 0 if hidden_out is None else hidden_out[0].numel() * hidden_out.element_size()
-        return _StepArgs(
+        fh = (None,) * 6
+        keep = None
+        if full_head is not None:
+            keep = _FullHead(full_head["h_prev"].shape[1], full_head["d_tower"], full_head["d_ff"],
+                             full_head["n_blocks"], full_head.get("eps", 1e-6), int(full_head.get("variant", 0)),
+                             _ptr(full_head["params"]))
+            fh = (ctypes.addressof(keep), _ptr(full_head["h_prev"]), _ptr(full_head["emb"]),
+                  _ptr(full_head["h_local"]), _ptr(full_head["scratch"]), full_head["scratch"].numel())
+        args = _StepArgs(
             batch, 1 if advance_seq_lens else 0, _ptr(q_local), _ptr(q_full), _ptr(k_cache),
             _ptr(v_cache), _ptr(block_table), _ptr(seq_lens), _ptr(feat_ext), _ptr(h.get("W1")),
             _ptr(h.get("b1")), _ptr(h.get("w2")), _ptr(h.get("b2")), float(threshold), 0,
             _ptr(override_flags), _ptr(out), _ptr(lse), _ptr(scores), _ptr(logits), _ptr(flags),
             _ptr(counters), _ptr(k_cur_local), _ptr(v_cur_local), _ptr(k_cur_full), _ptr(v_cur_full),
-            _ptr(hidden_local), _ptr(hidden_full), _ptr(hidden_out), row_bytes)
+            _ptr(hidden_local), _ptr(hidden_full), _ptr(hidden_out), row_bytes, fh[0], fh[1], fh[2], fh[3],
+            fh[4], fh[5] or 0)
+        args._keep = keep     # the head descriptor must outlive the call
+        return args
 
     def step(self, args: _StepArgs, stream=None):
         self._check(self.lib.oda_step(self._h, ctypes.byref(args), _stream() if stream is None else stream),

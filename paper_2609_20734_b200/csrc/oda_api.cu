@@ -680,7 +680,8 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
                                      a->seq_lens, a->out);
     if (s != ODA_OK || B == 0) return s;
     if (!a->scores || !a->flags) return fail(c, ODA_ERR_INVALID_ARG, "scores or flags is null");
-    if (f.head_d_hidden == 0 && !a->override_flags)
+    const bool paper_head = a->full_head != nullptr;
+    if (f.head_d_hidden == 0 && !paper_head && !a->override_flags)
         return fail(c, ODA_ERR_INVALID_ARG, "no head configured and no override_flags given");
     const void* qf = a->q_full ? a->q_full : a->q_local;
     if (!aligned16(qf)) return fail(c, ODA_ERR_INVALID_ARG, "q_full must be 16-byte aligned");
@@ -704,9 +705,14 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
         attn_last = static_cast<const char*>(a->out) + (size_t)c->last_gated * B * f.num_q_heads * f.head_dim * out_elem(c);
     // Without a head the decision is the caller's forced flags: the Full kernel reads them
     // directly and publishes them, which saves the decision kernel's launch.
-    const bool fused_decision = f.head_d_hidden == 0 && c->last_gated >= 0;
+    const bool fused_decision = !paper_head && f.head_d_hidden == 0 && c->last_gated >= 0;
     const uint8_t* decided = fused_decision ? a->override_flags : a->flags;  // valid once the head (if any) has run
-    if (!fused_decision) {
+    if (paper_head) {
+        s = oda_recall_score_full(c, B, a->full_head, a->head_h_prev, a->head_emb, a->head_h_local, a->threshold,
+                                  a->override_flags, a->scores, a->logits, a->flags, a->counters, a->head_scratch,
+                                  a->head_scratch_bytes, stream);
+        if (s != ODA_OK) return s;
+    } else if (!fused_decision) {
         s = oda_recall_score(c, B, a->feat_ext, attn_last, a->W1, a->b1, a->w2, a->b2, a->threshold,
                              a->override_flags, a->scores, a->logits, a->flags, a->counters, stream);
         if (s != ODA_OK) return s;
@@ -748,8 +754,8 @@ oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream,
     if (d2h_bytes) *d2h_bytes = 0;
     if (B == 0) return ODA_OK;
     if (!a->q_local || !a->out || !a->scores || !a->flags) return fail(c, ODA_ERR_INVALID_ARG, "null host pointer");
-    if (a->k_cur_local || a->v_cur_local || a->k_cur_full || a->v_cur_full || a->hidden_out)
-        return fail(c, ODA_ERR_INVALID_ARG, "the commit fields take device pointers: use oda_step");
+    if (a->k_cur_local || a->v_cur_local || a->k_cur_full || a->v_cur_full || a->hidden_out || a->full_head)
+        return fail(c, ODA_ERR_INVALID_ARG, "the commit and full-head fields take device pointers: use oda_step");
     if (f.head_d_ext > 0 && f.head_d_hidden > 0 && !a->feat_ext) return fail(c, ODA_ERR_INVALID_ARG, "feat_ext is null");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t rows = (size_t)f.num_layers * B * f.num_q_heads;

@@ -116,3 +116,57 @@ def test_fused_head_graph_replay_is_bitwise_stable_and_forced_variant_limits():
         ctx.recall_score_full(5, pd, T, F, nb, x5[0], x5[1], x5[2], 0.5, None, torch.zeros(5, device="cuda"), None,
                               torch.zeros(5, dtype=torch.uint8, device="cuda"), variant=2)
     assert e.value.status == 2
+
+
+def test_step_decides_with_the_papers_head():
+    """oda_step with the paper's head in place of the two-layer one: Local pass, the head on the
+    caller's hidden states, gated Full pass for the requests it flags -- against the oracle's head
+    feeding the oracle's step, eager and as one CUDA graph."""
+    L, B, Hq, Hkv, D = 3, 4, 8, 2, 128
+    windows, sinks, gated = [64, 32, 64], [4, 0, 4], [1, 0, 1]
+    prob = make_problem(77, L, B, Hq, Hkv, D, [100, 900, 33, 2500])
+    dm, T, F, nb = 128, 64, 96, 2
+    params = _params(8, dm, T, F, nb)
+    x = [synth.gauss_f32_tensor(9, i, (B, dm)) for i in range(3)]
+    q_ref, s_ref = orc.full_head(params, *x, d_tower=T, d_ff=F, n_blocks=nb)
+    srt = np.sort(s_ref)
+    tau = float(0.5 * (srt[1] + srt[2]))
+    assert srt[2] - tau > 2 * gh.FLAG_BAND and tau - srt[1] > 2 * gh.FLAG_BAND
+    want_flags = orc.flags(q_ref, s_ref, tau)
+    assert want_flags.sum() == 2
+    ref = orc.step(prob["q"], None, prob["k"], prob["v"], prob["table"], prob["seq_lens"], num_kv_heads=Hkv,
+                   block_size=16, layout=prob["layout"], layer_window=windows, layer_sinks=sinks,
+                   layer_gated=gated, override_flags=want_flags, nthreads=4)
+    ctx = gh.make_ctx(prob, windows, sinks, gated)          # no two-layer head configured
+    dev = gh.upload(prob)
+    out, lse = gh.new_out(prob)
+    scores = torch.zeros(B, device="cuda")
+    logits = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    fh = dict(params=torch.from_numpy(params).cuda(), d_tower=T, d_ff=F, n_blocks=nb,
+              h_prev=torch.from_numpy(x[0]).cuda(), emb=torch.from_numpy(x[1]).cuda(),
+              h_local=torch.from_numpy(x[2]).cuda(), scratch=ctx.full_head_scratch(B, dm, T, F, nb))
+    args = ctx.step_args(B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out, scores, flags,
+                         threshold=tau, lse=lse, logits=logits, full_head=fh)
+    ctx.step(args)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(flags.cpu().numpy(), want_flags)
+    np.testing.assert_allclose(scores.cpu().numpy(), s_ref, rtol=0, atol=2e-5)
+    np.testing.assert_allclose(logits.cpu().numpy(), q_ref, rtol=0, atol=1e-4)
+    gh.assert_close(out.cpu().numpy(), ref.out, gh.ATOL_OUT, "out")
+    gh.assert_close(lse.cpu().numpy(), ref.lse, gh.ATOL_LSE, "lse")
+    eager = out.clone()
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            ctx.step(args, stream=s.cuda_stream)
+    out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager)
+    assert ctx.read_device_status() == 0
+    # the host-buffer form has no place for the head's device inputs
+    with pytest.raises(binding.OdaError):
+        ctx.step_host(args)
