@@ -27,7 +27,11 @@ namespace oda {
 __device__ unsigned long long g_timeline[1024 * 8];
 #define ODA_TL(slot) do { if ((threadIdx.x & 31) == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_timeline[blockIdx.x * 8 + (slot)] = t_; } } while (0)
 extern "C" int oda_debug_timeline(unsigned long long* host, int n) { return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n); }
+__device__ long long g_tl_acc[1024 * 8];
+extern "C" int oda_debug_acc(long long* host, int n) { return (int)cudaMemcpyFromSymbol(host, g_tl_acc, sizeof(long long) * n); }
+#define ODA_CLK(v) const long long v = clock64()
 #else
+#define ODA_CLK(v) do { } while (0)
 #define ODA_TL(slot) do { } while (0)
 #endif
 
@@ -46,6 +50,10 @@ struct Ctl {  // barriers and small hand-off slots, after the Plan in shared mem
     int32_t abort;
     int32_t pad;
     EpiMeta meta;
+    // the producer decodes every item anyway (it needs the pages); it hands the descriptor to the
+    // consumers with the item's first tile, so that they do not decode it again on their critical path
+    Item items[kMaxStages];
+    int32_t item_take[kMaxStages];  // axis pages the item covers
 };
 
 template <int D>
@@ -143,6 +151,8 @@ struct PageRun {
     const __nv_bfloat16* q;  // q rows of the item, copied with the first tile of the item
     int pg, n;               // first logical page, pages in the run (1..32)
     bool first;              // first run of its item
+    Item item;               // the item (meaningful in its first run)
+    int take;
 };
 
 template <int D, int G>
@@ -207,6 +217,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             r.pg = pg;
             r.n = min(32, end - pg);
             r.first = item_first;
+            if (item_first) { r.item = it; r.take = take; }
             item_first = false;
             blk = lane < r.n ? __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + pg + lane) : 0;
             pg += r.n;
@@ -239,8 +250,13 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { dead = true; break; }
                 const bool with_q = cur.first && t0 == 0;
                 if (cnt == 0) ODA_TL(3);
-                if (lane == 0)
+                if (lane == 0) {
+                    if (with_q) {  // visible to the consumers once the stage's barrier completes
+                        ctl.items[s] = cur.item;
+                        ctl.item_take[s] = cur.take;
+                    }
                     mbar_expect_tx(full0 + 8 * s, (uint32_t)np * 2 * C::kPageBytes + (with_q ? kQBytes : 0u));
+                }
                 __syncwarp();
                 const int blk = __shfl_sync(0xffffffffu, blk_cur, t0 + (lane & 3));
                 if (lane < np) {
@@ -449,15 +465,24 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         int x, x_end;
         span_range(plan, span, x, x_end);
         span_pages = x_end - x;
+#ifdef ODA_TIMELINE
+        long long a_dec = 0, a_first = 0, a_tiles = 0, a_wait = 0, a_merge = 0, a_items = 0;
+#endif
         while (x < x_end && !aborted) {
             Item it;
-            x += decode_item(p, plan, span, x, x_end, it);
-            // Q^T fragments come with the item's first tile; heads >= G stay zero
+            ODA_CLK(c0);
+            ODA_CLK(c1);
+            // the item's descriptor and its Q^T fragments come with the item's first tile; heads >= G stay zero
             uint32_t qa[D / 16][2];
             {
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
+                it = ctl.items[s];
+                x += ctl.item_take[s];
                 if (cnt == 0 && warp == 0) ODA_TL(4);
+#ifdef ODA_TIMELINE
+                { const long long c2 = clock64(); a_dec += c1 - c0; a_first += c2 - c1; a_items += 1; }
+#endif
                 if (cnt == 0 && p.sm_stats) t_first = globaltimer_ns();
                 const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
 #pragma unroll
@@ -472,10 +497,15 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;  // heads qc and qc+1
 
             TileWalk tw;
+            ODA_CLK(c3);
             for (tw.start(it); !tw.done(); tw.next(it)) {
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 ++cnt;
+                ODA_CLK(c4);
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
+#ifdef ODA_TIMELINE
+                a_wait += clock64() - c4;
+#endif
                 if (warp < tw.npages) {
                     const int pos0 = (tw.pg + warp) * kPage;
                     const int vlo = tw.seg ? it.win_lo : 0, vhi = tw.seg ? it.win_hi : it.sink_hi;
@@ -552,6 +582,10 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             }
             if (aborted || *abort_flag) { aborted = true; break; }
             if (warp == 0) ODA_TL(5);
+            ODA_CLK(c5);
+#ifdef ODA_TIMELINE
+            a_tiles += c5 - c3;
+#endif
 
             // ---- fold warps 1..3 into warp 0 through shared memory (all use the same fragment
             //      layout), then leave the item to the epilogue warp ----
@@ -611,7 +645,16 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (lane == 0) mbar_arrive(efull);
             }
             ++ecnt;
+#ifdef ODA_TIMELINE
+            a_merge += clock64() - c5;
+#endif
         }
+#ifdef ODA_TIMELINE
+        if (tid == 0) {
+            long long* a = g_tl_acc + blockIdx.x * 8;
+            a[0] = a_dec; a[1] = a_first; a[2] = a_tiles; a[3] = a_wait; a[4] = a_merge; a[5] = a_items;
+        }
+#endif
     }
     // calibration run: how long this SM took to stream how many pages
     if (p.sm_stats && tid == 0 && !aborted && plan.nseg == (int)gridDim.x) {
