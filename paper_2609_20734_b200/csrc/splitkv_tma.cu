@@ -497,8 +497,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;  // heads qc and qc+1
 
             TileWalk tw;
+            uint32_t s_last = 0;  // the stage of the item's last tile: kept until the fold below is done with it
             ODA_CLK(c3);
-            for (tw.start(it); !tw.done(); tw.next(it)) {
+            for (tw.start(it); !tw.done();) {
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 ++cnt;
                 ODA_CLK(c4);
@@ -578,7 +579,11 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * s);
+                tw.next(it);
+                if (tw.done())
+                    s_last = s;
+                else if (lane == 0)
+                    mbar_arrive(empty0 + 8 * s);
             }
             if (aborted || *abort_flag) { aborted = true; break; }
             if (warp == 0) ODA_TL(5);
@@ -587,62 +592,86 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             a_tiles += c5 - c3;
 #endif
 
-            // ---- fold warps 1..3 into warp 0 through shared memory (all use the same fragment
-            //      layout), then leave the item to the epilogue warp ----
+            // ---- fold the four warps' states and leave the item to the epilogue warp.  Every warp
+            //      parks its fragment in its own page slot of the item's last stage (that data is
+            //      dead: a warp only ever reads its own page), then each warp finishes a quarter of
+            //      the rows from all four fragments, in warp order, into the hand-off buffer. ----
 #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {
                 lA += __shfl_xor_sync(0xffffffffu, lA, off);
                 lB += __shfl_xor_sync(0xffffffffu, lB, off);
             }
-            // the hand-off buffer doubles as the merge buffer: wait until the epilogue warp has
-            // taken the previous item out of it
-            if (!mbar_wait(efree, (ecnt & 1) ^ 1, abort_flag, p.status)) { aborted = true; break; }
-#pragma unroll 1
-            for (int src_warp = 1; src_warp < C::kConsumerWarps; ++src_warp) {
-                if (warp == src_warp) {
-#pragma unroll
-                    for (int n = 0; n < D / 16; ++n) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) mbuf[(4 * n + e) * 32 + lane] = o[n][e];
-                    }
-                    reinterpret_cast<float4*>(mlbuf)[lane] = make_float4(mA, lA, mB, lB);
-                }
-                consumer_sync();
-                if (warp == 0) {
-                    const float4 ml = reinterpret_cast<const float4*>(mlbuf)[lane];
-                    const float MA = fmaxf(mA, ml.x), MB = fmaxf(mB, ml.z);
-                    const float muA = (MA == -INFINITY) ? 0.f : MA, muB = (MB == -INFINITY) ? 0.f : MB;
-                    const float saA = ex2(mA - muA), sbA = ex2(ml.x - muA);
-                    const float saB = ex2(mB - muB), sbB = ex2(ml.z - muB);
-#pragma unroll
-                    for (int n = 0; n < D / 16; ++n) {
-                        o[n][0] = o[n][0] * saA + mbuf[(4 * n + 0) * 32 + lane] * sbA;
-                        o[n][1] = o[n][1] * saB + mbuf[(4 * n + 1) * 32 + lane] * sbB;
-                        o[n][2] = o[n][2] * saA + mbuf[(4 * n + 2) * 32 + lane] * sbA;
-                        o[n][3] = o[n][3] * saB + mbuf[(4 * n + 3) * 32 + lane] * sbB;
-                    }
-                    lA = lA * saA + ml.y * sbA;
-                    lB = lB * saB + ml.w * sbB;
-                    mA = MA;
-                    mB = MB;
-                }
-                consumer_sync();
-            }
-            if (warp == 0) {
+            {
+                uint8_t* stage = ring + s_last * C::kStageBytes;
+                float* fo = reinterpret_cast<float*>(stage + warp * C::kPageBytes);
+                float4* fml = reinterpret_cast<float4*>(stage + (C::kTilePages + warp) * C::kPageBytes);
 #pragma unroll
                 for (int n = 0; n < D / 16; ++n) {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) mbuf[(4 * n + e) * 32 + lane] = o[n][e];
+                    for (int e = 0; e < 4; ++e) fo[(4 * n + e) * 32 + lane] = o[n][e];
                 }
-                reinterpret_cast<float4*>(mlbuf)[lane] = make_float4(mA, lA, mB, lB);
-                if (lane == 0) {
-                    EpiMeta m;
-                    m.layer = it.layer; m.b = it.b; m.g = it.g; m.chunk = it.chunk; m.nchunks = it.nchunks;
-                    m.slot_base = it.slot_base; m.valid = 1; m.pad = 0;
-                    ctl.meta = m;
+                fml[lane] = make_float4(mA, lA, mB, lB);
+            }
+            consumer_sync();
+            {
+                const uint8_t* stage = ring + s_last * C::kStageBytes;
+                float4 mlf[C::kConsumerWarps];
+#pragma unroll
+                for (int f = 0; f < C::kConsumerWarps; ++f)
+                    mlf[f] = reinterpret_cast<const float4*>(stage + (C::kTilePages + f) * C::kPageBytes)[lane];
+                float MA = mlf[0].x, MB = mlf[0].z;
+#pragma unroll
+                for (int f = 1; f < C::kConsumerWarps; ++f) { MA = fmaxf(MA, mlf[f].x); MB = fmaxf(MB, mlf[f].z); }
+                const float muA = (MA == -INFINITY) ? 0.f : MA, muB = (MB == -INFINITY) ? 0.f : MB;
+                float scA[C::kConsumerWarps], scB[C::kConsumerWarps];
+                float lAf = 0.f, lBf = 0.f;
+#pragma unroll
+                for (int f = 0; f < C::kConsumerWarps; ++f) {
+                    scA[f] = ex2(mlf[f].x - muA);
+                    scB[f] = ex2(mlf[f].z - muB);
+                    lAf = fmaf(mlf[f].y, scA[f], lAf);
+                    lBf = fmaf(mlf[f].w, scB[f], lBf);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(efull);
+                constexpr int kRows = (D / 16) / C::kConsumerWarps;  // fragment rows this warp finishes
+                float fin[kRows][4];
+#pragma unroll
+                for (int r = 0; r < kRows; ++r) {
+                    const int n = warp * kRows + r;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float a = 0.f;
+#pragma unroll
+                        for (int f = 0; f < C::kConsumerWarps; ++f) {
+                            const float v = reinterpret_cast<const float*>(stage + f * C::kPageBytes)[(4 * n + e) * 32 + lane];
+                            a = fmaf(v, (e & 1) ? scB[f] : scA[f], a);
+                        }
+                        fin[r][e] = a;
+                    }
+                }
+                // the hand-off buffer is free once the epilogue warp has taken the previous item out of it
+                if (!mbar_wait(efree, (ecnt & 1) ^ 1, abort_flag, p.status)) { aborted = true; break; }
+#pragma unroll
+                for (int r = 0; r < kRows; ++r) {
+                    const int n = warp * kRows + r;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) mbuf[(4 * n + e) * 32 + lane] = fin[r][e];
+                }
+                if (warp == 0) {
+                    reinterpret_cast<float4*>(mlbuf)[lane] = make_float4(MA, lAf, MB, lBf);
+                    if (lane == 0) {
+                        EpiMeta m;
+                        m.layer = it.layer; m.b = it.b; m.g = it.g; m.chunk = it.chunk; m.nchunks = it.nchunks;
+                        m.slot_base = it.slot_base; m.valid = 1; m.pad = 0;
+                        ctl.meta = m;
+                    }
+                }
+            }
+            // generic-proxy writes into the stage are ordered before the copies that will refill it
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            consumer_sync();
+            if (lane == 0) {
+                mbar_arrive(empty0 + 8 * s_last);
+                if (warp == 0) mbar_arrive(efull);
             }
             ++ecnt;
 #ifdef ODA_TIMELINE
