@@ -460,7 +460,11 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     bool aborted = false;
 
     int span_pages = 0;
-    uint64_t t_first = 0;
+    // calibration: the rate is taken over the first half of the span, while every other CTA is still
+    // streaming too (a slow CTA speeds up once the fast ones have left, which would hide part of the
+    // difference the weights are meant to remove)
+    uint64_t t_first = 0, t_half = 0;
+    int pages_done = 0, pages_half = 0;
     {
         int x, x_end;
         span_range(plan, span, x, x_end);
@@ -579,6 +583,13 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                     }
                 }
                 __syncwarp();
+                if (p.sm_stats) {
+                    pages_done += tw.npages;
+                    if (pages_half == 0 && 2 * pages_done >= span_pages) {
+                        pages_half = pages_done;
+                        t_half = globaltimer_ns();
+                    }
+                }
                 tw.next(it);
                 if (tw.done())
                     s_last = s;
@@ -686,12 +697,12 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
 #endif
     }
     // calibration run: how long this SM took to stream how many pages
-    if (p.sm_stats && tid == 0 && !aborted && plan.nseg == (int)gridDim.x) {
+    if (p.sm_stats && tid == 0 && !aborted && pages_half > 0 && plan.nseg == (int)gridDim.x) {
         unsigned smid;
         asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
         if ((int)smid < p.num_sms) {
-            atomicAdd(p.sm_stats + 2 * smid, (unsigned long long)span_pages);
-            atomicAdd(p.sm_stats + 2 * smid + 1, (unsigned long long)(globaltimer_ns() - t_first));
+            atomicAdd(p.sm_stats + 2 * smid, (unsigned long long)pages_half);
+            atomicAdd(p.sm_stats + 2 * smid + 1, (unsigned long long)(t_half - t_first));
         }
     }
     // end marker for the epilogue warp (also on the abort path, where its own waits are bounded)
