@@ -195,6 +195,7 @@ def config_dict(wl, args, realised):
             "global_batch": wl.B * args.gpus, "parallelism": f"dp{args.gpus} (requests sharded, no collective)",
             "l2": "flushed between timed steps (256 MiB write, then 256 MiB read so that no dirty lines are left; untimed)",
             "launch": "one CUDA graph replay per step",
+            "arithmetic": "bf16 K/V/q, bf16 tensor-core products with f32 accumulation, f32 softmax and outputs",
             "gated_pass": "remainder S^F minus S^L merged with Local" if getattr(wl, "reuse_local", False) else "recomputes all of S^F"}
 
 
@@ -424,7 +425,7 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic", "config": config_dict(wl, args, realised),
             "gpu_launches": launches_per_step * args.steps,
             "step_gbs": step_bytes / (total_ms / args.steps * 1e-3) / 1e9,
