@@ -180,7 +180,8 @@ def reference_arm(args, wl, realised_rate=None):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": config_dict(wl, args, realised),
+            "data": "synthetic", "config": dict(config_dict(wl, args, realised), arithmetic="f64 (the oracle)",
+                                                launch="host threads over (layer, request, head) units"),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
