@@ -312,6 +312,15 @@ __device__ __forceinline__ void prefetch_block_table(const AttnParams& p)
     const char* base = reinterpret_cast<const char*>(p.block_table);
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < lines; i += (size_t)gridDim.x * blockDim.x)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + i * 128));
+    // the small arrays the plan starts from (a line that the previous kernel still rewrites is
+    // updated in L2, where it is read from later)
+    if (blockIdx.x == 0) {
+        const int t = threadIdx.x;
+        if (t * 32 < p.batch) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.seq_lens + t * 32));
+        if (p.flags && t * 128 < p.batch) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.flags + t * 128));
+        if (t * 4 < p.layer_end - p.layer_begin) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.layers + p.layer_begin + t * 4));
+        if (p.cum_share && t < 6) asm volatile("prefetch.global.L2 [%0];" ::"l"(p.cum_share + t * 64));
+    }
 }
 
 __device__ __forceinline__ int span_begin(const Plan& pl, int j)
