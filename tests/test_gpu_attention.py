@@ -235,3 +235,27 @@ def test_maximum_batch_many_layers_tiny_sequences(variant):
             else:
                 assert (full[l, b] == -3.0).all()
     assert ctx.read_device_status() == 0
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_layer_and_batch_limits_together(variant):
+    """256 layers x 128 requests (both limits of a context) with four layer classes and group
+    size 1: 32,768 units of 1..7 pages on one launch; one step beyond either limit is refused."""
+    B, L = 128, 256
+    rng = np.random.RandomState(11)
+    seq = rng.randint(1, 100, size=B).tolist()
+    prob = make_problem(57, L, B, 1, 1, 64, seq, kv_layers=2)
+    classes = [(16, 0, 1), (40, 4, 1), (7, 1, 0), (64, 2, 1)]
+    windows, sinks, gated = (list(v) for v in zip(*[classes[(l * 7) % 4] for l in range(L)]))
+    kv_index = [l % 2 for l in range(L)]
+    ctx = gh.make_ctx(prob, windows, sinks, gated, kv_index=kv_index, variant=variant)
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", windows, sinks, layer_kv_index=kv_index, nthreads=8)
+    gh.assert_close(out, ref, gh.ATOL_OUT, "limits local")
+    gh.assert_close(lse, rlse, gh.ATOL_LSE, "limits lse")
+    assert ctx.read_device_status() == 0
+    with pytest.raises(binding.OdaError):
+        gh.make_ctx(dict(prob, L=257), windows + [16], sinks + [0], gated + [1], kv_index=kv_index + [0], variant=variant)
+    with pytest.raises(binding.OdaError):
+        gh.make_ctx(prob, windows, sinks, gated, kv_index=kv_index, variant=variant, max_batch=129)
