@@ -14,6 +14,14 @@ from paper_2609_20734_b200 import sharding
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+def _free_port():
+    import socket
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def _worker(rank, world, port, ret):
     sys.path.insert(0, ROOT)
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
@@ -38,7 +46,7 @@ def test_request_sharding_two_ranks_gloo():
     world = 2
     with mp.Manager() as m:
         ret = m.dict()
-        mp.spawn(_worker, args=(world, 29611, ret), nprocs=world, join=True)
+        mp.spawn(_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
         res = dict(ret)
     from tests.helpers import make_problem, oracle_attention
 
@@ -115,7 +123,7 @@ def test_kv_head_tensor_parallel_two_ranks_gloo():
     world = 2
     with mp.Manager() as m:
         ret = m.dict()
-        mp.spawn(_tp_worker, args=(world, 29613, ret), nprocs=world, join=True)
+        mp.spawn(_tp_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
         res = dict(ret)
     from oracle import oda_oracle as orc
     from tests.helpers import oracle_attention
@@ -191,7 +199,7 @@ def test_sequence_sharded_full_two_ranks_gloo():
     world = 2
     with mp.Manager() as m:
         ret = m.dict()
-        mp.spawn(_sp_worker, args=(world, 29615, ret), nprocs=world, join=True)
+        mp.spawn(_sp_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
         res = dict(ret)
     from tests.helpers import make_problem, oracle_attention
 
