@@ -346,6 +346,35 @@ __device__ __forceinline__ int span_of(const Plan& pl, int x)
     return lo;
 }
 
+// span_of for a page known to lie at or before (dir < 0) / at or after (dir > 0) span j: a unit
+// rarely covers more than a few spans, so a short walk from j beats the search over all spans
+__device__ __forceinline__ int span_of_near(const Plan& pl, int x, int j, int dir)
+{
+    if (!pl.weighted) return span_of(pl, x);
+    if (dir < 0) {
+        for (int k = 0; k < 3; ++k) {
+            if (span_begin(pl, j) <= x) return j;
+            --j;
+        }
+        int lo = 0, hi = j + 1;  // span_begin(0) = 0 <= x
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (span_begin(pl, mid) <= x) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+    for (int k = 0; k < 3; ++k) {
+        if (span_begin(pl, j + 1) > x) return j;
+        ++j;
+    }
+    int lo = j, hi = pl.nseg;  // span_begin(nseg) = total_pages > x
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (span_begin(pl, mid) <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
 // The item of span j that starts at axis page x (x0 <= x < x_end of span_range(j)).
 // Returns the number of axis pages it covers (>= 1).
 __device__ inline int decode_item(const AttnParams& p, const Plan& pl, int j, int x, int x_end, Item& it)
@@ -370,7 +399,7 @@ __device__ inline int decode_item(const AttnParams& p, const Plan& pl, int j, in
     const int off = r2 - g * np;
     const int unit0 = x - off;                       // axis page where the unit starts
     const int take = min(np - off, x_end - x);
-    const int j0 = span_of(pl, unit0), j1 = span_of(pl, unit0 + np - 1);
+    const int j0 = span_of_near(pl, unit0, j, -1), j1 = span_of_near(pl, unit0 + np - 1, j, +1);
     it.layer = p.layer_begin + lo;
     it.b = blo;
     it.g = g;

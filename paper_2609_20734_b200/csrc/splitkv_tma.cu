@@ -243,7 +243,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         int blk_cur = 0, blk_nxt = 0;
         bool have = fetch(cur, blk_cur);
         while (have && !dead) {
-            const bool have_next = fetch(nxt, blk_nxt);  // block ids of the next run are in flight during this one
+            // the next run is decoded, and its block ids requested, once this run's first tile is on
+            // its way (at the start of the span nothing may delay the first copy)
+            bool have_next = false, fetched = false;
             for (int t0 = 0; t0 < cur.n; t0 += 4) {
                 const int np = min(4, cur.n - t0);
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
@@ -269,6 +271,10 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                     bulk_load(smem_u32(qring + s * C::kQSlotBytes), cur.q, kQBytes, full0 + 8 * s);
                 }
                 ++cnt;
+                if (!fetched) {
+                    have_next = fetch(nxt, blk_nxt);
+                    fetched = true;
+                }
             }
             cur = nxt;
             blk_cur = blk_nxt;
