@@ -376,14 +376,29 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             } else {
                 float4* slots = reinterpret_cast<float4*>(p.partials) + (size_t)it.slot_base * (kFragSlotFloats / 4);
                 float4* mine = slots + (size_t)it.chunk * (kFragSlotFloats / 4);
-#pragma unroll
-                for (int n = 0; n < D / 16; ++n) __stcg(mine + n * 32 + lane, make_float4(o[n][0], o[n][1], o[n][2], o[n][3]));
-                __stcg(mine + 8 * 32 + lane, ml);
-                __threadfence();
-                __syncwarp();
+                // If every other chunk of the unit has already arrived (the usual case for the last
+                // item of a span: its neighbour finished that unit long ago), this CTA merges, and its own
+                // chunk never has to leave its registers: no partial store, fence and ticket round trips.
                 int last = 0;
-                if (lane == 0) last = take_ticket(p, it);
+                if (lane == 0) {
+                    int* tk = p.tickets + ((size_t)it.layer * p.max_batch + it.b) * p.num_kv_heads + it.g;
+                    int seen;
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(tk) : "memory");
+                    if (seen == it.nchunks - 1) {
+                        *tk = 0;  // ready for the next launch
+                        last = 1;
+                    }
+                }
                 last = __shfl_sync(0xffffffffu, last, 0);
+                if (!last) {
+#pragma unroll
+                    for (int n = 0; n < D / 16; ++n) __stcg(mine + n * 32 + lane, make_float4(o[n][0], o[n][1], o[n][2], o[n][3]));
+                    __stcg(mine + 8 * 32 + lane, ml);
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) last = take_ticket(p, it);
+                    last = __shfl_sync(0xffffffffu, last, 0);
+                }
                 if (last) {
                     __threadfence();
                     // fold the chunks in index order (this CTA's own chunk comes from its registers);
