@@ -50,8 +50,8 @@ def sum_over_ranks(t, group=None):
     """The step's one collective: element-wise sum of a small fp32 tensor over the ranks."""
     import torch.distributed as dist
 
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    if dist.is_available() and dist.is_initialized():
+        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)   # a one-rank group reduces to itself
     return t
 
 
@@ -111,7 +111,7 @@ def gather_over_ranks(dst, src, group=None):
     """All-gather of equally shaped tensors into dst[rank] (dst has a leading world axis)."""
     import torch.distributed as dist
 
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+    if dist.is_available() and dist.is_initialized():
         dist.all_gather(list(dst.unbind(0)), src, group=group)   # dst[r] are contiguous views
     else:
         dst.copy_(src.reshape(dst.shape))

@@ -148,3 +148,69 @@ def test_sequence_sharded_full_pass_matches_oracle(world):
                 gh.assert_close(ls[l, b], want_lse[l, b], gh.ATOL_LSE, f"layer {l} request {b} lse")
             else:
                 assert (o[l, b] == 7.0).all() and (ls[l, b] == 7.0).all()   # untouched
+
+
+def test_sharded_steps_through_nccl_on_one_rank():
+    """The two sharded compositions with their collectives issued through torch.distributed's NCCL
+    backend (a one-rank group: the library calls and the collectives share the current stream the
+    way they do on several GPUs).  Results equal the unsharded library calls bitwise."""
+    import os
+    import socket
+
+    import torch.distributed as dist
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        L, B, Hq, Hkv, D, d_ext, d_h = 2, 3, 8, 2, 128, 8, 24
+        windows, sinks, gated = [64, 32], [4, 0], [1, 1]
+        prob = make_problem(91, L, B, Hq, Hkv, D, [300, 40, 1000])
+        head = dict(W1=synth.gauss_f32_tensor(9, synth.STREAM_W1, (d_h, d_ext + Hq * D), std=0.05),
+                    b1=synth.gauss_f32_tensor(9, synth.STREAM_B1, (d_h,), std=0.05),
+                    w2=synth.gauss_f32_tensor(9, synth.STREAM_W2, (d_h,), std=0.3),
+                    b2=synth.gauss_f32_tensor(9, synth.STREAM_B2, (1,), std=0.05), use_attn_out=1)
+        hd = gh.head_to_device(head)
+        fe = torch.from_numpy(synth.gauss_f32_tensor(9, synth.STREAM_FEAT, (B, d_ext))).cuda()
+        ctx = gh.make_ctx(prob, windows, sinks, gated, head=(d_ext, 1, d_h))
+        dev = gh.upload(prob)
+        # reference: the fused single-GPU step
+        out0, lse0 = gh.new_out(prob)
+        sc0 = torch.zeros(B, device="cuda")
+        fl0 = torch.zeros(B, dtype=torch.uint8, device="cuda")
+        ctx.step(ctx.step_args(B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out0, sc0, fl0,
+                               feat_ext=fe, head=hd, threshold=0.5, lse=lse0))
+        # tensor-parallel composition on the one rank
+        sh = tp.head_shard(0, 1, Hq, Hkv, D, d_ext, True)
+        out1, lse1 = gh.new_out(prob)
+        sc1 = torch.zeros(B, device="cuda")
+        fl1 = torch.zeros(B, dtype=torch.uint8, device="cuda")
+        pre = torch.zeros((B, d_h), device="cuda")
+        tp.tp_step(ctx, sh, B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out1, W1=hd["W1"],
+                   b1=hd["b1"], w2=hd["w2"], b2=hd["b2"], threshold=0.5, pre=pre, scores=sc1, flags=fl1,
+                   feat_ext=fe, lse=lse1)
+        torch.cuda.synchronize()
+        assert torch.equal(fl1, fl0)
+        np.testing.assert_allclose(sc1.cpu().numpy(), sc0.cpu().numpy(), rtol=0, atol=1e-6)
+        assert torch.equal(out1, out0) and torch.equal(lse1, lse0)
+        # sequence-sharded composition on the one rank: gather + merge of a single part is the identity
+        ones = torch.ones(B, dtype=torch.uint8, device="cuda")
+        part_out, part_lse = gh.new_out(prob)
+        parts_out = torch.zeros((1,) + tuple(part_out.shape), device="cuda")
+        parts_lse = torch.zeros((1,) + tuple(part_lse.shape), device="cuda")
+        out2 = torch.zeros_like(part_out)
+        lse2 = torch.zeros_like(part_lse)
+        tokens = dev["seq_lens"].reshape(1, B).contiguous()
+        tp.sp_full_step(ctx, 1, B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], tokens, ones,
+                        part_out, part_lse, parts_out, parts_lse, out2, lse2)
+        torch.cuda.synchronize()
+        full, flse = gh.new_out(prob)
+        ctx.full_decode_gated(0, L, B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], ones, full, flse)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(out2.cpu().numpy(), full.cpu().numpy(), rtol=0, atol=1e-6)
+        np.testing.assert_allclose(lse2.cpu().numpy(), flse.cpu().numpy(), rtol=0, atol=1e-6)
+        assert ctx.read_device_status() == 0
+    finally:
+        dist.destroy_process_group()
