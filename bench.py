@@ -158,12 +158,12 @@ def reference_arm(args, wl, realised_rate=None):
     flags = [wl.override_flags(s) for s in range(args.warmup + args.steps)]
     realised = float(np.mean([f.mean() for f in flags[args.warmup:]])) if realised_rate is None else realised_rate
 
-    def one(step, mode, n):
+    def one(step, mode, n, threads=None):
         q = wl.q_host(step)[:n]
         t0 = time.perf_counter()
         orc.attention(mode, q, k, v, table, np.asarray(wl.seq_lens0) + step, num_kv_heads=wl.Hkv,
                       block_size=16, layout=lay, layer_window=wl.windows[:n], layer_sinks=wl.sinks[:n],
-                      nthreads=cores)
+                      nthreads=cores if threads is None else threads)
         return time.perf_counter() - t0
 
     for s in range(args.warmup):
@@ -175,6 +175,8 @@ def reference_arm(args, wl, realised_rate=None):
             tf.append(one(args.warmup + s, "full", nf) * sum(wl.gated) / nf)
     step_s = float(np.mean(tl) + realised * np.mean(tf))
     val = wl.B / step_s
+    # the same sample on one thread (one Local and one Full call)
+    step_1 = one(args.warmup, "local", nl, 1) * wl.L / nl + realised * one(args.warmup, "full", nf, 1) * sum(wl.gated) / nf
     sample = (f"per step: Local on {nl} of {wl.L} layers (every step) and Full on {nf} of {wl.L} layers "
               f"({len(tf)} steps), scaled to all layers and combined at the realised recall rate {realised:.3f}")
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
@@ -182,7 +184,8 @@ def reference_arm(args, wl, realised_rate=None):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": dict(config_dict(wl, args, realised), arithmetic="f64 (the oracle)",
                                                 launch="host threads over (layer, request, head) units"),
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "value_1_thread": wl.B / step_1},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
