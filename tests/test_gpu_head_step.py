@@ -266,3 +266,39 @@ def test_remainder_only_gated_pass_equals_full():
     gh.assert_close(outs[(1, True)][1], ref.lse, gh.ATOL_LSE, "merged lse")
     np.testing.assert_allclose(outs[(1, True)][0], outs[(0, True)][0], rtol=0, atol=1e-5)
     np.testing.assert_array_equal(outs[(1, False)][0], outs[(1, True)][0])
+
+
+@pytest.mark.parametrize("first_k,expect", [(2, 126), (4, 252), (8, 504)])
+def test_prescribed_schedule_counts_over_1008_routed_steps(first_k, expect):
+    """The paper's timing protocol: Full on the first k of every 16 routed steps, 1,008 steps.  The
+    device counters of one graph-replayed step (head still running, lengths advancing on the device)
+    must read exactly 1,008 steps and 126 / 252 / 504 Full calls."""
+    steps = 1008
+    wl = workloads.make("tiny", seq_lens0=np.array([100], np.int32), steps=steps + 2, schedule="periodic")
+    st = workloads.materialize(wl)
+    ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks))
+    out = torch.zeros((wl.L, wl.B, wl.Hq, wl.D), device="cuda")
+    scores = torch.zeros(wl.B, device="cuda")
+    flags = torch.zeros(wl.B, dtype=torch.uint8, device="cuda")
+    counters = torch.zeros((wl.B, 2), dtype=torch.int32, device="cuda")
+    ov = torch.zeros(wl.B, dtype=torch.uint8, device="cuda")
+    fe = torch.from_numpy(wl.feat_host(0)).cuda()
+    q = workloads.q_device(wl, 0)
+    args = ctx.step_args(wl.B, q, st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, scores, flags,
+                         feat_ext=fe, head=st.head, threshold=0.5, override_flags=ov, counters=counters,
+                         advance_seq_lens=True)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            ctx.step(args, stream=s.cuda_stream)
+    sched = torch.from_numpy(np.stack([synth.periodic_flags(t, wl.B, first_k) for t in range(steps)])).cuda()
+    for t in range(steps):
+        ov.copy_(sched[t])
+        g.replay()
+    torch.cuda.synchronize()
+    c = counters.cpu().numpy()
+    assert c[0, 0] == steps and c[0, 1] == expect
+    assert st.seq_lens.item() == 100 + steps
+    assert ctx.read_device_status() == 0
