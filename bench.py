@@ -515,6 +515,25 @@ def main():
                 torch.cuda.synchronize()
                 if r >= 2:
                     kt_warm[name].append(e0.elapsed_time(e1))
+        # what a backbone with other work between its layers sees: the Local pass as one launch per
+        # layer (chained by programmatic dependent launch inside one graph)
+        g_layers = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g_layers, stream=side):
+                for l in range(L):
+                    ctx.local_decode(l, l + 1, B, qs[0], st.k_cache, st.v_cache, st.block_table, st.seq_lens,
+                                     out, lse, stream=side.cuda_stream)
+        torch.cuda.synchronize()
+        t_layers = []
+        for r in range(reps + 2):
+            flush.fill_(r)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g_layers.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            if r >= 2:
+                t_layers.append(e0.elapsed_time(e1))
         lb, fb = wl.algorithmic_bytes(np.asarray(wl.seq_lens0), np.ones(B))
         kernels = {}
         for name, nbytes in (("local", lb), ("full", fb)):
@@ -527,6 +546,10 @@ def main():
         line["roofline"] = dict(kernels[dominant], kernel=f"splitkv ({dominant} pass)", peak_source=peak_src)
         line["roofline_other"] = dict(kernels["local" if dominant == "full" else "full"],
                                       kernel=f"splitkv ({'local' if dominant == 'full' else 'full'} pass)")
+        line["local_pass_one_launch_per_layer"] = {
+            "us": float(np.mean(t_layers)) * 1e3, "launches": L,
+            "gbs": lb / (float(np.mean(t_layers)) * 1e-3) / 1e9,
+            "note": "context: the same Local work as one launch per layer in one graph, L2 flushed before the graph"}
         traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(traffic_path):  # DRAM bytes per launch from the committed ncu summary
             tr = json.load(open(traffic_path))
