@@ -138,6 +138,24 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def schedule_flags(wl, warmup, steps):
+    """Forced flags of a run, one uint8 array [B] per step (None if the head decides).  For the seeded
+    Bernoulli schedule the draw is conditioned on its sum: every request recalls on exactly
+    round(rate * steps) of the timed steps, at positions chosen by a seeded shuffle, so that the
+    realised rate equals the target whatever the number of timed steps is (an unconditioned draw over
+    a handful of steps can land anywhere: 0.8 instead of 0.25 over 5 steps).  Warm-up steps keep the
+    plain hashed draw."""
+    if wl.schedule != "bernoulli":
+        return [wl.override_flags(s) for s in range(warmup + steps)]
+    flags = [wl.override_flags(s) for s in range(warmup)]
+    timed = np.zeros((steps, wl.B), np.uint8)
+    k = int(round(wl.recall_rate * steps))
+    for b in range(wl.B):
+        order = np.random.default_rng([wl.seed, b, steps]).permutation(steps)
+        timed[order[:k], b] = 1
+    return flags + [timed[s] for s in range(steps)]
+
+
 def reference_arm(args, wl, realised_rate=None):
     """The oracle, as it stands, timed on the host cores.  A step is a bounded sample of the
     workload: Local on `nl` layers and Full on `nf` layers of the stack, extrapolated to all
@@ -155,7 +173,7 @@ def reference_arm(args, wl, realised_rate=None):
     kk, vk = synth.stream_key(wl.seed, synth.STREAM_K), synth.stream_key(wl.seed, synth.STREAM_V)
     idx = np.arange(0, nl * lay.layer_stride, dtype=np.uint64)
     k, v = synth.gauss_bf16(kk, idx), synth.gauss_bf16(vk, idx)
-    flags = [wl.override_flags(s) for s in range(args.warmup + args.steps)]
+    flags = schedule_flags(wl, args.warmup, args.steps)
     realised = float(np.mean([f.mean() for f in flags[args.warmup:]])) if realised_rate is None else realised_rate
 
     def one(step, mode, n, threads=None):
@@ -193,7 +211,8 @@ def reference_arm(args, wl, realised_rate=None):
 def config_dict(wl, args, realised):
     return {"workload": f"{wl.name}: L={wl.L} B={wl.B} Hq={wl.Hq} Hkv={wl.Hkv} D={wl.D} "
                         f"context={int(np.max(wl.seq_lens0))} window={wl.windows[0]} sinks={wl.sinks[0]} block=16 "
-                        f"bf16 KV ~N(0,1), {wl.schedule} flags, "
+                        f"bf16 KV ~N(0,1), "
+                        f"{'seeded Bernoulli flags conditioned on their count' if wl.schedule == 'bernoulli' else wl.schedule + ' flags'}, "
                         f"{'shuffled' if wl.shuffled else 'in-order'} block tables",
             "recall_rate_target": wl.recall_rate, "recall_rate_realised": realised,
             "global_batch": wl.B * args.gpus, "parallelism": f"dp{args.gpus} (requests sharded, no collective)",
@@ -334,7 +353,7 @@ def main():
     shape = (L, B, wl.Hq, wl.D)
     nsteps = args.warmup + args.steps
     qs = [workloads.q_device(wl, s) for s in range(nsteps)]
-    flags_h = [wl.override_flags(s) for s in range(nsteps)]
+    flags_h = schedule_flags(wl, args.warmup, args.steps)
     head_decides = flags_h[0] is None        # flags come from the recall head (no forced schedule)
     ovs = None if head_decides else [torch.from_numpy(f).cuda() for f in flags_h]
     flags_log = torch.zeros((nsteps, B), dtype=torch.uint8, device="cuda")
@@ -564,7 +583,7 @@ def main():
             n_sw = min(args.steps, 32)
             for rate in SWEEP_RATES:
                 wl_r = workloads.make(args.config, recall_rate=rate)
-                fl = [wl_r.override_flags(s) for s in range(n_sw)]
+                fl = schedule_flags(wl_r, 0, n_sw)
                 st.seq_lens.copy_(seq0)
                 tms = []
                 for s in range(n_sw):
