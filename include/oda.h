@@ -185,6 +185,39 @@ oda_status_t oda_recall_finalize(oda_ctx_t* ctx, int32_t batch, const float* pre
                                  uint8_t* flags, int32_t* counters, void* stream);
 
 /*
+ * The same decision with the exchange inside the kernel (no collective library call): every rank
+ * stores its share of W1 x into slot [rank] of every rank's receive buffer (plain peer stores),
+ * raises an arrival flag carrying `epoch` in every rank's flag array, waits -- at most timeout_ns
+ * (0 => 1 s) -- for all ranks' flags in its own array, adds the shares in rank order and applies
+ * oda_recall_finalize's arithmetic.  All ranks therefore take the same decision bit for bit.
+ *   recv [world] (host array of device pointers): recv[r] is rank r's receive buffer,
+ *     2 * world * batch_max * d_hidden floats, 16-byte aligned, mapped into this GPU's address
+ *     space for every r (peer access / symmetric memory); only recv[own rank] is read;
+ *   arrived [world] (host array): arrived[r] is rank r's flag array of `world` u32, zero at set-up;
+ *   epoch: 1, 2, 3, ... one more on every call, the same on all ranks (buffers alternate by parity;
+ *     a rank can run at most one exchange ahead of the slowest);
+ *   ranks [n_local] (host array): the buffers of the ranks THIS launch runs, ranks rank_base ..
+ *     rank_base + n_local - 1.  In production n_local = 1 (one process per GPU, one CTA).  n_local
+ *     > 1 runs several ranks as the CTAs of one cooperative launch on one GPU (the CTAs wait on one
+ *     another, so they must be co-resident): that is how the protocol is checked without several GPUs.
+ * A wait that runs out sets bit 2 of the device status word and leaves scores / flags untouched.
+ * world <= 8.  The caller makes sure every rank of the group issues the call for the same epoch.
+ */
+typedef struct {
+    const float* pre_local; /* [batch, d_hidden]: oda_recall_preact's output on this rank */
+    float* scores;
+    float* logits;          /* nullable */
+    uint8_t* flags;
+    int32_t* counters;      /* nullable */
+} oda_exchange_rank_t;
+oda_status_t oda_recall_finalize_exchange(oda_ctx_t* ctx, int32_t batch, int32_t world, int32_t rank_base,
+                                          int32_t n_local, const oda_exchange_rank_t* ranks,
+                                          float* const* recv, uint32_t* const* arrived, uint32_t epoch,
+                                          uint64_t timeout_ns, const float* b1, const float* w2,
+                                          const float* b2, float threshold, const uint8_t* override_flags,
+                                          void* stream);
+
+/*
  * Sequence sharding of the gated Full pass (the paper runs on one GPU; this is how the history of
  * Eq. 1's S^F splits over ranks that each hold a range of positions).  Every rank runs
  * oda_full_decode_gated over its own slice (its block table and lengths) and gets, per row,

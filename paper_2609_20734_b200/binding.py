@@ -26,6 +26,7 @@ EXPORTS = [
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
     "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
+    "oda_recall_finalize_exchange",
 ]
 
 
@@ -55,6 +56,11 @@ class _FullHead(ctypes.Structure):
     _fields_ = [("d_model", ctypes.c_int32), ("d_tower", ctypes.c_int32), ("d_ff", ctypes.c_int32),
                 ("n_blocks", ctypes.c_int32), ("eps", ctypes.c_float), ("variant", ctypes.c_int32),
                 ("params", ctypes.c_void_p)]
+
+
+class _ExchangeRank(ctypes.Structure):
+    _fields_ = [("pre_local", ctypes.c_void_p), ("scores", ctypes.c_void_p), ("logits", ctypes.c_void_p),
+                ("flags", ctypes.c_void_p), ("counters", ctypes.c_void_p)]
 
 
 class _StepArgs(ctypes.Structure):
@@ -103,6 +109,9 @@ def load_library():
         lib.oda_recall_finalize.restype = i32
         lib.oda_merge_partials.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_merge_partials.restype = i32
+        lib.oda_recall_finalize_exchange.argtypes = [vp, i32, i32, i32, i32, ctypes.POINTER(_ExchangeRank), vp, vp,
+                                                     ctypes.c_uint32, ctypes.c_uint64, vp, vp, vp, f32, vp, vp]
+        lib.oda_recall_finalize_exchange.restype = i32
         lib.oda_full_decode_gated.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
         lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
@@ -286,6 +295,22 @@ class OdaContext:
         self._check(self.lib.oda_merge_partials(
             self._h, n_parts, layer_begin, layer_end, batch, _ptr(parts_out), _ptr(parts_lse), _ptr(part_tokens),
             _ptr(flags), _ptr(out), _ptr(lse), _stream() if stream is None else stream), "oda_merge_partials")
+
+    def recall_finalize_exchange(self, batch, world, rank_base, ranks, recv, arrived, epoch, b1, w2, b2,
+                                 threshold, override_flags=None, timeout_ns=0, stream=None):
+        """ranks: list of dicts(pre_local, scores, flags[, logits, counters]) for the ranks this launch
+        runs; recv / arrived: the receive buffers and flag arrays of ALL ranks of the group, in rank order."""
+        n_local = len(ranks)
+        arr = (_ExchangeRank * n_local)(*[
+            _ExchangeRank(_ptr(r["pre_local"]), _ptr(r["scores"]), _ptr(r.get("logits")), _ptr(r["flags"]),
+                          _ptr(r.get("counters"))) for r in ranks])
+        recv_p = (ctypes.c_void_p * world)(*[_ptr(t) for t in recv])
+        arr_p = (ctypes.c_void_p * world)(*[_ptr(t) for t in arrived])
+        self._check(self.lib.oda_recall_finalize_exchange(
+            self._h, batch, world, rank_base, n_local, arr, ctypes.cast(recv_p, ctypes.c_void_p),
+            ctypes.cast(arr_p, ctypes.c_void_p), int(epoch), int(timeout_ns), _ptr(b1), _ptr(w2), _ptr(b2),
+            float(threshold), _ptr(override_flags), _stream() if stream is None else stream),
+            "oda_recall_finalize_exchange")
 
     def full_decode_gated(self, layer_begin, layer_end, batch, q_full, k_cache, v_cache, block_table,
                           seq_lens, flags, out, lse=None, stream=None):

@@ -21,7 +21,7 @@ NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 CFLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
-ODA_SOURCES = ["oda_api.cu", "splitkv_simt.cu", "splitkv_tma.cu", "recall_head.cu", "recall_head_full.cu", "recall_head_fused.cu", "commit.cu", "oda_static.cu"]
+ODA_SOURCES = ["oda_api.cu", "splitkv_simt.cu", "splitkv_tma.cu", "recall_head.cu", "recall_exchange.cu", "recall_head_full.cu", "recall_head_fused.cu", "commit.cu", "oda_static.cu"]
 SYNTH_SOURCES = ["synth_fill.cu"]
 
 

@@ -564,6 +564,53 @@ oda_status_t oda_recall_finalize(oda_ctx_t* c, int32_t batch, const float* pre_s
     return ODA_OK;
 }
 
+oda_status_t oda_recall_finalize_exchange(oda_ctx_t* c, int32_t batch, int32_t world, int32_t rank_base,
+                                          int32_t n_local, const oda_exchange_rank_t* ranks, float* const* recv,
+                                          uint32_t* const* arrived, uint32_t epoch, uint64_t timeout_ns,
+                                          const float* b1, const float* w2, const float* b2, float threshold,
+                                          const uint8_t* override_flags, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0) return ODA_OK;
+    if (c->cfg.head_d_hidden <= 0) return fail(c, ODA_ERR_INVALID_ARG, "no recall head configured");
+    if (world < 1 || world > kExchangeMaxWorld) return fail(c, ODA_ERR_UNSUPPORTED, "world outside [1, 8]");
+    if (n_local < 1 || rank_base < 0 || rank_base + n_local > world) return fail(c, ODA_ERR_INVALID_ARG, "ranks of this launch outside [0, world)");
+    if (epoch == 0) return fail(c, ODA_ERR_INVALID_ARG, "epoch starts at 1 (the flag arrays start at 0)");
+    if (!ranks || !recv || !arrived || !b1 || !w2 || !b2) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    ExchangeParams p;
+    std::memset(&p, 0, sizeof p);
+    for (int i = 0; i < n_local; ++i) {
+        if (!ranks[i].pre_local || !ranks[i].scores || !ranks[i].flags) return fail(c, ODA_ERR_INVALID_ARG, "null rank buffer");
+        if (!aligned16(ranks[i].pre_local)) return fail(c, ODA_ERR_INVALID_ARG, "pre_local must be 16-byte aligned");
+        p.ranks[i].pre_local = ranks[i].pre_local;
+        p.ranks[i].scores = ranks[i].scores;
+        p.ranks[i].logits = ranks[i].logits;
+        p.ranks[i].flags = ranks[i].flags;
+        p.ranks[i].counters = ranks[i].counters;
+    }
+    for (int r = 0; r < world; ++r) {
+        if (!recv[r] || !arrived[r]) return fail(c, ODA_ERR_INVALID_ARG, "null receive buffer or flag array");
+        if (!aligned16(recv[r])) return fail(c, ODA_ERR_INVALID_ARG, "receive buffers must be 16-byte aligned");
+        p.recv[r] = recv[r];
+        p.arrived[r] = arrived[r];
+    }
+    p.b1 = b1; p.w2 = w2; p.b2 = b2;
+    p.override_flags = override_flags;
+    p.status = c->ws ? reinterpret_cast<int32_t*>(c->ws + c->lay.status) : nullptr;
+    p.timeout_ns = timeout_ns ? timeout_ns : 1000000000ull;
+    p.batch = batch;
+    p.d_hidden = c->cfg.head_d_hidden;
+    p.world = world;
+    p.rank_base = rank_base;
+    p.epoch = epoch;
+    p.threshold = threshold;
+    cudaError_t e = launch_recall_exchange(p, n_local, static_cast<cudaStream_t>(stream), c->use_pdl && n_local == 1);
+    if (e != cudaSuccess) return cuda_fail(c, e, "recall head (exchange + second layer) launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
 oda_status_t oda_write_current_kv(oda_ctx_t* c, int32_t batch, const void* k_cur, const void* v_cur,
                                   const uint8_t* mask, void* k_cache, void* v_cache, const int32_t* bt,
                                   const int32_t* sl, void* stream)

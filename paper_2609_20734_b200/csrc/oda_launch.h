@@ -76,6 +76,30 @@ struct HeadParams {
 
 constexpr int kMaxHeadBatch = 128;
 
+// the tensor-parallel decision with its exchange fused in (recall_exchange.cu)
+constexpr int kExchangeThreads = 256;
+constexpr int kExchangeMaxWorld = 8;
+struct ExchangeRank {            // one rank's own buffers
+    const float* pre_local;      // [batch][d_hidden] this rank's share of W1 x
+    float* scores;
+    float* logits;               // nullable
+    uint8_t* flags;
+    int32_t* counters;           // nullable
+};
+struct ExchangeParams {
+    ExchangeRank ranks[kExchangeMaxWorld];   // the ranks this launch runs: one in production
+    float* recv[kExchangeMaxWorld];          // recv[r]: rank r's receive buffer [2][world][batch * d_hidden]
+    uint32_t* arrived[kExchangeMaxWorld];    // arrived[r]: rank r's arrival flags [world]
+    const float *b1, *w2, *b2;
+    const uint8_t* override_flags;
+    int32_t* status;
+    unsigned long long timeout_ns;
+    int32_t batch, d_hidden, world, rank_base;
+    uint32_t epoch;
+    float threshold;
+};
+cudaError_t launch_recall_exchange(const ExchangeParams& p, int n_local, cudaStream_t st, bool pdl = false);
+
 int recall_head_grid(int d_hidden);
 int recall_head_ksplits(int d_in);
 cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl = false);

@@ -131,3 +131,63 @@ def sp_full_step(ctx, world, batch, q_full, k_cache, v_cache, block_table_local,
     gather(parts_out, part_out)
     gather(parts_lse, part_lse)
     ctx.merge_partials(world, 0, L, batch, parts_out, parts_lse, flags, out, lse, part_tokens=part_tokens)
+
+
+# ---- the decision's exchange fused into the kernel (no collective call) ------------------------
+class ExchangeBuffers:
+    """Receive buffers and arrival flags of every rank of a group, as the library wants them: in
+    rank order, each entry a tensor (ranks living in this process) or a raw device address (a
+    peer's buffer mapped into this GPU's address space).  `epoch` counts the exchanges."""
+
+    def __init__(self, recv, arrived, keep=None):
+        self.recv, self.arrived, self.keep, self.epoch = recv, arrived, keep, 0
+
+    @classmethod
+    def local(cls, world, batch, d_hidden, device="cuda"):
+        """All ranks in this process on one GPU: for checking the protocol with one cooperative launch."""
+        import torch
+
+        recv = [torch.zeros((2, world, batch, d_hidden), device=device) for _ in range(world)]
+        arrived = [torch.zeros(world, dtype=torch.int32, device=device) for _ in range(world)]
+        return cls(recv, arrived)
+
+    @classmethod
+    def symmetric(cls, group, batch, d_hidden, device="cuda"):
+        """One rank per process and GPU: buffers in torch's symmetric memory, peers' addresses from
+        its rendezvous.  Not tested on a GPU (this build had one): the addresses are used for plain
+        peer stores only, never for multicast or TMA."""
+        import torch
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm
+
+        world = dist.get_world_size(group)
+        recv = symm.empty((2, world, batch, d_hidden), dtype=torch.float32, device=device)
+        arrived = symm.empty((world,), dtype=torch.int32, device=device)
+        recv.zero_()
+        arrived.zero_()
+        h_recv = symm.rendezvous(recv, group)
+        h_arr = symm.rendezvous(arrived, group)
+        dist.barrier(group)    # every rank's flags are zero before the first exchange
+        return cls([int(p) for p in h_recv.buffer_ptrs], [int(p) for p in h_arr.buffer_ptrs],
+                   keep=(recv, arrived, h_recv, h_arr))
+
+    def next_epoch(self):
+        self.epoch += 1
+        return self.epoch
+
+
+def tp_step_fused(ctx, shard: HeadShard, batch, q_local, k_cache, v_cache, block_table, seq_lens, out, *,
+                  W1, b1, w2, b2, threshold, pre, scores, flags, buffers: ExchangeBuffers, feat_ext=None,
+                  q_full=None, logits=None, lse=None, override_flags=None, counters=None, timeout_ns=0):
+    """tp_step with the all-reduce replaced by the library's own exchange kernel: Local pass, the rank's
+    share of W1 x, then ONE kernel that pushes the share to every peer, waits for theirs and decides, then
+    the gated Full pass.  Every rank of the group must make this call once per step."""
+    tp_local_and_preact(ctx, shard, batch, q_local, k_cache, v_cache, block_table, seq_lens, out,
+                        W1=W1, pre=pre, feat_ext=feat_ext, lse=lse)
+    ctx.recall_finalize_exchange(batch, shard.world, shard.rank,
+                                 [dict(pre_local=pre, scores=scores, logits=logits, flags=flags, counters=counters)],
+                                 buffers.recv, buffers.arrived, buffers.next_epoch(), b1, w2, b2, threshold,
+                                 override_flags=override_flags, timeout_ns=timeout_ns)
+    ctx.full_decode_gated(0, ctx.cfg.num_layers, batch, q_local if q_full is None else q_full, k_cache, v_cache,
+                          block_table, seq_lens, flags, out, lse)
+    return flags

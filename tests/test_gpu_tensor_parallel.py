@@ -222,3 +222,104 @@ def test_sharded_steps_through_nccl_on_one_rank():
         assert ctx.read_device_status() == 0
     finally:
         dist.destroy_process_group()
+
+
+def _exchange_setup(world, B, d_h, seed=3):
+    recv = [torch.full((2, world, B, d_h), float("nan"), device="cuda") for _ in range(world)]
+    arrived = [torch.zeros(world, dtype=torch.int32, device="cuda") for _ in range(world)]
+    return recv, arrived
+
+
+@pytest.mark.parametrize("world", [1, 2, 4, 8])
+def test_fused_exchange_decision_matches_oracle_and_agrees_across_ranks(world):
+    """The tensor-parallel decision with its exchange inside the kernel (peer stores + arrival
+    flags instead of a collective call).  The ranks are the CTAs of one cooperative launch with
+    separate buffers; three consecutive steps exercise the epoch flags and the alternating buffers."""
+    B, d_in, d_h = 5, 8 * 64, 40
+    ctx = gh.make_ctx(make_problem(1, 1, B, 8, 8, 64, [20] * B), [8], [0], [1], head=(0, 1, d_h))
+    head = dict(W1=synth.gauss_f32_tensor(9, synth.STREAM_W1, (d_h, d_in), std=0.05),
+                b1=synth.gauss_f32_tensor(9, synth.STREAM_B1, (d_h,), std=0.05),
+                w2=synth.gauss_f32_tensor(9, synth.STREAM_W2, (d_h,), std=0.3),
+                b2=synth.gauss_f32_tensor(9, synth.STREAM_B2, (1,), std=0.05), use_attn_out=1)
+    hd = gh.head_to_device(head)
+    recv, arrived = _exchange_setup(world, B, d_h)
+    cols = d_in // world
+    for step in range(3):
+        x = synth.gauss_f32_tensor(20 + step, synth.STREAM_FEAT, (B, d_in))
+        z, s = orc.recall_head(None, x.astype(np.float64), head["W1"], head["b1"], head["w2"], head["b2"])
+        srt = np.sort(s)
+        tau = float(0.5 * (srt[B // 2 - 1] + srt[B // 2]))
+        xd = torch.from_numpy(x).cuda()
+        ranks = []
+        for r in range(world):   # each rank's share of W1 x: its columns only (fp64 product rounded to fp32)
+            share = (xd[:, r * cols:(r + 1) * cols].double() @ hd["W1"][:, r * cols:(r + 1) * cols].double().T).float()
+            ranks.append(dict(pre_local=share.contiguous(), scores=torch.zeros(B, device="cuda"),
+                              logits=torch.zeros(B, device="cuda"),
+                              flags=torch.full((B,), 7, dtype=torch.uint8, device="cuda"),
+                              counters=torch.zeros((B, 2), dtype=torch.int32, device="cuda")))
+        ctx.recall_finalize_exchange(B, world, 0, ranks, recv, arrived, step + 1, hd["b1"], hd["w2"], hd["b2"], tau)
+        torch.cuda.synchronize()
+        want = orc.flags(z, s, tau)
+        decided = np.abs(s - tau) >= gh.FLAG_BAND
+        for r in range(world):
+            np.testing.assert_allclose(ranks[r]["scores"].cpu().numpy(), s, rtol=0, atol=gh.ATOL_SCORE)
+            np.testing.assert_array_equal(ranks[r]["flags"].cpu().numpy()[decided], want[decided])
+            assert torch.equal(ranks[r]["logits"], ranks[0]["logits"])       # bit for bit on every rank
+            assert torch.equal(ranks[r]["flags"], ranks[0]["flags"])
+            assert (ranks[r]["counters"][:, 0] == 1).all()
+            assert (arrived[r] == step + 1).all()
+    assert ctx.read_device_status() == 0
+
+
+def test_fused_exchange_wait_runs_out_when_a_rank_never_arrives():
+    """Three of four ranks make the call; the fourth never does.  Their waits end after the given
+    limit, the status word says so, and the outputs are left alone (no trap, no hang)."""
+    world, B, d_h = 4, 3, 16
+    ctx = gh.make_ctx(make_problem(1, 1, B, 2, 2, 64, [20] * B), [8], [0], [1], head=(0, 1, d_h))
+    recv, arrived = _exchange_setup(world, B, d_h)
+    w = torch.zeros(d_h, device="cuda")
+    one = torch.zeros(1, device="cuda")
+    ranks = [dict(pre_local=torch.zeros((B, d_h), device="cuda"), scores=torch.full((B,), -1.0, device="cuda"),
+                  flags=torch.full((B,), 9, dtype=torch.uint8, device="cuda")) for _ in range(3)]
+    ctx.recall_finalize_exchange(B, world, 0, ranks, recv, arrived, 1, w, w, one, 0.5, timeout_ns=2_000_000)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() & 4
+    for r in ranks:
+        assert (r["scores"] == -1.0).all() and (r["flags"] == 9).all()
+    assert ctx.read_device_status() == 0          # reading the word clears it
+
+
+def test_tp_step_fused_on_one_rank_equals_the_fused_single_gpu_step():
+    """world = 1: the step with the exchange kernel (a rank that only exchanges with itself) against
+    the library's own single-GPU step, bit for bit on the attention outputs."""
+    L, B, Hq, Hkv, D, d_ext, d_h = 2, 3, 8, 2, 128, 8, 24
+    windows, sinks, gated = [64, 32], [4, 0], [1, 1]
+    prob = make_problem(93, L, B, Hq, Hkv, D, [300, 40, 1000])
+    head = dict(W1=synth.gauss_f32_tensor(9, synth.STREAM_W1, (d_h, d_ext + Hq * D), std=0.05),
+                b1=synth.gauss_f32_tensor(9, synth.STREAM_B1, (d_h,), std=0.05),
+                w2=synth.gauss_f32_tensor(9, synth.STREAM_W2, (d_h,), std=0.3),
+                b2=synth.gauss_f32_tensor(9, synth.STREAM_B2, (1,), std=0.05), use_attn_out=1)
+    hd = gh.head_to_device(head)
+    fe = torch.from_numpy(synth.gauss_f32_tensor(9, synth.STREAM_FEAT, (B, d_ext))).cuda()
+    ctx = gh.make_ctx(prob, windows, sinks, gated, head=(d_ext, 1, d_h))
+    dev = gh.upload(prob)
+    out0, lse0 = gh.new_out(prob)
+    sc0 = torch.zeros(B, device="cuda")
+    fl0 = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    ctx.step(ctx.step_args(B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out0, sc0, fl0,
+                           feat_ext=fe, head=hd, threshold=0.5, lse=lse0))
+    sh = tp.head_shard(0, 1, Hq, Hkv, D, d_ext, True)
+    bufs = tp.ExchangeBuffers.local(1, B, d_h)
+    out1, lse1 = gh.new_out(prob)
+    sc1 = torch.zeros(B, device="cuda")
+    fl1 = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    pre = torch.zeros((B, d_h), device="cuda")
+    for _ in range(2):   # two steps: epochs 1 and 2
+        tp.tp_step_fused(ctx, sh, B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out1, W1=hd["W1"],
+                         b1=hd["b1"], w2=hd["w2"], b2=hd["b2"], threshold=0.5, pre=pre, scores=sc1, flags=fl1,
+                         buffers=bufs, feat_ext=fe, lse=lse1)
+    torch.cuda.synchronize()
+    assert bufs.epoch == 2
+    assert torch.equal(fl1, fl0) and torch.equal(out1, out0) and torch.equal(lse1, lse0)
+    np.testing.assert_allclose(sc1.cpu().numpy(), sc0.cpu().numpy(), rtol=0, atol=1e-6)
+    assert ctx.read_device_status() == 0
