@@ -238,6 +238,32 @@ oda_status_t oda_merge_partials(oda_ctx_t* ctx, int32_t n_parts, int32_t layer_b
                                 void* stream);
 
 /*
+ * oda_merge_partials with the exchange inside the kernel, by the protocol of
+ * oda_recall_finalize_exchange: the rows are cut into 64 blocks; CTA c of every rank stores its
+ * rows of block c (the rank's part_out / part_lse, lse = -inf where tokens_local[b] = 0) into slot
+ * [rank] of every rank's receive buffers, raises flag [rank][c] carrying `epoch` in every rank's
+ * flag array, waits -- at most timeout_ns (0 => 1 s) -- for the other ranks' flag c in its own
+ * array, and combines block c in rank order into out / lse.
+ *   recv_out [world]: rank r's buffer of 2 * world * L * batch * q_heads * head_dim floats;
+ *   recv_lse [world]: 2 * world * L * batch * q_heads floats;  arrived [world]: world * 64 u32, zero
+ *   at set-up; all mapped into this GPU's address space; epoch and n_local as above.
+ * flags (per rank, nullable = all requests) must hold the same values on every rank.
+ */
+typedef struct {
+    const float* part_out;       /* [L, batch, q_heads, head_dim] fp32: this rank's oda_full_decode_gated output */
+    const float* part_lse;       /* [L, batch, q_heads] */
+    const int32_t* tokens_local; /* [batch] positions this rank holds (NULL: some of every request) */
+    const uint8_t* flags;        /* [batch] gate (NULL: all requests) */
+    void* out;                   /* [L, batch, q_heads, head_dim] fp32 */
+    float* lse;                  /* nullable */
+} oda_merge_exchange_rank_t;
+oda_status_t oda_merge_partials_exchange(oda_ctx_t* ctx, int32_t world, int32_t rank_base, int32_t n_local,
+                                         const oda_merge_exchange_rank_t* ranks, float* const* recv_out,
+                                         float* const* recv_lse, uint32_t* const* arrived, uint32_t epoch,
+                                         uint64_t timeout_ns, int32_t layer_begin, int32_t layer_end,
+                                         int32_t batch, void* stream);
+
+/*
  * The paper's own recall head (appendix "Recall-head architecture"; Eq. 2): three
  * RMSNorm -> Linear(d_model -> d_tower) -> SiLU towers over (h_{t-1}, E(x_t), h_t^L), the interaction
  * vector u = [a;b;c;a.b;|a-b|;a.c;|a-c|;b.c;|b-c|], z0 = (a+b+c+SiLU(W_f u + b_f))/2, n_blocks

@@ -26,7 +26,7 @@ EXPORTS = [
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
     "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
-    "oda_recall_finalize_exchange",
+    "oda_recall_finalize_exchange", "oda_merge_partials_exchange",
 ]
 
 
@@ -61,6 +61,11 @@ class _FullHead(ctypes.Structure):
 class _ExchangeRank(ctypes.Structure):
     _fields_ = [("pre_local", ctypes.c_void_p), ("scores", ctypes.c_void_p), ("logits", ctypes.c_void_p),
                 ("flags", ctypes.c_void_p), ("counters", ctypes.c_void_p)]
+
+
+class _MergeExchangeRank(ctypes.Structure):
+    _fields_ = [("part_out", ctypes.c_void_p), ("part_lse", ctypes.c_void_p), ("tokens_local", ctypes.c_void_p),
+                ("flags", ctypes.c_void_p), ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p)]
 
 
 class _StepArgs(ctypes.Structure):
@@ -112,6 +117,9 @@ def load_library():
         lib.oda_recall_finalize_exchange.argtypes = [vp, i32, i32, i32, i32, ctypes.POINTER(_ExchangeRank), vp, vp,
                                                      ctypes.c_uint32, ctypes.c_uint64, vp, vp, vp, f32, vp, vp]
         lib.oda_recall_finalize_exchange.restype = i32
+        lib.oda_merge_partials_exchange.argtypes = [vp, i32, i32, i32, ctypes.POINTER(_MergeExchangeRank), vp, vp, vp,
+                                                    ctypes.c_uint32, ctypes.c_uint64, i32, i32, i32, vp]
+        lib.oda_merge_partials_exchange.restype = i32
         lib.oda_full_decode_gated.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
         lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
@@ -311,6 +319,19 @@ class OdaContext:
             ctypes.cast(arr_p, ctypes.c_void_p), int(epoch), int(timeout_ns), _ptr(b1), _ptr(w2), _ptr(b2),
             float(threshold), _ptr(override_flags), _stream() if stream is None else stream),
             "oda_recall_finalize_exchange")
+
+    def merge_partials_exchange(self, world, rank_base, ranks, recv_out, recv_lse, arrived, epoch, layer_begin,
+                                layer_end, batch, timeout_ns=0, stream=None):
+        """ranks: list of dicts(part_out, part_lse, out[, tokens_local, flags, lse]) for the ranks this launch runs."""
+        n_local = len(ranks)
+        arr = (_MergeExchangeRank * n_local)(*[
+            _MergeExchangeRank(_ptr(r["part_out"]), _ptr(r["part_lse"]), _ptr(r.get("tokens_local")),
+                               _ptr(r.get("flags")), _ptr(r["out"]), _ptr(r.get("lse"))) for r in ranks])
+        tabs = [(ctypes.c_void_p * world)(*[_ptr(t) for t in tab]) for tab in (recv_out, recv_lse, arrived)]
+        self._check(self.lib.oda_merge_partials_exchange(
+            self._h, world, rank_base, n_local, arr, *[ctypes.cast(t, ctypes.c_void_p) for t in tabs], int(epoch),
+            int(timeout_ns), layer_begin, layer_end, batch, _stream() if stream is None else stream),
+            "oda_merge_partials_exchange")
 
     def full_decode_gated(self, layer_begin, layer_end, batch, q_full, k_cache, v_cache, block_table,
                           seq_lens, flags, out, lse=None, stream=None):

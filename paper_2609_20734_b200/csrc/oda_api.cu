@@ -611,6 +611,56 @@ oda_status_t oda_recall_finalize_exchange(oda_ctx_t* c, int32_t batch, int32_t w
     return ODA_OK;
 }
 
+oda_status_t oda_merge_partials_exchange(oda_ctx_t* c, int32_t world, int32_t rank_base, int32_t n_local,
+                                         const oda_merge_exchange_rank_t* ranks, float* const* recv_out,
+                                         float* const* recv_lse, uint32_t* const* arrived, uint32_t epoch,
+                                         uint64_t timeout_ns, int32_t lb, int32_t le, int32_t batch, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (!c->ws) return fail(c, ODA_ERR_WORKSPACE, "oda_set_workspace has not been called");
+    const oda_config_t& f = c->cfg;
+    if (world < 1 || world > kExchangeMaxWorld) return fail(c, ODA_ERR_UNSUPPORTED, "world outside [1, 8]");
+    if (n_local < 1 || rank_base < 0 || rank_base + n_local > world) return fail(c, ODA_ERR_INVALID_ARG, "ranks of this launch outside [0, world)");
+    if (lb < 0 || le > f.num_layers || lb > le) return fail(c, ODA_ERR_INVALID_ARG, "bad layer range");
+    if (batch < 0 || batch > f.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0 || lb == le) return ODA_OK;
+    if (f.out_dtype != 0) return fail(c, ODA_ERR_UNSUPPORTED, "parts are merged in fp32: create the context with out_dtype 0");
+    if (epoch == 0) return fail(c, ODA_ERR_INVALID_ARG, "epoch starts at 1 (the flag arrays start at 0)");
+    if (!ranks || !recv_out || !recv_lse || !arrived) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    MergeExchangeParams p;
+    std::memset(&p, 0, sizeof p);
+    for (int i = 0; i < n_local; ++i) {
+        if (!ranks[i].part_out || !ranks[i].part_lse || !ranks[i].out) return fail(c, ODA_ERR_INVALID_ARG, "null rank buffer");
+        p.ranks[i].part_out = ranks[i].part_out;
+        p.ranks[i].part_lse = ranks[i].part_lse;
+        p.ranks[i].tokens_local = ranks[i].tokens_local;
+        p.ranks[i].flags = ranks[i].flags;
+        p.ranks[i].out = static_cast<float*>(ranks[i].out);
+        p.ranks[i].lse = ranks[i].lse;
+    }
+    for (int r = 0; r < world; ++r) {
+        if (!recv_out[r] || !recv_lse[r] || !arrived[r]) return fail(c, ODA_ERR_INVALID_ARG, "null receive buffer or flag array");
+        p.recv_out[r] = recv_out[r];
+        p.recv_lse[r] = recv_lse[r];
+        p.arrived[r] = arrived[r];
+    }
+    p.layers = reinterpret_cast<const LayerInfo*>(c->ws + c->lay.layers);
+    p.status = reinterpret_cast<int32_t*>(c->ws + c->lay.status);
+    p.timeout_ns = timeout_ns ? timeout_ns : 1000000000ull;
+    p.batch = batch;
+    p.q_heads = f.num_q_heads;
+    p.num_layers = f.num_layers;
+    p.layer_begin = lb;
+    p.layer_end = le;
+    p.world = world;
+    p.rank_base = rank_base;
+    p.epoch = epoch;
+    cudaError_t e = launch_merge_exchange(p, n_local, f.head_dim, static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "partial exchange + merge launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
 oda_status_t oda_write_current_kv(oda_ctx_t* c, int32_t batch, const void* k_cur, const void* v_cur,
                                   const uint8_t* mask, void* k_cache, void* v_cache, const int32_t* bt,
                                   const int32_t* sl, void* stream)

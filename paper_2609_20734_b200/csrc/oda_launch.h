@@ -100,6 +100,29 @@ struct ExchangeParams {
 };
 cudaError_t launch_recall_exchange(const ExchangeParams& p, int n_local, cudaStream_t st, bool pdl = false);
 
+// sequence-sharded Full pass: exchange of (out, lse) rows fused with their combination
+constexpr int kMergeBlocks = 64;           // row blocks, each with its own arrival flag
+struct MergeExchangeRank {
+    const float* part_out;       // [L, batch, q_heads, D] this rank's rows
+    const float* part_lse;       // [L, batch, q_heads]
+    const int32_t* tokens_local; // [batch] positions this rank holds (nullable: all > 0)
+    const uint8_t* flags;        // [batch] gate (nullable: all requests)
+    float* out;
+    float* lse;                  // nullable
+};
+struct MergeExchangeParams {
+    MergeExchangeRank ranks[kExchangeMaxWorld];
+    float* recv_out[kExchangeMaxWorld];    // rank r's buffer [2][world][L*batch*q_heads][D]
+    float* recv_lse[kExchangeMaxWorld];    // [2][world][L*batch*q_heads]
+    uint32_t* arrived[kExchangeMaxWorld];  // [world][kMergeBlocks]
+    const LayerInfo* layers;
+    int32_t* status;
+    unsigned long long timeout_ns;
+    int32_t batch, q_heads, num_layers, layer_begin, layer_end, world, rank_base;
+    uint32_t epoch;
+};
+cudaError_t launch_merge_exchange(const MergeExchangeParams& p, int n_local, int head_dim, cudaStream_t st, bool pdl = false);
+
 int recall_head_grid(int d_hidden);
 int recall_head_ksplits(int d_in);
 cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl = false);

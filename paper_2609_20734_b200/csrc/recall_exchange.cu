@@ -20,6 +20,7 @@
 // returns.
 #include "launch_ex.cuh"
 #include "mbar.cuh"
+#include "oda_device.cuh"
 #include "oda_launch.h"
 
 namespace oda {
@@ -125,6 +126,137 @@ cudaError_t launch_recall_exchange(const ExchangeParams& p, int n_local, cudaStr
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, recall_exchange_kernel, p);
+}
+
+}  // namespace oda
+
+// ---------------------------------------------------------------------------------------------------
+// Sequence-sharded Full pass: the exchange of the per-rank (out, lse) rows fused with their
+// log-sum-exp combination, by the same protocol.  The rows are cut into kMergeBlocks blocks; CTA c
+// of every rank pushes its rows of block c into every rank's receive buffer, raises flag
+// [rank][c] everywhere, waits for the other ranks' flag c in its own array and combines block c in
+// rank order -- so blocks flow independently and no CTA waits for rows it does not need.
+namespace oda {
+
+template <int V>
+__global__ void __launch_bounds__(kExchangeThreads) merge_exchange_kernel(const __grid_constant__ MergeExchangeParams p)
+{
+    __shared__ int s_ok;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    constexpr int D = V * 32;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c = blockIdx.x, slot = blockIdx.y;
+    const int rank = p.rank_base + slot;
+    const MergeExchangeRank& me = p.ranks[slot];
+    const long long all_rows = (long long)p.num_layers * p.batch * p.q_heads;   // rows of a whole [L,B,Hq] array
+    const long long rows = (long long)(p.layer_end - p.layer_begin) * p.batch * p.q_heads;
+    const long long r0 = rows * c / kMergeBlocks, r1 = rows * (c + 1) / kMergeBlocks;
+    const size_t par = (size_t)(p.epoch & 1u) * p.world;
+    auto row_of = [&](long long w, int& b, bool& live) {
+        const int h = (int)(w % p.q_heads);
+        b = (int)((w / p.q_heads) % p.batch);
+        const int l = p.layer_begin + (int)(w / ((long long)p.q_heads * p.batch));
+        live = p.layers[l].gated && (!me.flags || me.flags[b]);
+        return ((long long)l * p.batch + b) * p.q_heads + h;
+    };
+    // 1. this rank's rows of block c -> slot [rank] of every rank's receive buffers
+    for (long long w = r0 + warp; w < r1; w += kExchangeThreads / 32) {
+        int b;
+        bool live;
+        const long long row = row_of(w, b, live);
+        if (!live) continue;
+        const float lr = (!me.tokens_local || me.tokens_local[b] > 0) ? me.part_lse[row] : -INFINITY;
+        float v[V];
+        if (lr != -INFINITY) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) v[e] = me.part_out[row * D + lane * V + e];
+        }
+        for (int peer = 0; peer < p.world; ++peer) {
+            const size_t base = (par + rank) * (size_t)all_rows + (size_t)row;
+            if (lane == 0) p.recv_lse[peer][base] = lr;
+            if (lr != -INFINITY) {
+                float* dst = p.recv_out[peer] + base * D + lane * V;
+#pragma unroll
+                for (int e = 0; e < V; ++e) dst[e] = v[e];
+            }
+        }
+    }
+    // 2. visible everywhere, then flag [rank][c] in every rank's array
+    __threadfence_system();
+    __syncthreads();
+    if (tid < p.world) st_release_sys(p.arrived[tid] + (size_t)rank * kMergeBlocks + c, p.epoch);
+    // 3. bounded wait for the other ranks' block c
+    if (tid == 0) s_ok = 1;
+    __syncthreads();
+    if (tid < p.world) {
+        const uint32_t* f = p.arrived[rank] + (size_t)tid * kMergeBlocks + c;
+        const uint64_t t0 = globaltimer_ns();
+        uint32_t spins = 0;
+        while (ld_acquire_sys(f) != p.epoch) {
+            if ((++spins & 63u) == 0 && globaltimer_ns() - t0 > p.timeout_ns) {
+                s_ok = 0;
+                break;
+            }
+        }
+    }
+    __syncthreads();
+    if (!s_ok) {
+        if (tid == 0 && p.status) atomicOr(p.status, kStatusWaitTimeout);
+        return;
+    }
+    // 4. log-sum-exp combination of block c, parts in rank order
+    const float* my_lse = p.recv_lse[rank];
+    const float* my_out = p.recv_out[rank];
+    for (long long w = r0 + warp; w < r1; w += kExchangeThreads / 32) {
+        int b;
+        bool live;
+        const long long row = row_of(w, b, live);
+        if (!live) continue;
+        float m = -INFINITY;
+        for (int r = 0; r < p.world; ++r) m = fmaxf(m, __ldcg(my_lse + (par + r) * (size_t)all_rows + row));
+        float acc[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+        float sum = 0.f;
+        if (m > -INFINITY) {
+            for (int r = 0; r < p.world; ++r) {
+                const size_t base = (par + r) * (size_t)all_rows + row;
+                const float lr = __ldcg(my_lse + base);
+                if (lr == -INFINITY) continue;
+                const float wgt = expf(lr - m);
+                sum += wgt;
+                const float* src = my_out + base * D + lane * V;
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = fmaf(wgt, __ldcg(src + e), acc[e]);
+            }
+        }
+        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        float* dst = me.out + row * D + lane * V;
+#pragma unroll
+        for (int e = 0; e < V; ++e) dst[e] = acc[e] * inv;
+        if (me.lse && lane == 0) me.lse[row] = sum > 0.f ? m + logf(sum) : -INFINITY;
+    }
+}
+
+cudaError_t launch_merge_exchange(const MergeExchangeParams& p, int n_local, int head_dim, cudaStream_t st, bool pdl)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kMergeBlocks, n_local);
+    cfg.blockDim = dim3(kExchangeThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (n_local > 1) {   // ranks sharing one GPU wait on one another: all CTAs must be resident
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (n_local > 1 || pdl) ? 1 : 0;
+    if (head_dim == 128) return cudaLaunchKernelEx(&cfg, merge_exchange_kernel<4>, p);
+    return cudaLaunchKernelEx(&cfg, merge_exchange_kernel<2>, p);
 }
 
 }  // namespace oda

@@ -191,3 +191,58 @@ def tp_step_fused(ctx, shard: HeadShard, batch, q_local, k_cache, v_cache, block
     ctx.full_decode_gated(0, ctx.cfg.num_layers, batch, q_local if q_full is None else q_full, k_cache, v_cache,
                           block_table, seq_lens, flags, out, lse)
     return flags
+
+
+# ---- the sequence-sharded Full pass with the exchange inside the merge kernel ------------------
+MERGE_BLOCKS = 64    # row blocks (and arrival flags per rank) of the fused exchange + merge
+
+
+class MergeExchangeBuffers(ExchangeBuffers):
+    """Receive buffers (partial rows and their log-sum-exps, two parities) and per-block arrival
+    flags of every rank, in rank order; entries as in ExchangeBuffers."""
+
+    def __init__(self, recv_out, recv_lse, arrived, keep=None):
+        self.recv_out, self.recv_lse, self.arrived, self.keep, self.epoch = recv_out, recv_lse, arrived, keep, 0
+
+    @classmethod
+    def local(cls, world, num_layers, batch, q_heads, head_dim, device="cuda"):
+        import torch
+
+        rows = num_layers * batch * q_heads
+        return cls([torch.zeros((2, world, rows, head_dim), device=device) for _ in range(world)],
+                   [torch.zeros((2, world, rows), device=device) for _ in range(world)],
+                   [torch.zeros((world, MERGE_BLOCKS), dtype=torch.int32, device=device) for _ in range(world)])
+
+    @classmethod
+    def symmetric(cls, group, num_layers, batch, q_heads, head_dim, device="cuda"):
+        """One rank per process and GPU (torch's symmetric memory; plain peer stores only).  Not
+        tested on a GPU: this build had one."""
+        import torch
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm
+
+        world = dist.get_world_size(group)
+        rows = num_layers * batch * q_heads
+        bufs = [symm.empty((2, world, rows, head_dim), dtype=torch.float32, device=device),
+                symm.empty((2, world, rows), dtype=torch.float32, device=device),
+                symm.empty((world, MERGE_BLOCKS), dtype=torch.int32, device=device)]
+        for t in bufs:
+            t.zero_()
+        hs = [symm.rendezvous(t, group) for t in bufs]
+        dist.barrier(group)
+        return cls(*[[int(p) for p in h.buffer_ptrs] for h in hs], keep=(bufs, hs))
+
+
+def sp_full_step_fused(ctx, world, rank, batch, q_full, k_cache, v_cache, block_table_local, seq_lens_local, flags,
+                       part_out, part_lse, out, lse=None, *, buffers: MergeExchangeBuffers, timeout_ns=0):
+    """sp_full_step without a collective call: two launches, the gated Full pass over this rank's
+    positions and the kernel that pushes its partial rows to the peers, waits for theirs block by
+    block and merges.  seq_lens_local doubles as this rank's token counts."""
+    L = ctx.cfg.num_layers
+    ctx.full_decode_gated(0, L, batch, q_full, k_cache, v_cache, block_table_local, seq_lens_local, flags,
+                          part_out, part_lse)
+    ctx.merge_partials_exchange(world, rank, [dict(part_out=part_out, part_lse=part_lse, tokens_local=seq_lens_local,
+                                                   flags=flags, out=out, lse=lse)],
+                                buffers.recv_out, buffers.recv_lse, buffers.arrived, buffers.next_epoch(), 0, L, batch,
+                                timeout_ns=timeout_ns)
+

@@ -323,3 +323,138 @@ def test_tp_step_fused_on_one_rank_equals_the_fused_single_gpu_step():
     assert torch.equal(fl1, fl0) and torch.equal(out1, out0) and torch.equal(lse1, lse0)
     np.testing.assert_allclose(sc1.cpu().numpy(), sc0.cpu().numpy(), rtol=0, atol=1e-6)
     assert ctx.read_device_status() == 0
+
+
+def _sp_problem(world, seed=41):
+    L, B, Hq, Hkv, D = 3, 6, 8, 2, 128
+    windows, sinks, gated = [64, 32, 64], [4, 0, 4], [1, 0, 1]
+    seq = [100, 900, 5, 2500, 64, 17]
+    prob = make_problem(seed, L, B, Hq, Hkv, D, seq)
+    lay = prob["layout"]
+    cfg = dict(num_layers=L, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=B,
+               max_blocks_per_seq=prob["table"].shape[1], layer_window=windows, layer_sinks=sinks,
+               layer_gated=gated, kv_layer_stride=lay.layer_stride, kv_block_stride=lay.block_stride,
+               kv_token_stride=lay.token_stride, kv_head_stride=lay.head_stride, allow_empty=1)
+    from paper_2609_20734_b200 import binding
+    ctx = binding.OdaContext(binding.OdaConfig(**cfg))
+    width = prob["table"].shape[1]
+    tables, tokens = [], np.zeros((world, B), np.int32)
+    for r in range(world):
+        table_r = np.zeros((B, width), np.int32)
+        for b, t in enumerate(seq):
+            lo, hi, held = tp.sequence_shard(r, world, t)
+            table_r[b, :hi - lo] = prob["table"][b, lo:hi]
+            tokens[r, b] = held
+        tables.append(torch.from_numpy(table_r).cuda())
+    return ctx, prob, (windows, sinks, gated), tables, tokens
+
+
+@pytest.mark.parametrize("world", [1, 2, 4, 8])
+def test_fused_merge_exchange_matches_oracle_on_every_rank(world):
+    """Sequence-sharded Full pass whose exchange runs inside the merge kernel.  The ranks are the
+    CTA columns of one cooperative launch (kernels that wait on one another never run as separate
+    launches on one GPU).  Three exchanges in a row with different flags: every rank ends with the
+    oracle's whole-history rows, bit-identical across ranks; unflagged rows stay untouched."""
+    ctx, prob, (windows, sinks, gated), tables, tokens = _sp_problem(world)
+    L, B, Hq, D = prob["q"].shape
+    dev = gh.upload(prob)
+    bufs = tp.MergeExchangeBuffers.local(world, L, B, Hq, D)
+    for step, flags_h in enumerate([np.array([1, 1, 1, 1, 0, 1], np.uint8), np.array([0, 1, 0, 0, 1, 0], np.uint8),
+                                    np.ones(6, np.uint8)]):
+        want, want_lse = orc.attention("full", prob["q"], prob["k"], prob["v"], prob["table"], prob["seq_lens"],
+                                       num_kv_heads=2, block_size=16,
+                                       layout=prob["layout"], layer_window=windows, layer_sinks=sinks,
+                                       request_mask=flags_h, nthreads=4)
+        flags = torch.from_numpy(flags_h).cuda()
+        ranks = []
+        for r in range(world):
+            po = torch.full((L, B, Hq, D), float("nan"), device="cuda")
+            pl = torch.full((L, B, Hq), float("nan"), device="cuda")
+            tok = torch.from_numpy(tokens[r]).cuda()
+            ctx.full_decode_gated(0, L, B, dev["q"], dev["k"], dev["v"], tables[r], tok, flags, po, pl)
+            ranks.append(dict(part_out=po, part_lse=pl, tokens_local=tok, flags=flags,
+                              out=torch.full((L, B, Hq, D), 7.0, device="cuda"),
+                              lse=torch.full((L, B, Hq), 7.0, device="cuda")))
+        ctx.merge_partials_exchange(world, 0, ranks, bufs.recv_out, bufs.recv_lse, bufs.arrived, bufs.next_epoch(),
+                                    0, L, B, timeout_ns=2_000_000_000)
+        torch.cuda.synchronize()
+        assert ctx.read_device_status() == 0
+        o0, l0 = ranks[0]["out"].cpu().numpy(), ranks[0]["lse"].cpu().numpy()
+        for r in range(1, world):
+            np.testing.assert_array_equal(ranks[r]["out"].cpu().numpy(), o0)
+            np.testing.assert_array_equal(ranks[r]["lse"].cpu().numpy(), l0)
+        for l in range(L):
+            for b in range(B):
+                if gated[l] and flags_h[b]:
+                    gh.assert_close(o0[l, b], want[l, b], gh.ATOL_OUT, f"step {step} layer {l} request {b} out")
+                    gh.assert_close(l0[l, b], want_lse[l, b], gh.ATOL_LSE, f"step {step} layer {l} request {b} lse")
+                else:
+                    assert (o0[l, b] == 7.0).all() and (l0[l, b] == 7.0).all()
+        for r in range(world):
+            assert (bufs.arrived[r] == step + 1).all()
+
+
+def test_fused_merge_exchange_equals_the_gathered_merge():
+    """Same partial rows through the gathered merge and through the exchange kernel: same bits
+    (both combine the parts in rank order with the same arithmetic)."""
+    world = 4
+    ctx, prob, _, tables, tokens = _sp_problem(world, seed=43)
+    L, B, Hq, D = prob["q"].shape
+    dev = gh.upload(prob)
+    flags = torch.ones(B, dtype=torch.uint8, device="cuda")
+    parts_out = torch.zeros((world, L, B, Hq, D), device="cuda")
+    parts_lse = torch.zeros((world, L, B, Hq), device="cuda")
+    toks = [torch.from_numpy(tokens[r]).cuda() for r in range(world)]
+    for r in range(world):
+        ctx.full_decode_gated(0, L, B, dev["q"], dev["k"], dev["v"], tables[r], toks[r], flags, parts_out[r], parts_lse[r])
+    out_a = torch.zeros((L, B, Hq, D), device="cuda")
+    lse_a = torch.zeros((L, B, Hq), device="cuda")
+    ctx.merge_partials(world, 0, L, B, parts_out, parts_lse, flags, out_a, lse_a, part_tokens=torch.from_numpy(tokens).cuda())
+    bufs = tp.MergeExchangeBuffers.local(world, L, B, Hq, D)
+    ranks = [dict(part_out=parts_out[r], part_lse=parts_lse[r], tokens_local=toks[r], flags=flags,
+                  out=torch.zeros((L, B, Hq, D), device="cuda"), lse=torch.zeros((L, B, Hq), device="cuda"))
+             for r in range(world)]
+    ctx.merge_partials_exchange(world, 0, ranks, bufs.recv_out, bufs.recv_lse, bufs.arrived, bufs.next_epoch(), 0, L, B)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() == 0
+    np.testing.assert_array_equal(ranks[2]["out"].cpu().numpy(), out_a.cpu().numpy())
+    np.testing.assert_array_equal(ranks[2]["lse"].cpu().numpy(), lse_a.cpu().numpy())
+
+
+def test_fused_merge_exchange_wait_runs_out_when_a_rank_never_arrives():
+    """One of two ranks makes the call.  Its wait ends at the limit, the status word says so, the
+    output stays as it was."""
+    world = 2
+    ctx, prob, _, tables, tokens = _sp_problem(world)
+    L, B, Hq, D = prob["q"].shape
+    bufs = tp.MergeExchangeBuffers.local(world, L, B, Hq, D)
+    rank0 = dict(part_out=torch.zeros((L, B, Hq, D), device="cuda"), part_lse=torch.zeros((L, B, Hq), device="cuda"),
+                 out=torch.full((L, B, Hq, D), 7.0, device="cuda"), lse=torch.full((L, B, Hq), 7.0, device="cuda"))
+    ctx.merge_partials_exchange(world, 0, [rank0], bufs.recv_out, bufs.recv_lse, bufs.arrived, 1, 0, L, B,
+                                timeout_ns=2_000_000)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() & 4
+    assert (rank0["out"] == 7.0).all() and (rank0["lse"] == 7.0).all()
+
+
+def test_sp_full_step_fused_on_one_rank_equals_the_plain_full_pass():
+    ctx, prob, (windows, sinks, gated), tables, tokens = _sp_problem(1)
+    L, B, Hq, D = prob["q"].shape
+    dev = gh.upload(prob)
+    flags = torch.from_numpy(np.array([1, 0, 1, 1, 0, 1], np.uint8)).cuda()
+    tok = torch.from_numpy(tokens[0]).cuda()
+    ref_out = torch.full((L, B, Hq, D), 7.0, device="cuda")
+    ref_lse = torch.full((L, B, Hq), 7.0, device="cuda")
+    ctx.full_decode_gated(0, L, B, dev["q"], dev["k"], dev["v"], tables[0], tok, flags, ref_out, ref_lse)
+    out = torch.full((L, B, Hq, D), 7.0, device="cuda")
+    lse = torch.full((L, B, Hq), 7.0, device="cuda")
+    bufs = tp.MergeExchangeBuffers.local(1, L, B, Hq, D)
+    for _ in range(2):
+        tp.sp_full_step_fused(ctx, 1, 0, B, dev["q"], dev["k"], dev["v"], tables[0], tok, flags,
+                              torch.zeros((L, B, Hq, D), device="cuda"), torch.zeros((L, B, Hq), device="cuda"),
+                              out, lse, buffers=bufs)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), ref_out.cpu().numpy())
+    np.testing.assert_array_equal(lse.cpu().numpy(), ref_lse.cpu().numpy())
+
