@@ -41,6 +41,7 @@ struct oda_ctx {
     int variant = ODA_VARIANT_SIMT;
     int grid = 148;
     int min_span_pages = 8;
+    int snap_span_pages = 128;  // launches of up to 1 MiB per CTA may be cut at unit boundaries
     bool calibrated = false;  // the per-SM split table in the workspace is valid
     bool calibrating = false; // attention launches record per-SM streaming rates
     double calib_spread = 0.0; // slowest / fastest SM share seen by oda_calibrate
@@ -163,6 +164,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     p.mode = mode;
     p.ncls = c->ncls;
     p.min_span_pages = c->min_span_pages;
+    p.snap_span_pages = c->snap_span_pages;
     p.max_items = c->max_items;
     p.scale_log2e = c->scale * 1.4426950408889634f;
     bool any = false;

@@ -42,6 +42,7 @@ struct AttnParams {
                            //     merged into the Local result that out/lse already hold
     int32_t ncls;
     int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
+    int32_t snap_span_pages; // launches with spans up to this long may be cut at unit boundaries (0: never)
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)
     int32_t cls_window[kMaxClasses], cls_sinks[kMaxClasses], cls_gated[kMaxClasses];
@@ -97,7 +98,8 @@ struct Plan {  // shared memory, one per CTA
     int32_t my_span;                         // the span this CTA streams (-1: none)
     int32_t total_pages;
     int32_t nseg;
-    int32_t pad;
+    int32_t snap;                            // unit-aligned split: this CTA streams axis pages [x0, x1), whole units
+    int32_t x0, x1;
 };
 static_assert(sizeof(Plan) % 8 == 0, "Plan is followed by 8-byte aligned barriers in shared memory");
 
@@ -235,6 +237,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             if (i < nl) pl.lb[i] = (int32_t)(carry + x - own);
             carry += __shfl_sync(0xffffffffu, x, 31);
         }
+        int span = -1, nseg = 0;
         if (lane == 0) {
             if (carry > 0x7fffffffll) {  // beyond the 32-bit page axis: refuse rather than wrap
                 atomicOr(p.status, kStatusItemOverflow);
@@ -246,10 +249,12 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
             long long n = (carry + minS - 1) / minS;
             if (n > g) n = g;
-            pl.nseg = (int32_t)n;
+            nseg = (int)n;
+            pl.nseg = nseg;
             // the weighted split needs every CTA to have real work; small launches stay equal
             pl.weighted = weighted && n == g;
-            int span = (int)blockIdx.x;
+            pl.snap = 0;
+            span = (int)blockIdx.x;
             if (pl.weighted) {
                 span = -1;
                 if (claim_slot < 2) {
@@ -264,7 +269,65 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
                     }
                 }
             }
-            pl.my_span = span >= 0 && span < pl.nseg ? span : -1;
+            if (span >= nseg) span = -1;
+            pl.my_span = span;
+        }
+        // Unit-aligned split.  A short launch whose units (one request's pages of one kv head of
+        // one layer) are about as long as a span is cut at unit boundaries instead: each unit is
+        // streamed by one CTA, which writes the unit's rows itself -- no partials, tickets or
+        // merge at the end, where a launch of a few tens of microseconds notices them.  Some CTAs
+        // get no unit; such a launch is bound by DRAM, not by the number of streaming CTAs.  Not
+        // during calibration (which measures the equal split), and not when units are much
+        // shorter (uneven spans) or much longer (idle CTAs) than a span.
+        span = __shfl_sync(0xffffffffu, span, 0);
+        nseg = __shfl_sync(0xffffffffu, nseg, 0);
+        const int total = (int)__shfl_sync(0xffffffffu, (int)carry, 0);
+        if (p.snap_span_pages > 0 && !p.sm_stats && span >= 0 && nseg == (int)gridDim.x && total > 0 &&
+            total <= p.snap_span_pages * nseg) {
+            int umin = 0x7fffffff, umax = 0;
+            for (int c = 0; c < p.ncls; ++c) {
+                if (p.cls_layers_in_call[c] <= 0) continue;
+                for (int b = lane; b < B; b += 32) {
+                    const int np = pl.pb[c][b + 1] - pl.pb[c][b];
+                    if (np > 0) { umin = min(umin, np); umax = max(umax, np); }
+                }
+            }
+            for (int o = 16; o > 0; o >>= 1) {
+                umin = min(umin, __shfl_xor_sync(0xffffffffu, umin, o));
+                umax = max(umax, __shfl_xor_sync(0xffffffffu, umax, o));
+            }
+            if (4 * umin * nseg >= 3 * total && 2 * umax * nseg <= 3 * total) {  // 3/4 span <= unit <= 3/2 span
+                __syncwarp();  // lb[] was written by other lanes of this warp
+                int x = 0;
+                const int j = span + lane;  // lane 0: where the span starts, lane 1: where it ends
+                if (lane < 2) {
+                    x = j >= nseg ? total : (j * total) / nseg;
+                    if (j > 0 && j < nseg) {  // the nearer end of the unit that holds axis page x
+                        int lo = 0, hi = nl;  // last layer with lb <= x
+                        while (hi - lo > 1) {
+                            const int mid = (lo + hi) >> 1;
+                            if (pl.lb[mid] <= x) lo = mid; else hi = mid;
+                        }
+                        const int c = pl.cls[lo];
+                        const int r = x - pl.lb[lo];
+                        int blo = 0, bhi = B;  // last request with H * pb <= r
+                        while (bhi - blo > 1) {
+                            const int mid = (blo + bhi) >> 1;
+                            if (p.num_kv_heads * pl.pb[c][mid] <= r) blo = mid; else bhi = mid;
+                        }
+                        const int np = pl.pb[c][blo + 1] - pl.pb[c][blo];
+                        const int off = (r - p.num_kv_heads * pl.pb[c][blo]) % np;
+                        x = 2 * off < np ? x - off : x - off + np;
+                    }
+                }
+                const int x0 = __shfl_sync(0xffffffffu, x, 0), x1 = __shfl_sync(0xffffffffu, x, 1);
+                if (lane == 0) {
+                    pl.snap = 1;
+                    pl.x0 = x0;
+                    pl.x1 = x1;
+                    if (x0 >= x1) pl.my_span = -1;  // no unit begins in this span
+                }
+            }
         }
     }
     __syncthreads();
@@ -331,6 +394,11 @@ __device__ __forceinline__ int span_begin(const Plan& pl, int j)
 }
 __device__ __forceinline__ void span_range(const Plan& pl, int j, int& x0, int& x1)
 {
+    if (pl.snap) {  // only ever asked for the CTA's own span
+        x0 = pl.x0;
+        x1 = pl.x1;
+        return;
+    }
     x0 = span_begin(pl, j);
     x1 = span_begin(pl, j + 1);
 }
@@ -399,7 +467,9 @@ __device__ inline int decode_item(const AttnParams& p, const Plan& pl, int j, in
     const int off = r2 - g * np;
     const int unit0 = x - off;                       // axis page where the unit starts
     const int take = min(np - off, x_end - x);
-    const int j0 = span_of_near(pl, unit0, j, -1), j1 = span_of_near(pl, unit0 + np - 1, j, +1);
+    // a unit-aligned span holds whole units: one chunk each
+    const int j0 = pl.snap ? j : span_of_near(pl, unit0, j, -1);
+    const int j1 = pl.snap ? j : span_of_near(pl, unit0 + np - 1, j, +1);
     it.layer = p.layer_begin + lo;
     it.b = blo;
     it.g = g;

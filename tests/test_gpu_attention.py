@@ -259,3 +259,37 @@ def test_layer_and_batch_limits_together(variant):
         gh.make_ctx(dict(prob, L=257), windows + [16], sinks + [0], gated + [1], kv_index=kv_index + [0], variant=variant)
     with pytest.raises(binding.OdaError):
         gh.make_ctx(prob, windows, sinks, gated, kv_index=kv_index, variant=variant, max_batch=129)
+
+
+@pytest.mark.parametrize("layout", ["hnd", "nhd"])
+def test_unit_aligned_split_parity(layout):
+    """A short launch whose (layer, request, kv head) units are about one CTA's share each is cut at
+    unit boundaries: every unit is streamed whole by one CTA and written without partials.  The
+    shape below falls under that rule on the launch grid in use (asserted), with units of 32 and 33
+    pages, a sink page each, and more CTAs than units; so does the Full pass over the same requests
+    (units of 94 and 95 pages)."""
+    L, Hq, Hkv, D = 10, 16, 8, 128
+    seq = [1500, 1504, 1519]        # windows of 33, 32 and 33 pages
+    windows, sinks, gated = [512] * L, [4] * L, [1] * L
+    prob = make_problem(321, L, len(seq), Hq, Hkv, D, seq, layout=layout)
+    ctx = gh.make_ctx(prob, windows, sinks, gated, variant=binding.VARIANT_TMA_MMA)
+    units, pages = L * len(seq) * Hkv, L * Hkv * (33 + 32 + 33)
+    span = pages / ctx.attention_grid
+    assert pages >= 8 * ctx.attention_grid and span <= 128 and 0.75 * span <= 32 and 33 <= 1.5 * span, \
+        f"{units} units of 32-33 pages on {ctx.attention_grid} CTAs: outside the unit-aligned rule"
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8)
+    gh.assert_close(out, ref, gh.ATOL_OUT, "local out")
+    gh.assert_close(lse, rlse, gh.ATOL_LSE, "local lse")
+    again, _ = gh.gpu_local(ctx, prob, dev)
+    np.testing.assert_array_equal(again, out)
+    fo, fl = gh.new_out(prob)
+    ctx.full_decode_gated(0, L, len(seq), dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"],
+                          torch.ones(len(seq), dtype=torch.uint8, device="cuda"), fo, fl)
+    torch.cuda.synchronize()
+    ref, rlse = oracle_attention(prob, "full", windows, sinks, nthreads=8)
+    gh.assert_close(fo.cpu().numpy(), ref, gh.ATOL_OUT, "full out")
+    gh.assert_close(fl.cpu().numpy(), rlse, gh.ATOL_LSE, "full lse")
+    assert ctx.read_device_status() == 0
+
