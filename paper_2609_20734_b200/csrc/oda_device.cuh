@@ -100,6 +100,7 @@ struct Plan {  // shared memory, one per CTA
     int32_t nseg;
     int32_t snap;                            // unit-aligned split: this CTA streams axis pages [x0, x1), whole units
     int32_t x0, x1;
+    int32_t umin[kMaxClasses], umax[kMaxClasses];  // shortest / longest unit of each class (pages; 0 pages not counted)
 };
 static_assert(sizeof(Plan) % 8 == 0, "Plan is followed by 8-byte aligned barriers in shared memory");
 
@@ -201,6 +202,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     const int warp = tid >> 5, lane = tid & 31, nwarps = nth >> 5;
     for (int c = warp; c < p.ncls; c += nwarps) {  // one warp scans one class
         int carry = 0;
+        int umin = 0x7fffffff, umax = 0;
         for (int b0 = 0; b0 < B; b0 += 32) {
             const int b = b0 + lane;
             int np = 0;
@@ -213,6 +215,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
                     np = r.pg1 - r.pg0;
                 }
             }
+            if (np > 0) { umin = min(umin, np); umax = max(umax, np); }
             int x = np;
             for (int o = 1; o < 32; o <<= 1) {
                 int y = __shfl_up_sync(0xffffffffu, x, o);
@@ -221,7 +224,13 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             if (b < B) pl.pb[c][b + 1] = carry + x;
             carry += __shfl_sync(0xffffffffu, x, 31);
         }
-        if (lane == 0) pl.pb[c][0] = 0;
+        umin = __reduce_min_sync(0xffffffffu, umin);
+        umax = __reduce_max_sync(0xffffffffu, umax);
+        if (lane == 0) {
+            pl.pb[c][0] = 0;
+            pl.umin[c] = umin;
+            pl.umax[c] = umax;
+        }
     }
     __syncthreads();
     if (tid < 32) {  // exclusive scan over the layers of the call
@@ -247,8 +256,8 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             pl.total_pages = (int32_t)carry;
             const int g = (int)gridDim.x;
             const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
-            long long n = (carry + minS - 1) / minS;
-            if (n > g) n = g;
+            long long n = g;  // the usual case, without the division
+            if (carry < (long long)g * minS) n = (carry + minS - 1) / minS;
             nseg = (int)n;
             pl.nseg = nseg;
             // the weighted split needs every CTA to have real work; small launches stay equal
@@ -286,15 +295,8 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             total <= p.snap_span_pages * nseg) {
             int umin = 0x7fffffff, umax = 0;
             for (int c = 0; c < p.ncls; ++c) {
-                if (p.cls_layers_in_call[c] <= 0) continue;
-                for (int b = lane; b < B; b += 32) {
-                    const int np = pl.pb[c][b + 1] - pl.pb[c][b];
-                    if (np > 0) { umin = min(umin, np); umax = max(umax, np); }
-                }
-            }
-            for (int o = 16; o > 0; o >>= 1) {
-                umin = min(umin, __shfl_xor_sync(0xffffffffu, umin, o));
-                umax = max(umax, __shfl_xor_sync(0xffffffffu, umax, o));
+                umin = min(umin, pl.umin[c]);
+                umax = max(umax, pl.umax[c]);
             }
             if (4 * umin * nseg >= 3 * total && 2 * umax * nseg <= 3 * total) {  // 3/4 span <= unit <= 3/2 span
                 __syncwarp();  // lb[] was written by other lanes of this warp
