@@ -400,7 +400,10 @@ class OdaContext:
             _ptr(counters), _ptr(k_cur_local), _ptr(v_cur_local), _ptr(k_cur_full), _ptr(v_cur_full),
             _ptr(hidden_local), _ptr(hidden_full), _ptr(hidden_out), row_bytes, fh[0], fh[1], fh[2], fh[3],
             fh[4], fh[5] or 0)
-        args._keep = keep     # the head descriptor must outlive the call
+        # the head descriptor and every buffer whose address is in the block must outlive the call
+        args._keep = (keep, q_local, q_full, k_cache, v_cache, block_table, seq_lens, feat_ext, head, override_flags,
+                      out, lse, scores, logits, flags, counters, k_cur_local, v_cur_local, k_cur_full, v_cur_full,
+                      hidden_local, hidden_full, hidden_out, full_head)
         return args
 
     def step(self, args: _StepArgs, stream=None):

@@ -207,6 +207,46 @@ def test_step_forms_agree_eager_host_graph():
     assert ctx.read_device_status() == 0
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_step_without_a_head(pinned):
+    """Head-less stack, forced flags, host buffers pinned or pageable: the host-buffer entry point
+    gives the bits of the device-pointer one (which is checked against the oracle), twice in a row."""
+    from tests.helpers import make_problem
+    L, Hq, Hkv, D = 3, 8, 2, 128
+    seq = [700, 33, 1, 2100, 257]
+    B = len(seq)
+    windows, sinks, gated = [64, 32, 64], [4, 0, 4], [1, 0, 1]
+    prob = make_problem(77, L, B, Hq, Hkv, D, seq)
+    ctx = gh.make_ctx(prob, windows, sinks, gated)
+    dev = gh.upload(prob)
+    ov_h = np.array([1, 0, 1, 1, 0], np.uint8)
+    out, lse = gh.new_out(prob)
+    scores = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    ctx.step(ctx.step_args(B, dev["q"], dev["k"], dev["v"], dev["table"], dev["seq_lens"], out, scores, flags,
+                           override_flags=torch.from_numpy(ov_h).cuda(), lse=lse))
+    torch.cuda.synchronize()
+    ref = orc.step(prob["q"], None, prob["k"], prob["v"], prob["table"], prob["seq_lens"], num_kv_heads=Hkv,
+                   block_size=16, layout=prob["layout"], layer_window=windows, layer_sinks=sinks, layer_gated=gated,
+                   override_flags=ov_h, nthreads=4)
+    gh.assert_close(out.cpu().numpy(), ref.out, gh.ATOL_OUT, "eager out")
+
+    place = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    q_h = place(dev["q"].cpu())
+    out_h = place(torch.full((L, B, Hq, D), 9.0))
+    lse_h = place(torch.full((L, B, Hq), 9.0))
+    sc_h, fl_h = place(torch.zeros(B)), place(torch.zeros(B, dtype=torch.uint8))
+    ov_p = place(torch.from_numpy(ov_h.copy()))     # the argument block holds addresses, not references
+    args = ctx.step_args(B, q_h, dev["k"], dev["v"], dev["table"], dev["seq_lens"], out_h, sc_h, fl_h,
+                         override_flags=ov_p, lse=lse_h)
+    for _ in range(2):
+        up, down = ctx.step_host(args)
+        assert up == q_h.numel() * 2 + B and down == out_h.numel() * 4 + lse_h.numel() * 4 + B * 4 + B
+        assert torch.equal(out_h, out.cpu()) and torch.equal(lse_h, lse.cpu())
+        np.testing.assert_array_equal(fl_h.numpy(), ov_h)
+    assert ctx.read_device_status() == 0
+
+
 def test_step_flag_invariants_on_device():
     wl = _small_batched()
     st = workloads.materialize(wl)
