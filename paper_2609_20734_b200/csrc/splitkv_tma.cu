@@ -123,33 +123,38 @@ __device__ __forceinline__ void consumer_sync()
 // ------------------------------------------------------------------ tile sequence of an item
 // Both the producer and the consumers walk the same sequence: sink pages first (the item that
 // starts a two-segment Local set), then the item's window / full pages, four pages per tile.
+// An item's pages in the order they are streamed: its sink pages (if it has any), then its
+// window / history pages, numbered 0 .. nv-1 and cut into tiles of four without regard to where
+// one segment ends and the other begins.
+__device__ __forceinline__ int item_pages(const Item& it) { return it.sink_pg1 + it.win_pg1 - it.win_pg0; }
+__device__ __forceinline__ int item_logical_page(const Item& it, int v)
+{
+    return v < it.sink_pg1 ? v : it.win_pg0 + v - it.sink_pg1;
+}
 struct TileWalk {
-    int seg;       // 0 = sinks, 1 = window/full, 2 = done
-    int pg;        // first logical page of the current tile
-    int npages;    // pages in the current tile (1..4)
+    int v;         // first page (in streaming order) of the current tile
+    int nv;        // pages of the item
+    int npages;    // pages in the current tile (1..4; 0 when done)
     __device__ __forceinline__ void start(const Item& it)
     {
-        seg = it.sink_pg1 > 0 ? 0 : 1;
-        pg = seg ? it.win_pg0 : 0;
-        settle(it);
+        v = 0;
+        nv = item_pages(it);
+        npages = min(4, nv);
     }
-    __device__ __forceinline__ void settle(const Item& it)
+    __device__ __forceinline__ void next()
     {
-        int end = seg == 0 ? it.sink_pg1 : it.win_pg1;
-        if (seg == 0 && pg >= end) { seg = 1; pg = it.win_pg0; end = it.win_pg1; }
-        if (seg == 1 && pg >= end) { seg = 2; npages = 0; return; }
-        npages = min(4, end - pg);
+        v += 4;
+        npages = max(0, min(4, nv - v));
     }
-    __device__ __forceinline__ void next(const Item& it) { pg += 4; settle(it); }
-    __device__ __forceinline__ bool done() const { return seg == 2; }
+    __device__ __forceinline__ bool done() const { return v >= nv; }
 };
 
-// Producer's view: runs of up to 32 consecutive logical pages of one item (8 tiles), whose block
+// Producer's view: runs of up to 32 consecutive pages (in streaming order) of one item (8 tiles), whose block
 // ids are fetched with one warp-wide load well before the copies that need them are issued.
 struct PageRun {
     int g, kv_layer, b;
     const __nv_bfloat16* q;  // q rows of the item, copied with the first tile of the item
-    int pg, n;               // first logical page, pages in the run (1..32)
+    int n;                   // pages in the run (1..32)
     bool first;              // first run of its item
     Item item;               // the item (meaningful in its first run)
     int take;
@@ -206,35 +211,27 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         span_range(plan, span, x, x_end);
         Item it;
         int take = decode_item(p, plan, span, x, x_end, it);
-        int seg = it.sink_pg1 > 0 ? 0 : 1;
-        int pg = seg ? it.win_pg0 : 0;
+        int v = 0, nv = item_pages(it);  // next page of the item in streaming order, pages it has
         bool more = true, item_first = true;
         auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when the span is done
             if (!more) return false;
-            const int end = seg ? it.win_pg1 : it.sink_pg1;
             r.g = it.g; r.kv_layer = it.kv_layer; r.b = it.b;
             r.q = p.q + (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + (size_t)it.g * G) * D;
-            r.pg = pg;
-            r.n = min(32, end - pg);
+            r.n = min(32, nv - v);
             r.first = item_first;
             if (item_first) { r.item = it; r.take = take; }
             item_first = false;
-            blk = lane < r.n ? __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + pg + lane) : 0;
-            pg += r.n;
-            if (pg >= end) {
-                if (seg == 0) {
-                    seg = 1;
-                    pg = it.win_pg0;
+            blk = lane < r.n ? __ldg(p.block_table + (size_t)it.b * p.max_blocks_per_seq + item_logical_page(it, v + lane)) : 0;
+            v += r.n;
+            if (v >= nv) {
+                x += take;
+                if (x < x_end) {
+                    take = decode_item(p, plan, span, x, x_end, it);
+                    v = 0;
+                    nv = item_pages(it);
+                    item_first = true;
                 } else {
-                    x += take;
-                    if (x < x_end) {
-                        take = decode_item(p, plan, span, x, x_end, it);
-                        seg = it.sink_pg1 > 0 ? 0 : 1;
-                        pg = seg ? it.win_pg0 : 0;
-                        item_first = true;
-                    } else {
-                        more = false;
-                    }
+                    more = false;
                 }
             }
             return true;
@@ -533,8 +530,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 a_wait += clock64() - c4;
 #endif
                 if (warp < tw.npages) {
-                    const int pos0 = (tw.pg + warp) * kPage;
-                    const int vlo = tw.seg ? it.win_lo : 0, vhi = tw.seg ? it.win_hi : it.sink_hi;
+                    const bool sink = tw.v + warp < it.sink_pg1;
+                    const int pos0 = item_logical_page(it, tw.v + warp) * kPage;
+                    const int vlo = sink ? 0 : it.win_lo, vhi = sink ? it.sink_hi : it.win_hi;
                     const bool edge = pos0 < vlo || pos0 + kPage > vhi;
                     const uint32_t kpage = smem_u32(ring + s * C::kStageBytes + warp * C::kPageBytes);
                     const uint32_t vpage = kpage + C::kTilePages * C::kPageBytes;
@@ -611,7 +609,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                         t_half = globaltimer_ns();
                     }
                 }
-                tw.next(it);
+                tw.next();
                 if (tw.done())
                     s_last = s;
                 else if (lane == 0)
