@@ -293,3 +293,39 @@ def test_unit_aligned_split_parity(layout):
     gh.assert_close(fl.cpu().numpy(), rlse, gh.ATOL_LSE, "full lse")
     assert ctx.read_device_status() == 0
 
+
+def _unit_aligned_case(case, grid):
+    """Draws shapes until one falls under the unit-aligned rule of the plan (average span of at most
+    128 pages, at least 8; every unit between 3/4 and 3/2 of it) on a launch of `grid` CTAs."""
+    rng = np.random.default_rng(4400 + case)
+    for _ in range(10000):
+        L, B, Hkv = int(rng.integers(2, 13)), int(rng.integers(1, 5)), int(rng.choice([1, 2, 4, 8]))
+        w, s = int(rng.choice([128, 200, 256, 384, 512, 777])), int(rng.choice([0, 4, 17]))
+        seq = [int(rng.integers(max(2, w // 2), 3 * w)) for _ in range(B)]
+        pages = []
+        for t in seq:   # pages of the window segment (Eq. 1); a separate sink page is not part of the unit's length
+            lo = 0 if t - w <= s else t - w
+            pages.append((t + 15) // 16 - lo // 16)
+        total, span = L * Hkv * sum(pages), L * Hkv * sum(pages) / grid
+        if total >= 8 * grid and span <= 128 and 0.75 * span <= min(pages) and max(pages) <= 1.5 * span:
+            return dict(L=L, B=B, Hkv=Hkv, w=w, s=s, seq=seq, G=int(rng.choice([1, 2, 4, 8])),
+                        layout=str(rng.choice(["hnd", "nhd"])), seed=int(rng.integers(1, 10**6)))
+    raise AssertionError("no eligible shape drawn")
+
+
+@pytest.mark.parametrize("case", range(6))
+def test_unit_aligned_split_random_shapes(case):
+    probe = gh.make_ctx(make_problem(1, 1, 1, 8, 8, 128, [40]), [16], [0], [1], variant=binding.VARIANT_TMA_MMA)
+    c = _unit_aligned_case(case, probe.attention_grid)
+    L, B, Hkv = c["L"], c["B"], c["Hkv"]
+    windows, sinks, gated = [c["w"]] * L, [c["s"]] * L, [1] * L
+    prob = make_problem(c["seed"], L, B, c["G"] * Hkv, Hkv, 128, c["seq"], layout=c["layout"])
+    ctx = gh.make_ctx(prob, windows, sinks, gated, variant=binding.VARIANT_TMA_MMA)
+    assert ctx.attention_grid == probe.attention_grid
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8)
+    gh.assert_close(out, ref, gh.ATOL_OUT, f"local out {c}")
+    gh.assert_close(lse, rlse, gh.ATOL_LSE, f"local lse {c}")
+    assert ctx.read_device_status() == 0
+
