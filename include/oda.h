@@ -121,6 +121,19 @@ oda_status_t oda_workspace_bytes(const oda_ctx_t* ctx, size_t* bytes);
 oda_status_t oda_set_workspace(oda_ctx_t* ctx, void* dev_ptr, size_t bytes, void* stream);
 
 /*
+ * Optional: keep part of the Local pass's working set in L2 between steps.  A decode loop reads
+ * nearly the same windows step after step; when they are larger than L2 a plain stream evicts
+ * every line before its next use.  With a budget set, the Local pass loads the pages of as many
+ * leading layers as fit `bytes` (batch x kv heads x (window + sinks) x head_dim x 4 bytes per
+ * layer) with an L2 evict-last hint and streams the rest evict-first as before, so that part of
+ * the next step's reads hits L2.  About half of the L2 is a good budget; 0 (the default) turns it
+ * off.  Host-only call, takes effect at the next launch (captured graphs keep what they were
+ * captured with).  The paper has no counterpart (its runtime copies the window into a ring
+ * workspace instead).
+ */
+oda_status_t oda_set_cache_resident_bytes(oda_ctx_t* ctx, size_t bytes);
+
+/*
  * Optional calibration of the split of work across SMs.  HBM bandwidth is not shared evenly among
  * the SMs of a GPU (on a B200, equal spans of KV finish +-10 % apart, in a pattern that is a fixed
  * property of the chip).  Between oda_calibration_begin() and oda_calibration_end() the attention

@@ -26,7 +26,7 @@ EXPORTS = [
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
     "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
-    "oda_recall_finalize_exchange", "oda_merge_partials_exchange",
+    "oda_recall_finalize_exchange", "oda_merge_partials_exchange", "oda_set_cache_resident_bytes",
 ]
 
 
@@ -120,6 +120,8 @@ def load_library():
         lib.oda_merge_partials_exchange.argtypes = [vp, i32, i32, i32, ctypes.POINTER(_MergeExchangeRank), vp, vp, vp,
                                                     ctypes.c_uint32, ctypes.c_uint64, i32, i32, i32, vp]
         lib.oda_merge_partials_exchange.restype = i32
+        lib.oda_set_cache_resident_bytes.argtypes = [vp, ctypes.c_size_t]
+        lib.oda_set_cache_resident_bytes.restype = i32
         lib.oda_full_decode_gated.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_step.argtypes = [vp, ctypes.POINTER(_StepArgs), vp]
         lib.oda_step_host.argtypes = [vp, ctypes.POINTER(_StepArgs), vp,
@@ -416,6 +418,10 @@ class OdaContext:
                                            _stream() if stream is None else stream,
                                            ctypes.byref(up), ctypes.byref(down)), "oda_step_host")
         return up.value, down.value
+
+    def set_cache_resident_bytes(self, nbytes: int):
+        """Local working set (leading layers) to keep in L2 between steps; 0 turns it off."""
+        self._check(self.lib.oda_set_cache_resident_bytes(self._h, int(nbytes)), "oda_set_cache_resident_bytes")
 
     # ---- introspection ----------------------------------------------------------------
     def read_device_status(self, stream=None) -> int:

@@ -41,6 +41,7 @@ struct oda_ctx {
     int variant = ODA_VARIANT_SIMT;
     int grid = 148;
     int min_span_pages = 8;
+    size_t l2_resident_bytes = 0;  // Local working set to keep in L2 between steps (oda_set_cache_resident_bytes)
     int snap_span_pages = 128;  // launches of up to 1 MiB per CTA may be cut at unit boundaries
     bool calibrated = false;  // the per-SM split table in the workspace is valid
     bool calibrating = false; // attention launches record per-SM streaming rates
@@ -165,6 +166,20 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     p.ncls = c->ncls;
     p.min_span_pages = c->min_span_pages;
     p.snap_span_pages = c->snap_span_pages;
+    if (mode == 0 && c->l2_resident_bytes > 0) {
+        // leading layers of the call whose Local working set fits the budget: their pages are loaded
+        // with an evict-last hint, so the next step finds them in L2
+        size_t used = 0;
+        int keep = lb;
+        for (; keep < le; ++keep) {
+            const int cls = c->layers[keep].cls;
+            const size_t tokens = (size_t)c->cls_window[cls] + (size_t)c->cls_sinks[cls];
+            const size_t bytes = (size_t)batch * f.num_kv_heads * tokens * f.head_dim * 4;  // K and V, bf16
+            if (used + bytes > c->l2_resident_bytes) break;
+            used += bytes;
+        }
+        p.l2_keep_layer_end = keep;
+    }
     p.max_items = c->max_items;
     p.scale_log2e = c->scale * 1.4426950408889634f;
     bool any = false;
@@ -376,6 +391,13 @@ oda_status_t oda_set_workspace(oda_ctx_t* c, void* dev_ptr, size_t bytes, void* 
     if (e != cudaSuccess) return cuda_fail(c, e, "workspace initialisation");
     c->ws = ws;
     c->calibrated = false;  // the table lives in the workspace
+    return ODA_OK;
+}
+
+oda_status_t oda_set_cache_resident_bytes(oda_ctx_t* c, size_t bytes)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    c->l2_resident_bytes = bytes;
     return ODA_OK;
 }
 

@@ -42,6 +42,7 @@ struct AttnParams {
                            //     merged into the Local result that out/lse already hold
     int32_t ncls;
     int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
+    int32_t l2_keep_layer_end; // Local pass: pages of layers below this one are loaded with an L2 evict-last hint (0: none)
     int32_t snap_span_pages; // launches with spans up to this long may be cut at unit boundaries (0: never)
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)

@@ -152,7 +152,7 @@ struct TileWalk {
 // Producer's view: runs of up to 32 consecutive pages (in streaming order) of one item (8 tiles), whose block
 // ids are fetched with one warp-wide load well before the copies that need them are issued.
 struct PageRun {
-    int g, kv_layer, b;
+    int g, kv_layer, b, layer;
     const __nv_bfloat16* q;  // q rows of the item, copied with the first tile of the item
     int n;                   // pages in the run (1..32)
     bool first;              // first run of its item
@@ -203,7 +203,8 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
 
     if (warp == C::kProducerWarp) {
         // ============================ producer warp ============================
-        const uint64_t policy = 0x12F0000000000000ull;  // L2 evict-first: the KV stream is read once
+        const uint64_t policy_stream = 0x12F0000000000000ull;  // L2 evict-first: the KV stream is read once
+        const uint64_t policy_keep = 0x14F0000000000000ull;    // L2 evict-last: windows the next step reads again
         uint32_t cnt = 0;
         bool dead = false;
         // walker over the runs of the CTA's span
@@ -215,7 +216,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         bool more = true, item_first = true;
         auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when the span is done
             if (!more) return false;
-            r.g = it.g; r.kv_layer = it.kv_layer; r.b = it.b;
+            r.g = it.g; r.kv_layer = it.kv_layer; r.b = it.b; r.layer = it.layer;
             r.q = p.q + (((size_t)it.layer * p.batch + it.b) * p.num_q_heads + (size_t)it.g * G) * D;
             r.n = min(32, nv - v);
             r.first = item_first;
@@ -262,6 +263,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                     const uint32_t kdst = smem_u32(ring + s * C::kStageBytes + lane * C::kPageBytes);
                     const uint32_t vdst = kdst + C::kTilePages * C::kPageBytes;
                     const int bcoord = cur.kv_layer * blocks_per_layer + blk;
+                    const uint64_t policy = cur.layer < p.l2_keep_layer_end ? policy_keep : policy_stream;
                     tma_load_page(kdst, &kmap, full0 + 8 * s, cur.g, bcoord, policy);
                     tma_load_page(vdst, &vmap, full0 + 8 * s, cur.g, bcoord, policy);
                 } else if (lane == 4 && with_q) {

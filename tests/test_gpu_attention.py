@@ -329,3 +329,24 @@ def test_unit_aligned_split_random_shapes(case):
     gh.assert_close(lse, rlse, gh.ATOL_LSE, f"local lse {c}")
     assert ctx.read_device_status() == 0
 
+
+def test_cache_resident_hint_changes_no_bits():
+    """The L2 evict-last hint on the leading layers' windows is a hint: same bits with any budget."""
+    L, Hq, Hkv, D = 6, 8, 2, 128
+    seq = [900, 70, 2053]
+    windows, sinks, gated = [256] * L, [4] * L, [1] * L
+    prob = make_problem(55, L, len(seq), Hq, Hkv, D, seq)
+    ctx = gh.make_ctx(prob, windows, sinks, gated, variant=binding.VARIANT_TMA_MMA)
+    dev = gh.upload(prob)
+    base, base_lse = gh.gpu_local(ctx, prob, dev)
+    per_layer = len(seq) * Hkv * (256 + 4) * D * 4
+    for budget in (per_layer - 1, 3 * per_layer, 1 << 40):   # no layer, three layers, all of them
+        ctx.set_cache_resident_bytes(budget)
+        out, lse = gh.gpu_local(ctx, prob, dev)
+        np.testing.assert_array_equal(out, base)
+        np.testing.assert_array_equal(lse, base_lse)
+    ctx.set_cache_resident_bytes(0)
+    ref, _ = oracle_attention(prob, "local", windows, sinks, nthreads=8)
+    gh.assert_close(base, ref, gh.ATOL_OUT, "local out")
+    assert ctx.read_device_status() == 0
+
