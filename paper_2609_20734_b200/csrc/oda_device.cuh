@@ -368,6 +368,30 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     }
 }
 
+// A gated pass in which no request is flagged has nothing to plan: every CTA finds that out from
+// the flags alone and leaves; CTA 0 does the step's bookkeeping (lengths, published decision,
+// counters) that the last CTA through the plan would otherwise do.  Uniform over the launch,
+// since every CTA reads the same flags.
+__device__ inline bool gated_pass_is_empty(const AttnParams& p)
+{
+    if (p.mode == 0 || p.sm_stats || !p.flags) return false;
+    int f = 0;
+    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) f |= p.flags[b];
+    if (__syncthreads_or(f)) return false;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        for (int b = 0; b < p.batch; ++b) {
+            if (p.advance_seq_lens) p.advance_seq_lens[b] += 1;
+            if (p.flags_out) {
+                p.flags_out[b] = 0;
+                if (p.scores_out) p.scores_out[b] = 0.5f;
+                if (p.logits_out) p.logits_out[b] = 0.f;
+                if (p.counters_out) p.counters_out[2 * b] += 1;
+            }
+        }
+    }
+    return true;
+}
+
 // Warms L2 with the block table while the plan is being built (the table is not produced by the
 // kernels of this library, so this may run before griddep_wait()).
 __device__ __forceinline__ void prefetch_block_table(const AttnParams& p)

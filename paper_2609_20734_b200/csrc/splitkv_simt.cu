@@ -49,6 +49,10 @@ splitkv_simt_kernel(const __grid_constant__ AttnParams p)
 
     prefetch_block_table(p);
     griddep_wait();
+    if (gated_pass_is_empty(p)) {
+        griddep_launch_dependents();
+        return;
+    }
     build_plan(p, plan);
     griddep_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;

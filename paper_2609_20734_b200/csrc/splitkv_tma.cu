@@ -193,6 +193,10 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     prefetch_block_table(p);
     griddep_wait();       // everything above is independent of the previous kernel in the stream
     if (tid == 0) ODA_TL(1);
+    if (gated_pass_is_empty(p)) {
+        griddep_launch_dependents();
+        return;
+    }
     build_plan(p, plan);  // ends with a barrier
     griddep_launch_dependents();
     if (tid == 0) ODA_TL(2);
