@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(kExchangeThreads) recall_exchange_kernel(const
         const uint32_t* f = p.arrived[rank] + tid;
         const uint64_t t0 = globaltimer_ns();
         uint32_t spins = 0;
-        while (ld_acquire_sys(f) != p.epoch) {
+        while ((int32_t)(ld_acquire_sys(f) - p.epoch) < 0) {  // a rank that is already one exchange ahead has arrived too
             if ((++spins & 63u) == 0 && globaltimer_ns() - t0 > p.timeout_ns) {
                 s_ok = 0;
                 break;
@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kExchangeThreads) merge_exchange_kernel(const 
         const uint32_t* f = p.arrived[rank] + (size_t)tid * kMergeBlocks + c;
         const uint64_t t0 = globaltimer_ns();
         uint32_t spins = 0;
-        while (ld_acquire_sys(f) != p.epoch) {
+        while ((int32_t)(ld_acquire_sys(f) - p.epoch) < 0) {  // a rank that is already one exchange ahead has arrived too
             if ((++spins & 63u) == 0 && globaltimer_ns() - t0 > p.timeout_ns) {
                 s_ok = 0;
                 break;
