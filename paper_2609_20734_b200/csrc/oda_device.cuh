@@ -287,8 +287,9 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         // streamed by one CTA, which writes the unit's rows itself -- no partials, tickets or
         // merge at the end, where a launch of a few tens of microseconds notices them.  Some CTAs
         // get no unit; such a launch is bound by DRAM, not by the number of streaming CTAs.  Not
-        // during calibration (which measures the equal split), and not when units are much
-        // shorter (uneven spans) or much longer (idle CTAs) than a span.
+        // during calibration (which measures the equal split), and not when units are shorter than
+        // a span (some CTAs would get two: measured 4-6 us slower than the equal split) or much
+        // longer (idle CTAs).
         span = __shfl_sync(0xffffffffu, span, 0);
         nseg = __shfl_sync(0xffffffffu, nseg, 0);
         const int total = (int)__shfl_sync(0xffffffffu, (int)carry, 0);
@@ -299,7 +300,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
                 umin = min(umin, pl.umin[c]);
                 umax = max(umax, pl.umax[c]);
             }
-            if (4 * umin * nseg >= 3 * total && 2 * umax * nseg <= 3 * total) {  // 3/4 span <= unit <= 3/2 span
+            if (umin * nseg >= total && 2 * umax * nseg <= 3 * total) {  // span <= unit <= 3/2 span
                 __syncwarp();  // lb[] was written by other lanes of this warp
                 int x = 0;
                 const int j = span + lane;  // lane 0: where the span starts, lane 1: where it ends
