@@ -397,6 +397,11 @@ oda_status_t oda_step(oda_ctx_t* ctx, const oda_step_args_t* args, void* stream)
  * weights and counters stay device pointers (they are state, not per-step input).  Copies
  * the inputs into staging areas of the workspace, runs oda_step, copies the results back and
  * waits for the stream.  Reports the bytes copied each way if the pointers are non-NULL.
+ * When no kernel reads the outputs back (no recall head configured, options bit 1 clear) and
+ * out, lse, scores, logits, flags are all pinned buffers (out 16-byte, lse / scores / logits
+ * 4-byte aligned), the kernels write them in place over the bus and no copy follows the last
+ * kernel (d2h_bytes then counts every output element once); with a pageable buffer among them
+ * everything goes through the staging copies.
  */
 oda_status_t oda_step_host(oda_ctx_t* ctx, const oda_step_args_t* args, void* stream,
                            size_t* h2d_bytes, size_t* d2h_bytes);

@@ -863,6 +863,19 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     return ODA_OK;
 }
 
+// The device's address for a suitably aligned pointer into pinned (page-locked, mapped) host
+// memory; nullptr for anything else (pageable memory is only reachable through a copy).
+static void* device_view_of_pinned(const void* host, uintptr_t align)
+{
+    if (!host || (reinterpret_cast<uintptr_t>(host) & (align - 1))) return nullptr;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream, size_t* h2d_bytes,
                            size_t* d2h_bytes)
 {
@@ -905,11 +918,33 @@ oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream,
         d.override_flags = reinterpret_cast<const uint8_t*>(c->ws + c->lay.st_override);
     }
 #undef ODA_UP
-    d.out = c->ws + c->lay.st_out;
-    d.lse = a->lse ? reinterpret_cast<float*>(c->ws + c->lay.st_lse) : nullptr;
-    d.scores = reinterpret_cast<float*>(c->ws + c->lay.st_scores);
-    d.logits = a->logits ? reinterpret_cast<float*>(c->ws + c->lay.st_logits) : nullptr;
-    d.flags = reinterpret_cast<uint8_t*>(c->ws + c->lay.st_flags);
+    // Where no kernel reads the step's outputs back (no recall head, no remainder-only Full pass: the
+    // attention kernels only write them) and the caller's buffers are pinned memory the device can
+    // address, the kernels write every output straight into them and no copy follows the last
+    // kernel: the bus transfer overlaps the end of the launch and three engine switches go away.
+    bool direct = f.head_d_hidden == 0 && !c->reuse_local;
+    void* dv_out = nullptr; void* dv_lse = nullptr; void* dv_scores = nullptr; void* dv_logits = nullptr; void* dv_flags = nullptr;
+    if (direct) {
+        dv_out = device_view_of_pinned(a->out, 16);
+        dv_scores = device_view_of_pinned(a->scores, 4);
+        dv_flags = device_view_of_pinned(a->flags, 1);
+        dv_lse = a->lse ? device_view_of_pinned(a->lse, 4) : nullptr;
+        dv_logits = a->logits ? device_view_of_pinned(a->logits, 4) : nullptr;
+        direct = dv_out && dv_scores && dv_flags && (!a->lse || dv_lse) && (!a->logits || dv_logits);
+    }
+    if (direct) {
+        d.out = dv_out;
+        d.lse = static_cast<float*>(dv_lse);
+        d.scores = static_cast<float*>(dv_scores);
+        d.logits = static_cast<float*>(dv_logits);
+        d.flags = static_cast<uint8_t*>(dv_flags);
+    } else {
+        d.out = c->ws + c->lay.st_out;
+        d.lse = a->lse ? reinterpret_cast<float*>(c->ws + c->lay.st_lse) : nullptr;
+        d.scores = reinterpret_cast<float*>(c->ws + c->lay.st_scores);
+        d.logits = a->logits ? reinterpret_cast<float*>(c->ws + c->lay.st_logits) : nullptr;
+        d.flags = reinterpret_cast<uint8_t*>(c->ws + c->lay.st_flags);
+    }
     oda_status_t s = oda_step(c, &d, stream);
     if (s != ODA_OK) return s;
 #define ODA_DOWN(field, off, bytes)                                                                   \
@@ -918,11 +953,15 @@ oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream,
         if (e != cudaSuccess) return cuda_fail(c, e, "device-to-host copy of " #field);               \
         down += (bytes);                                                                              \
     } while (0)
-    ODA_DOWN(out, st_out, rows * f.head_dim * out_elem(c));
-    if (a->lse) ODA_DOWN(lse, st_lse, rows * 4);
-    ODA_DOWN(scores, st_scores, (size_t)B * 4);
-    if (a->logits) ODA_DOWN(logits, st_logits, (size_t)B * 4);
-    ODA_DOWN(flags, st_flags, (size_t)B);
+    if (direct) {  // already on their way; counted once per element
+        down = rows * f.head_dim * out_elem(c) + (a->lse ? rows * 4 : 0) + (size_t)B * 4 + (a->logits ? (size_t)B * 4 : 0) + (size_t)B;
+    } else {
+        ODA_DOWN(out, st_out, rows * f.head_dim * out_elem(c));
+        if (a->lse) ODA_DOWN(lse, st_lse, rows * 4);
+        ODA_DOWN(scores, st_scores, (size_t)B * 4);
+        if (a->logits) ODA_DOWN(logits, st_logits, (size_t)B * 4);
+        ODA_DOWN(flags, st_flags, (size_t)B);
+    }
 #undef ODA_DOWN
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronise");

@@ -209,8 +209,10 @@ def test_step_forms_agree_eager_host_graph():
 
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_step_without_a_head(pinned):
-    """Head-less stack, forced flags, host buffers pinned or pageable: the host-buffer entry point
-    gives the bits of the device-pointer one (which is checked against the oracle), twice in a row."""
+    """Head-less stack, forced flags.  With pinned buffers the kernels write every output in place
+    over the bus, with pageable ones everything goes through staging copies: either way the
+    host-buffer entry point gives the bits of the device-pointer one (which is checked against the
+    oracle), twice in a row, scores and flags included."""
     from tests.helpers import make_problem
     L, Hq, Hkv, D = 3, 8, 2, 128
     seq = [700, 33, 1, 2100, 257]
@@ -244,6 +246,8 @@ def test_host_step_without_a_head(pinned):
         assert up == q_h.numel() * 2 + B and down == out_h.numel() * 4 + lse_h.numel() * 4 + B * 4 + B
         assert torch.equal(out_h, out.cpu()) and torch.equal(lse_h, lse.cpu())
         np.testing.assert_array_equal(fl_h.numpy(), ov_h)
+        assert torch.equal(sc_h, scores.cpu())
+        out_h.fill_(9.0), lse_h.fill_(9.0), sc_h.fill_(9.0), fl_h.fill_(9)
     assert ctx.read_device_status() == 0
 
 
