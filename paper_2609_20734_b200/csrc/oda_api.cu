@@ -210,6 +210,21 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
         p.sm_claims = reinterpret_cast<int32_t*>(c->ws + c->lay.sm_claims);
     }
     if (advanced) *advanced = advance != nullptr;
+    // A Local call over few layers cannot fill the usual grid: the window bounds its pages whatever
+    // the lengths are.  Launch only the CTAs the plan can give a span to (it cuts the page axis into
+    // min(grid, pages / min_span_pages) spans either way, so the split and the bits are the same);
+    // the rest would only start, build the plan and leave.
+    int grid = c->grid;
+    if (mode == 0 && c->min_span_pages > 0) {
+        long long bound = 0;  // pages on the axis, at most
+        for (int l = lb; l < le; ++l) {
+            const int cls = c->layers[l].cls;
+            const long long tokens = (long long)c->cls_window[cls] + c->cls_sinks[cls];  // one range when they touch
+            bound += (long long)batch * f.num_kv_heads * (tokens / kPage + 2);
+        }
+        const long long need = (bound + c->min_span_pages - 1) / c->min_span_pages;
+        if (need < grid) grid = (int)std::max<long long>(need, 1);
+    }
     cudaError_t e;
     if (c->variant == ODA_VARIANT_TMA_MMA) {
         if (c->kmap_base != k) {
@@ -224,9 +239,9 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
                 return fail(c, ODA_ERR_CUDA, "cuTensorMapEncodeTiled failed for v_cache");
             c->vmap_base = v;
         }
-        e = launch_splitkv_tma(p, c->kmap, c->vmap, c->blocks_per_layer, f.head_dim, c->group, c->grid, st, c->use_pdl);
+        e = launch_splitkv_tma(p, c->kmap, c->vmap, c->blocks_per_layer, f.head_dim, c->group, grid, st, c->use_pdl);
     } else {
-        e = launch_splitkv_simt(p, f.head_dim, c->group, c->grid, st, c->use_pdl);
+        e = launch_splitkv_simt(p, f.head_dim, c->group, grid, st, c->use_pdl);
     }
     if (e != cudaSuccess) return cuda_fail(c, e, "attention kernel launch");
     c->launches += 1;
