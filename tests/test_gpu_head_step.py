@@ -238,16 +238,17 @@ def test_host_step_without_a_head(pinned):
     out_h = place(torch.full((L, B, Hq, D), 9.0))
     lse_h = place(torch.full((L, B, Hq), 9.0))
     sc_h, fl_h = place(torch.zeros(B)), place(torch.zeros(B, dtype=torch.uint8))
+    lg_h = place(torch.full((B,), 9.0))
     ov_p = place(torch.from_numpy(ov_h.copy()))     # the argument block holds addresses, not references
     args = ctx.step_args(B, q_h, dev["k"], dev["v"], dev["table"], dev["seq_lens"], out_h, sc_h, fl_h,
-                         override_flags=ov_p, lse=lse_h)
+                         override_flags=ov_p, lse=lse_h, logits=lg_h)
     for _ in range(2):
         up, down = ctx.step_host(args)
-        assert up == q_h.numel() * 2 + B and down == out_h.numel() * 4 + lse_h.numel() * 4 + B * 4 + B
+        assert up == q_h.numel() * 2 + B and down == out_h.numel() * 4 + lse_h.numel() * 4 + B * 4 + B * 4 + B
         assert torch.equal(out_h, out.cpu()) and torch.equal(lse_h, lse.cpu())
         np.testing.assert_array_equal(fl_h.numpy(), ov_h)
-        assert torch.equal(sc_h, scores.cpu())
-        out_h.fill_(9.0), lse_h.fill_(9.0), sc_h.fill_(9.0), fl_h.fill_(9)
+        assert torch.equal(sc_h, scores.cpu()) and (lg_h == 0).all()    # no head: score 0.5, logit 0
+        out_h.fill_(9.0), lse_h.fill_(9.0), sc_h.fill_(9.0), fl_h.fill_(9), lg_h.fill_(9.0)
     assert ctx.read_device_status() == 0
 
 
