@@ -491,7 +491,7 @@ def main():
             tot = float(t.item())
         e2e = {"value": world * B * args.steps / tot, "unit": UNIT, "h2d_bytes_per_step": up,
                "d2h_bytes_per_step": down, "ms_per_step": tot / args.steps * 1e3,
-               "note": "oda_step_host: pinned host q/flags copied in, out/scores/flags back in pinned host memory "
+               "note": "oda_step_host: pinned host q/flags pulled in by one kernel, out/scores/flags back in pinned host memory "
                        "(written in place over the bus by the kernels when the stack has no recall head, copied "
                        "otherwise), stream sync inside; KV cache, block table and head weights are device-resident state"}
 

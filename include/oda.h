@@ -394,9 +394,11 @@ oda_status_t oda_step(oda_ctx_t* ctx, const oda_step_args_t* args, void* stream)
  * The same step for a caller whose per-step data lives in HOST memory: q_local, q_full,
  * feat_ext, override_flags are host inputs, out, lse, scores, logits, flags host outputs
  * (pinned memory makes the copies asynchronous); the KV cache, block table, seq_lens, head
- * weights and counters stay device pointers (they are state, not per-step input).  Copies
+ * weights and counters stay device pointers (they are state, not per-step input).  Brings
  * the inputs into staging areas of the workspace, runs oda_step, copies the results back and
- * waits for the stream.  Reports the bytes copied each way if the pointers are non-NULL.
+ * waits for the stream.  Reports the bytes moved each way if the pointers are non-NULL.
+ * When every input is pinned (q 16-byte aligned), one kernel pulls them all over the bus
+ * instead of one copy-engine transfer each.
  * When no kernel reads the outputs back (no recall head configured, options bit 1 clear) and
  * out, lse, scores, logits, flags are all pinned buffers (out 16-byte, lse / scores / logits
  * 4-byte aligned), the kernels write them in place over the bus and no copy follows the last

@@ -130,6 +130,34 @@ cudaError_t launch_merge_partials(const float* parts_out, const float* parts_lse
                      out, lse, n_parts, layer_begin, layer_end, batch, q_heads, num_layers, batch);
 }
 
+__global__ void __launch_bounds__(256) stage_in_kernel(const __grid_constant__ StageIn s)
+{
+    griddep_wait();
+    griddep_launch_dependents();  // the kernels that follow start their own set-up while this one copies
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nth = (long long)gridDim.x * blockDim.x;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const long long n16 = s.bytes[k] >> 4;
+        const uint4* src = static_cast<const uint4*>(s.src[k]);
+        uint4* dst = static_cast<uint4*>(s.dst[k]);
+        for (long long i = tid; i < n16; i += nth) dst[i] = src[i];
+        const long long tail = s.bytes[k] & 15;   // fewer than 16 bytes left: byte by byte
+        if (tid < tail)
+            static_cast<uint8_t*>(s.dst[k])[(n16 << 4) + tid] = static_cast<const uint8_t*>(s.src[k])[(n16 << 4) + tid];
+    }
+}
+
+cudaError_t launch_stage_in(const StageIn& s, cudaStream_t st, bool pdl)
+{
+    long long most = 0;
+    for (int k = 0; k < 4; ++k) most = most > s.bytes[k] ? most : s.bytes[k];
+    int grid = (int)((most / 16 + 255) / 256);   // every 16-byte piece of the largest input in flight at once
+    if (grid > 592) grid = 592;
+    if (grid < 1) grid = 1;
+    return launch_ex(stage_in_kernel, dim3(grid), dim3(256), 0, st, pdl, s);
+}
+
 cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const uint8_t* mask, void* k_cache,
                                     void* v_cache, const int32_t* block_table, const int32_t* seq_lens,
                                     const LayerInfo* layers, int num_layers, int batch, int num_kv_heads,

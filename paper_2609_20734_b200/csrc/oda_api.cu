@@ -912,27 +912,44 @@ oda_status_t oda_step_host(oda_ctx_t* c, const oda_step_args_t* a, void* stream,
     size_t up = 0, down = 0;
     oda_step_args_t d = *a;
     cudaError_t e;
-#define ODA_UP(field, off, bytes)                                                                     \
-    do {                                                                                              \
-        e = cudaMemcpyAsync(c->ws + c->lay.off, a->field, (bytes), cudaMemcpyHostToDevice, st);       \
-        if (e != cudaSuccess) return cuda_fail(c, e, "host-to-device copy of " #field);               \
-        up += (bytes);                                                                                \
-    } while (0)
-    ODA_UP(q_local, st_q_local, qbytes);
+    // Inputs: when every one of them is pinned memory the device can address, one kernel pulls them
+    // all into the staging areas (one launch instead of up to four copy-engine transfers, and the
+    // first attention kernel's set-up overlaps it); otherwise one copy each.
+    const size_t feat_bytes = (a->feat_ext && f.head_d_ext > 0) ? (size_t)B * f.head_d_ext * 4 : 0;
+    StageIn si;
+    std::memset(&si, 0, sizeof si);
+    const void* hosts[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool pull = true;
+    int nsi = 0;
+    auto want = [&](const void* host, size_t off, size_t bytes) {
+        if (!host || !bytes) return;
+        void* dv = device_view_of_pinned(host, bytes >= 16 ? 16 : 1);
+        if (!dv) pull = false;
+        hosts[nsi] = host;
+        si.src[nsi] = dv;
+        si.dst[nsi] = c->ws + off;
+        si.bytes[nsi] = (long long)bytes;
+        ++nsi;
+        up += bytes;
+    };
+    want(a->q_local, c->lay.st_q_local, qbytes);
+    want(a->q_full, c->lay.st_q_full, qbytes);
+    want(a->feat_ext, c->lay.st_feat, feat_bytes);
+    want(a->override_flags, c->lay.st_override, (size_t)B);
+    if (pull) {
+        e = launch_stage_in(si, st, c->use_pdl);
+        if (e != cudaSuccess) return cuda_fail(c, e, "input staging kernel launch");
+        c->launches += 1;
+    } else {
+        for (int k = 0; k < nsi; ++k) {
+            e = cudaMemcpyAsync(si.dst[k], hosts[k], (size_t)si.bytes[k], cudaMemcpyHostToDevice, st);
+            if (e != cudaSuccess) return cuda_fail(c, e, "host-to-device copy of a step input");
+        }
+    }
     d.q_local = c->ws + c->lay.st_q_local;
-    if (a->q_full) {
-        ODA_UP(q_full, st_q_full, qbytes);
-        d.q_full = c->ws + c->lay.st_q_full;
-    }
-    if (a->feat_ext && f.head_d_ext > 0) {
-        ODA_UP(feat_ext, st_feat, (size_t)B * f.head_d_ext * 4);
-        d.feat_ext = reinterpret_cast<const float*>(c->ws + c->lay.st_feat);
-    }
-    if (a->override_flags) {
-        ODA_UP(override_flags, st_override, (size_t)B);
-        d.override_flags = reinterpret_cast<const uint8_t*>(c->ws + c->lay.st_override);
-    }
-#undef ODA_UP
+    if (a->q_full) d.q_full = c->ws + c->lay.st_q_full;
+    if (feat_bytes) d.feat_ext = reinterpret_cast<const float*>(c->ws + c->lay.st_feat);
+    if (a->override_flags) d.override_flags = reinterpret_cast<const uint8_t*>(c->ws + c->lay.st_override);
     // Where no kernel reads the step's outputs back (no recall head, no remainder-only Full pass: the
     // attention kernels only write them) and the caller's buffers are pinned memory the device can
     // address, the kernels write every output straight into them and no copy follows the last

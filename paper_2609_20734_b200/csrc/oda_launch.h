@@ -46,6 +46,15 @@ cudaError_t launch_write_current_kv(const void* k_cur, const void* v_cur, const 
                                     int head_dim, int max_blocks_per_seq, int64_t layer_stride,
                                     int64_t block_stride, int64_t token_stride, int64_t head_stride,
                                     int32_t* status, cudaStream_t st, bool pdl = false);
+// Per-step inputs that live in pinned host memory, pulled into their staging areas by one kernel
+// (plain loads over the bus) instead of one copy-engine transfer each.
+struct StageIn {
+    const void* src[4];   // device views of the host buffers (16-byte aligned where bytes >= 16)
+    void* dst[4];
+    long long bytes[4];   // 0: unused
+};
+cudaError_t launch_stage_in(const StageIn& s, cudaStream_t st, bool pdl);
+
 cudaError_t launch_select_rows(const void* local, const void* full, const uint8_t* flags, void* out, int batch,
                                size_t row_bytes, cudaStream_t st, bool pdl = false);
 
