@@ -83,3 +83,14 @@ def test_calls_without_workspace_fail_cleanly():
         ctx.set_workspace(4096, 16, stream=0)       # too small
     assert e.value.status == 3
     assert binding.load_library().oda_status_string(3) == b"workspace missing or too small"
+
+
+def test_host_only_calls_check_their_arguments():
+    """An entry point that does no device work: a NULL context is refused, any budget is accepted."""
+    lib = binding.load_library()
+    assert lib.oda_set_cache_resident_bytes(None, 0) == 1
+    ctx = binding.OdaContext(base_cfg(), allocate_workspace=False)
+    ctx.set_cache_resident_bytes(64 << 20)
+    ctx.set_cache_resident_bytes(0)
+    ctx.close()
+
