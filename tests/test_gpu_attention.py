@@ -265,7 +265,7 @@ def test_layer_and_batch_limits_together(variant):
 def test_unit_aligned_split_parity(layout):
     """A short launch whose (layer, request, kv head) units are about one CTA's share each is cut at
     unit boundaries: every unit is streamed whole by one CTA and written without partials.  The
-    shape below falls under that rule on the launch grid in use (asserted), with units of 32 and 33
+    shape below falls under that rule on a 148-SM part (checked; skipped elsewhere), with units of 32 and 33
     pages, a sink page each, and more CTAs than units; so does the Full pass over the same requests
     (units of 94 and 95 pages)."""
     L, Hq, Hkv, D = 10, 16, 8, 128
@@ -275,8 +275,8 @@ def test_unit_aligned_split_parity(layout):
     ctx = gh.make_ctx(prob, windows, sinks, gated, variant=binding.VARIANT_TMA_MMA)
     units, pages = L * len(seq) * Hkv, L * Hkv * (33 + 32 + 33)
     span = pages / ctx.attention_grid
-    assert pages >= 8 * ctx.attention_grid and span <= 128 and span <= 32 and 33 <= 1.5 * span, \
-        f"{units} units of 32-33 pages on {ctx.attention_grid} CTAs: outside the unit-aligned rule"
+    if not (pages >= 8 * ctx.attention_grid and span <= 128 and span <= 32 and 33 <= 1.5 * span):
+        pytest.skip(f"{units} units of 32-33 pages on {ctx.attention_grid} CTAs: outside the unit-aligned rule")
     dev = gh.upload(prob)
     out, lse = gh.gpu_local(ctx, prob, dev)
     ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8)
