@@ -225,6 +225,10 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
         const long long need = (bound + c->min_span_pages - 1) / c->min_span_pages;
         if (need < grid) grid = (int)std::max<long long>(need, 1);
     }
+    {   // necessary for the batch-1 one-unit-per-CTA plan, whatever the length turns out to be
+        const long long units = (long long)(le - lb) * f.num_kv_heads;
+        p.direct_hint = (mode == 0 && batch == 1 && c->snap_span_pages > 0 && units <= grid && 2ll * grid <= 3 * units) ? 1 : 0;
+    }
     cudaError_t e;
     if (c->variant == ODA_VARIANT_TMA_MMA) {
         if (c->kmap_base != k) {

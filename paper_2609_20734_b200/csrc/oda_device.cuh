@@ -43,6 +43,7 @@ struct AttnParams {
     int32_t ncls;
     int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
     int32_t l2_keep_layer_end; // Local pass: pages of layers below this one are loaded with an L2 evict-last hint (0: none)
+    int32_t direct_hint;     // batch-1 Local launch whose shape allows one unit per CTA (see build_plan)
     int32_t snap_span_pages; // launches with spans up to this long may be cut at unit boundaries (0: never)
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)
@@ -99,7 +100,8 @@ struct Plan {  // shared memory, one per CTA
     int32_t my_span;                         // the span this CTA streams (-1: none)
     int32_t total_pages;
     int32_t nseg;
-    int32_t snap;                            // unit-aligned split: this CTA streams axis pages [x0, x1), whole units
+    int32_t snap;                            // 1: unit-aligned split, this CTA streams axis pages [x0, x1), whole units;
+                                             // 2: batch 1, CTA u streams unit u (cls[0], kv_index[0] are its layer's)
     int32_t x0, x1;
     int32_t umin[kMaxClasses], umax[kMaxClasses];  // shortest / longest unit of each class (pages; 0 pages not counted)
 };
@@ -163,6 +165,48 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     const int tid = threadIdx.x, nth = blockDim.x;
     const int B = p.batch;
     const int nl = p.layer_end - p.layer_begin;
+    // Batch 1, Local pass, unit-aligned split: with one request every unit of a layer class has the
+    // same length, so whether the launch falls under the unit-aligned rule (see below) follows from
+    // the one length alone, and then CTA u simply takes unit u = (layer u / H, kv head u % H).  No
+    // scans, no claims, one barrier: this is the latency-critical launch of batch-1 decoding.
+    if (p.direct_hint && !p.sm_stats) {  // host side of the rule: mode 0, batch 1, units <= CTAs <= 3/2 units
+        const int g = (int)gridDim.x, H = p.num_kv_heads;
+        const int t = p.seq_lens[0];
+        LayerInfo li;
+        li.cls = li.kv_index = 0;
+        if (tid == 0) li = p.layers[p.layer_begin + min((int)blockIdx.x / H, nl - 1)];
+        long long total = 0;
+        int umin = 0x7fffffff, umax = 0;
+        if (t >= 1 && t <= p.max_blocks_per_seq * kPage) {  // anything else is the general path's to report
+            for (int c = 0; c < p.ncls; ++c) {
+                if (p.cls_layers_in_call[c] <= 0) continue;
+                const Ranges r = eq1_ranges(0, t, p.cls_window[c], p.cls_sinks[c]);
+                const int np = r.pg1 - r.pg0;
+                total += (long long)p.cls_layers_in_call[c] * H * np;
+                umin = min(umin, np);
+                umax = max(umax, np);
+            }
+        }
+        const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
+        if (total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
+            (long long)umin * g >= total && 2ll * umax * g <= 3 * total) {
+            if (tid == 0) {
+                pl.snap = 2;
+                pl.weighted = 0;
+                pl.nseg = g;
+                pl.total_pages = (int32_t)total;
+                pl.my_span = (int)blockIdx.x < nl * H ? (int)blockIdx.x : -1;
+                pl.x0 = 0;
+                pl.x1 = 1;
+                pl.seq[0] = t;
+                pl.active[0] = 1;
+                pl.cls[0] = (uint8_t)li.cls;          // of this CTA's layer
+                pl.kv_index[0] = (uint16_t)li.kv_index;
+            }
+            __syncthreads();
+            return;
+        }
+    }
     // weighted split: claim one of the two spans of the SM this CTA runs on (answer used at the end)
     const bool weighted = p.cum_share != nullptr && (int)gridDim.x == 2 * p.num_sms && (int)gridDim.x <= kMaxGrid;
     int claim_sm = 0, claim_slot = 0;
@@ -475,6 +519,26 @@ __device__ __forceinline__ int span_of_near(const Plan& pl, int x, int j, int di
 // Returns the number of axis pages it covers (>= 1).
 __device__ inline int decode_item(const AttnParams& p, const Plan& pl, int j, int x, int x_end, Item& it)
 {
+    if (pl.snap == 2) {  // batch 1, one unit per CTA: span j is unit (layer j / H, kv head j % H)
+        const int H = p.num_kv_heads;
+        const int lo = j / H, c = pl.cls[0], t = pl.seq[0];
+        const Ranges rg = eq1_ranges(p.mode, t, p.cls_window[c], p.cls_sinks[c]);
+        it.layer = p.layer_begin + lo;
+        it.b = 0;
+        it.g = j - lo * H;
+        it.chunk = 0;
+        it.nchunks = 1;
+        it.slot_base = 0;
+        it.kv_layer = pl.kv_index[0];
+        it.t = t;
+        it.win_pg0 = rg.pg0;
+        it.win_pg1 = rg.pg1;
+        it.win_lo = rg.lo;
+        it.win_hi = rg.hi;
+        it.sink_hi = rg.sink_hi;
+        it.sink_pg1 = (it.sink_hi + kPage - 1) / kPage;
+        return 1;  // the span is [0, 1) on a nominal axis
+    }
     const int nl = p.layer_end - p.layer_begin;
     int lo = 0, hi = nl;  // last layer with lb <= x
     while (hi - lo > 1) {

@@ -113,6 +113,7 @@ extern "C" oda_status_t oda_local_decode_static(int32_t batch, int32_t num_q_hea
     p.ncls = 1;
     p.min_span_pages = 8;
     p.snap_span_pages = 0;
+    p.direct_hint = 0;
     p.l2_keep_layer_end = 0;
     p.max_items = kStaticMaxItems;
     p.scale_log2e = (sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim)) * 1.4426950408889634f;

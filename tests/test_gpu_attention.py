@@ -350,3 +350,26 @@ def test_cache_resident_hint_changes_no_bits():
     gh.assert_close(base, ref, gh.ATOL_OUT, "local out")
     assert ctx.read_device_status() == 0
 
+
+@pytest.mark.parametrize("layout,t", [("hnd", 700), ("nhd", 1024), ("hnd", 263), ("hnd", 150)])
+def test_batch_one_unit_per_cta_parity(layout, t):
+    """Batch 1 with about as many (layer, kv head) units as CTAs: the plan gives CTA u unit u without
+    any scan.  Lengths: window and sinks apart (unaligned and page-aligned), window just past the
+    sinks, and shorter than the window (one range); layers alias three cache slices."""
+    L, Hq, Hkv, D = 30, 16, 8, 128
+    windows, sinks, gated = [256] * L, [4] * L, [1] * L
+    kv_index = [l % 3 for l in range(L)]
+    prob = make_problem(808 + t, L, 1, Hq, Hkv, D, [t], layout=layout, kv_layers=3)
+    ctx = gh.make_ctx(prob, windows, sinks, gated, kv_index=kv_index, variant=binding.VARIANT_TMA_MMA)
+    grid, units = ctx.attention_grid, L * Hkv
+    if not (units <= grid <= 1.5 * units):
+        pytest.skip(f"{units} units on {grid} CTAs: outside the one-unit-per-CTA rule")
+    dev = gh.upload(prob)
+    out, lse = gh.gpu_local(ctx, prob, dev)
+    ref, rlse = oracle_attention(prob, "local", windows, sinks, nthreads=8, layer_kv_index=kv_index)
+    gh.assert_close(out, ref, gh.ATOL_OUT, "local out")
+    gh.assert_close(lse, rlse, gh.ATOL_LSE, "local lse")
+    again, _ = gh.gpu_local(ctx, prob, dev)
+    np.testing.assert_array_equal(again, out)
+    assert ctx.read_device_status() == 0
+
