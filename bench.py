@@ -169,11 +169,11 @@ def reference_arm(args, wl, realised_rate=None):
     if rank != 0:
         return
     cores = orc.host_threads()
-    nl, nf = 1, 1
+    nl = nf = min(8, wl.L)      # sampled layers; they read one generated cache slice (each with its own queries)
     table, nb = wl.tables()
     lay = orc.hnd_layout(nb, wl.Hkv, 16, wl.D)
     kk, vk = synth.stream_key(wl.seed, synth.STREAM_K), synth.stream_key(wl.seed, synth.STREAM_V)
-    idx = np.arange(0, nl * lay.layer_stride, dtype=np.uint64)
+    idx = np.arange(0, lay.layer_stride, dtype=np.uint64)
     k, v = synth.gauss_bf16(kk, idx), synth.gauss_bf16(vk, idx)
     flags = schedule_flags(wl, args.warmup, args.steps)
     realised = float(np.mean([f.mean() for f in flags[args.warmup:]])) if realised_rate is None else realised_rate
@@ -183,7 +183,7 @@ def reference_arm(args, wl, realised_rate=None):
         t0 = time.perf_counter()
         orc.attention(mode, q, k, v, table, np.asarray(wl.seq_lens0) + step, num_kv_heads=wl.Hkv,
                       block_size=16, layout=lay, layer_window=wl.windows[:n], layer_sinks=wl.sinks[:n],
-                      nthreads=cores if threads is None else threads)
+                      layer_kv_index=[0] * n, nthreads=cores if threads is None else threads)
         return time.perf_counter() - t0
 
     for s in range(args.warmup):
