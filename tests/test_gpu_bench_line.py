@@ -1,0 +1,40 @@
+"""The benchmark's own arm on a GPU: one JSON line with every key of the contract, internally
+consistent (a short run of the real configuration; the numbers themselves are not judged here)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_bench_prints_one_contract_line():
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "8", "--warmup", "3", "--no-sweep",
+                        "--kernel-reps", "2"], capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["metric"] == "decode_attention_tokens_per_s" and d["unit"] == "tokens/s" and "impl" not in d
+    assert d["n_gpus"] == 1 and d["steps"] == 8 and d["warmup"] == 3 and d["higher_is_better"] is True
+    assert d["scaling"] == "weak" and d["vs_baseline"] is None and d["data"] == "synthetic" and d["dtype"] == "bf16"
+    assert abs(d["value"] - 1e3 / d["ms_per_step"]) < 1e-6 * d["value"]          # batch 1: tokens/s = 1 / step time
+    assert "llama8b" in d["config"]["workload"] and "flushed" in d["config"]["l2"]
+    assert d["config"]["recall_rate_realised"] == 0.25
+    assert d["gpu_launches"] == 2 * d["steps"]
+    roof = d["roofline"]
+    assert roof["bound"] == "hbm" and roof["unit"] == "GB/s" and roof["peak"] > 0 and roof["traffic"] > 0
+    assert abs(roof["frac"] - roof["achieved"] / roof["peak"]) < 1e-9
+    assert abs(roof["achieved"] - roof["algorithmic_bytes"] / (roof["us"] * 1e-6) / 1e9) < 1e-6 * roof["achieved"]
+    assert 0.98 < roof["traffic"] / roof["algorithmic_bytes"] < 1.1
+    e2e = d["e2e"]
+    assert e2e["unit"] == "tokens/s" and 0 < e2e["value"] < d["value"]
+    assert e2e["h2d_bytes_per_step"] == 32 * 32 * 128 * 2 + 1                       # q (bf16) and one forced flag
+    assert e2e["d2h_bytes_per_step"] == 32 * 32 * 128 * 4 + 4 + 1                   # rows (f32), score, flag
+    cpu = d["cpu_baseline"]
+    assert cpu["kind"] == "oracle" and cpu["cores"] >= 1 and cpu["value"] > 0 and cpu["sample"]
+    clk = d["clocks"]
+    assert clk["sm_max_mhz"] >= clk["sm_mhz"] > 0 and isinstance(clk["reasons"], list)
