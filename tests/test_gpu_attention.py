@@ -275,7 +275,7 @@ def test_unit_aligned_split_parity(layout):
     ctx = gh.make_ctx(prob, windows, sinks, gated, variant=binding.VARIANT_TMA_MMA)
     units, pages = L * len(seq) * Hkv, L * Hkv * (33 + 32 + 33)
     span = pages / ctx.attention_grid
-    if not (pages >= 8 * ctx.attention_grid and span <= 128 and span <= 32 and 33 <= 1.5 * span):
+    if not (pages >= 16 * ctx.attention_grid and span <= 128 and span <= 32 and 33 <= 1.5 * span):
         pytest.skip(f"{units} units of 32-33 pages on {ctx.attention_grid} CTAs: outside the unit-aligned rule")
     dev = gh.upload(prob)
     out, lse = gh.gpu_local(ctx, prob, dev)
@@ -296,7 +296,7 @@ def test_unit_aligned_split_parity(layout):
 
 def _unit_aligned_case(case, grid):
     """Draws shapes until one falls under the unit-aligned rule of the plan (average span of at most
-    128 pages, at least 8; every unit between 1 and 3/2 of it) on a launch of `grid` CTAs."""
+    128 pages, at least 16; every unit between 1 and 3/2 of it) on a launch of `grid` CTAs."""
     rng = np.random.default_rng(4400 + case)
     for _ in range(10000):
         L, B, Hkv = int(rng.integers(2, 13)), int(rng.integers(1, 5)), int(rng.choice([1, 2, 4, 8]))
@@ -307,7 +307,7 @@ def _unit_aligned_case(case, grid):
             lo = 0 if t - w <= s else t - w
             pages.append((t + 15) // 16 - lo // 16)
         total, span = L * Hkv * sum(pages), L * Hkv * sum(pages) / grid
-        if total >= 8 * grid and span <= 128 and span <= min(pages) and max(pages) <= 1.5 * span:
+        if total >= 16 * grid and span <= 128 and span <= min(pages) and max(pages) <= 1.5 * span:
             return dict(L=L, B=B, Hkv=Hkv, w=w, s=s, seq=seq, G=int(rng.choice([1, 2, 4, 8])),
                         layout=str(rng.choice(["hnd", "nhd"])), seed=int(rng.integers(1, 10**6)))
     raise AssertionError("no eligible shape drawn")
@@ -351,13 +351,13 @@ def test_cache_resident_hint_changes_no_bits():
     assert ctx.read_device_status() == 0
 
 
-@pytest.mark.parametrize("layout,t", [("hnd", 700), ("nhd", 1024), ("hnd", 263), ("hnd", 150)])
+@pytest.mark.parametrize("layout,t", [("hnd", 700), ("nhd", 1024), ("hnd", 519), ("hnd", 400)])
 def test_batch_one_unit_per_cta_parity(layout, t):
     """Batch 1 with about as many (layer, kv head) units as CTAs: the plan gives CTA u unit u without
     any scan.  Lengths: window and sinks apart (unaligned and page-aligned), window just past the
     sinks, and shorter than the window (one range); layers alias three cache slices."""
     L, Hq, Hkv, D = 30, 16, 8, 128
-    windows, sinks, gated = [256] * L, [4] * L, [1] * L
+    windows, sinks, gated = [512] * L, [4] * L, [1] * L
     kv_index = [l % 3 for l in range(L)]
     prob = make_problem(808 + t, L, 1, Hq, Hkv, D, [t], layout=layout, kv_layers=3)
     ctx = gh.make_ctx(prob, windows, sinks, gated, kv_index=kv_index, variant=binding.VARIANT_TMA_MMA)
