@@ -13,7 +13,7 @@
 // of the slowest one (it needs that rank's flag to get past step 3), so the buffer it writes at
 // epoch e+2 has been read by everybody at epoch e.
 //
-// No collective library call, no multicast, no load from a peer: only stores to peers and loads
+// No collective library call, no switch-side replication, no load from a peer: only stores to peers and loads
 // from local memory.  On one GPU the same kernel is checked by giving each "rank" a CTA of ONE
 // cooperative launch (the CTAs wait on one another, so they must be co-resident) and separate
 // buffers.  A wait that runs out sets bit 2 of the status word, leaves the outputs untouched and

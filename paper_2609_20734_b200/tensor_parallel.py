@@ -155,7 +155,7 @@ class ExchangeBuffers:
     def symmetric(cls, group, batch, d_hidden, device="cuda"):
         """One rank per process and GPU: buffers in torch's symmetric memory, peers' addresses from
         its rendezvous.  Not tested on a GPU (this build had one): the addresses are used for plain
-        peer stores only, never for multicast or TMA."""
+        peer stores only, never as the source of a copy-engine or tensor-map load."""
         import torch
         import torch.distributed as dist
         import torch.distributed._symmetric_memory as symm
