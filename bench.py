@@ -119,6 +119,9 @@ class ClockSampler:
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        deadline = time.time() + 2.0      # a very short run can end before nvidia-smi has printed its first row
+        while not self.rows and time.time() < deadline and self.proc.poll() is None:
+            time.sleep(0.02)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
