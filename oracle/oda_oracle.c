@@ -39,7 +39,9 @@
  * oda_oracle_full_head: three RMSNorm -> Linear -> SiLU towers, the 9-way
  * interaction vector, the fusion projection, pre-norm residual SwiGLU blocks and a
  * normalised scalar output, in the paper's order; its parameter count is pinned to
- * the 28,325,889 the paper states.
+ * the 28,325,889 the paper states, the order of the nine interaction segments by
+ * one-hot rows of the fusion matrix read against a hand-made table, and a SwiGLU
+ * block, the fusion bias and the placement of eps by values worked out by hand.
  *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py
  * (brute force over literal 1-based sets in extended precision, an independent
