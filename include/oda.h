@@ -442,6 +442,9 @@ int32_t oda_attention_grid(const oda_ctx_t* ctx);
  * current) -- make that first call outside any stream capture.
  * Every call on a device uses the same array: a call clears what it needs to start from zero,
  * but two calls that overlap on the GPU (different streams) race.  Serialise them.
+ * Problems only the device can see (a request with seq_len < 1: its rows are left untouched;
+ * a seq_len beyond max_blocks_per_seq*16: clamped to it) set bits in a status word inside the
+ * same array; it keeps them across calls until oda_local_decode_static_status() reads it.
  */
 oda_status_t oda_local_decode_static(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads,
                                      int32_t head_dim, int32_t window, int32_t sinks, float sm_scale,
@@ -449,6 +452,12 @@ oda_status_t oda_local_decode_static(int32_t batch, int32_t num_q_heads, int32_t
                                      int64_t kv_head_stride, int32_t max_blocks_per_seq, const void* q,
                                      const void* k_cache, const void* v_cache, const int32_t* block_table,
                                      const int32_t* seq_lens, float* out, float* lse, void* stream);
+
+/* Reads and clears the status word that the oda_local_decode_static() calls on the current
+ * device have been setting (same bits as oda_read_device_status; no counterpart in the paper).
+ * Allocates nothing; synchronises the stream.  Returns ODA_ERR_DEVICE_STATUS when *code != 0.
+ * Like the entry point itself, its first call on a device must come outside stream capture. */
+oda_status_t oda_local_decode_static_status(void* stream, int32_t* code);
 
 const char* oda_status_string(oda_status_t s);
 const char* oda_last_error(const oda_ctx_t* ctx); /* host string describing the last failure */

@@ -23,6 +23,7 @@ EXPORTS = [
     "oda_recall_score", "oda_full_decode_gated", "oda_step", "oda_step_host",
     "oda_read_device_status", "oda_launch_count", "oda_resolved_variant", "oda_attention_grid",
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
+    "oda_local_decode_static_status",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
     "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
@@ -129,6 +130,7 @@ def load_library():
         lib.oda_local_decode_static.argtypes = [i32, i32, i32, i32, i32, i32, f32, ctypes.c_int64,
                                                 ctypes.c_int64, ctypes.c_int64, i32, vp, vp, vp, vp, vp,
                                                 vp, vp, vp]
+        lib.oda_local_decode_static_status.argtypes = [vp, ctypes.POINTER(i32)]
         lib.oda_write_current_kv.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_select_rows.argtypes = [vp, i32, vp, vp, vp, vp, ctypes.c_int64, vp]
         lib.oda_full_head_param_count.argtypes = [i32, i32, i32, i32]
@@ -457,6 +459,17 @@ def local_decode_static(batch, num_q_heads, num_kv_heads, head_dim, window, sink
         _ptr(block_table), _ptr(seq_lens), _ptr(out), _ptr(lse), _stream() if stream is None else stream)
     if st != 0:
         raise OdaError(st, "oda_local_decode_static", load_library().oda_status_string(st).decode())
+
+
+def local_decode_static_status(stream=None) -> int:
+    """Reads and clears the status word of the local_decode_static calls made on the current device
+    (bit 0: a request had seq_len < 1 and was skipped; same bits as OdaContext.read_device_status).
+    Synchronises the stream; allocates nothing."""
+    code = ctypes.c_int32(0)
+    st = load_library().oda_local_decode_static_status(_stream() if stream is None else stream, ctypes.byref(code))
+    if st not in (0, 5):
+        raise OdaError(st, "oda_local_decode_static_status", load_library().oda_status_string(st).decode())
+    return int(code.value)
 
 
 def version() -> str:
