@@ -176,6 +176,40 @@ def make(name: str, **ov) -> Workload:
     return replace(wl, **ov) if ov else wl
 
 
+def full_head_layout(d_model: int, d_tower: int, d_ff: int, n_blocks: int):
+    """(name, shape) of the parameters of the paper's recall head in storage order: three towers
+    (norm gain, weight, bias), the fusion projection, the SwiGLU blocks (norm gain, gate, up, down),
+    the output norm gain, output vector and output bias."""
+    out = []
+    for i in range(3):
+        out += [(f"g{i}", (d_model,)), (f"W{i}", (d_tower, d_model)), (f"b{i}", (d_tower,))]
+    out += [("Wf", (d_tower, 9 * d_tower)), ("bf", (d_tower,))]
+    for k in range(n_blocks):
+        out += [(f"bg{k}", (d_tower,)), (f"Wg{k}", (d_ff, d_tower)), (f"Wu{k}", (d_ff, d_tower)),
+                (f"Wd{k}", (d_tower, d_ff))]
+    out += [("go", (d_tower,)), ("w", (d_tower,)), ("bias", (1,))]
+    return out
+
+
+def full_head_params(seed: int, d_model: int, d_tower: int, d_ff: int, n_blocks: int) -> np.ndarray:
+    """Random-init parameters of the paper's head as one flat fp32 array: weights ~ N(0, 1/fan_in),
+    biases ~ N(0, 0.1^2), norm gains 1 + N(0, 0.1^2)."""
+    parts = []
+    for i, (name, shape) in enumerate(full_head_layout(d_model, d_tower, d_ff, n_blocks)):
+        std = 1.0 / np.sqrt(shape[-1]) if len(shape) == 2 else 0.1
+        x = synth.gauss_f32_tensor(seed, 200 + i, shape, std=std)
+        if name.startswith("g") or name.startswith("bg"):
+            x = (1.0 + x).astype(np.float32)
+        parts.append(x.reshape(-1))
+    return np.concatenate(parts)
+
+
+def full_head_input(seed: int, which: int, batch: int, d_model: int) -> np.ndarray:
+    """Synthetic input of the paper's head: which = 0 preceding hidden state, 1 embedding, 2 Local
+    hidden state; fp32 ~ N(0,1), [batch, d_model]."""
+    return synth.gauss_f32_tensor(seed, 300 + which, (batch, d_model))
+
+
 @dataclass
 class DeviceState:
     wl: Workload

@@ -221,3 +221,58 @@ def test_sequence_shard_covers_every_position_once():
             assert parts[0][0] == 0 and parts[-1][1] == (t + 15) // 16
             assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
             assert sum(p[2] for p in parts) == t
+
+
+def _bench_mode_worker(rank, world, port, ret):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    from paper_2609_20734_b200 import sharded_bench, sharding, workloads
+
+    res = {}
+    for shard, name in (("heads", "llama8b"), ("sequence", "batched")):
+        # the same argument path as `bench.py --gpus 2 --shard ...`
+        args = bench.parse(["--gpus", str(world), "--shard", shard, "--config", name, "--steps", "4", "--warmup", "3"])
+        wl = workloads.make(args.config)
+        mine, info = sharded_bench.plan(wl, shard, rank, world)
+        infos = [None] * world
+        dist.all_gather_object(infos, info)
+        total_ms = sharding.max_over_ranks(10.0 * (rank + 1))       # the slowest rank's time counts
+        line = sharded_bench.line(bench, args, wl, shard, world, total_ms, 1e9, 3, {}) if rank == 0 else None
+        res[shard] = (mine, infos, line)
+    ret[rank] = res
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_bench_shard_modes_two_ranks_gloo():
+    """`bench.py --shard heads|sequence`: what each rank holds tiles the workload exactly once, and rank 0's
+    line has the contract's keys with the slowest rank's time (the timed half needs one GPU per rank)."""
+    world = 2
+    with mp.Manager() as m:
+        ret = m.dict()
+        mp.spawn(_bench_mode_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
+        res = dict(ret)
+    from paper_2609_20734_b200 import workloads
+
+    wl = workloads.make("llama8b")
+    mine0, infos, line = res[0]["heads"]
+    assert [i["kv_heads"] for i in infos] == [[0, 4], [4, 8]]
+    assert [i["w1_columns"] for i in infos] == [[0, 2048], [2048, 4096]] and infos[0]["d_in"] == 4096
+    assert infos[0]["exchange_bytes_per_step"] == wl.B * 256 * 4
+    assert sum(res[r]["heads"][0].kv_token_bytes for r in range(world)) == wl.kv_token_bytes
+    assert (mine0.Hq, mine0.Hkv) == (16, 4) and res[1]["heads"][0].seed != mine0.seed
+    assert line["scaling"] == "strong" and line["n_gpus"] == 2 and line["ms_per_step"] == 20.0 / 4
+    assert line["value"] == wl.B * 4 / 20e-3 and line["config"]["parallelism"].startswith("tp2")
+    assert line["config"]["global_batch"] == wl.B and "llama8b" in line["config"]["workload"]
+    wl = workloads.make("batched")
+    _, infos, line = res[0]["sequence"]
+    lens = np.asarray(wl.seq_lens0)
+    assert (np.asarray(infos[0]["tokens_held"]) + np.asarray(infos[1]["tokens_held"]) == lens).all()
+    for b in range(wl.B):
+        (a0, a1), (b0, b1) = infos[0]["pages"][b], infos[1]["pages"][b]
+        assert a0 == 0 and a1 == b0 and b1 == (int(lens[b]) + 15) // 16
+    assert line["config"]["parallelism"].startswith("sp2") and line["shard"] == "sequence"
+    for key in ("metric", "value", "unit", "steps", "warmup", "higher_is_better", "vs_baseline", "dtype", "data", "gpu_launches"):
+        assert key in line

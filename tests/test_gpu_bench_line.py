@@ -13,7 +13,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def test_bench_prints_one_contract_line():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "8", "--warmup", "3", "--no-sweep",
-                        "--kernel-reps", "2"], capture_output=True, text=True, timeout=900, cwd=ROOT)
+                        "--kernel-reps", "2", "--configs", "tiny", "--no-paper-head"], capture_output=True, text=True, timeout=900, cwd=ROOT)
     assert r.returncode == 0, r.stderr[-2000:]
     lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
     assert len(lines) == 1
@@ -37,4 +37,13 @@ def test_bench_prints_one_contract_line():
     cpu = d["cpu_baseline"]
     assert cpu["kind"] == "oracle" and cpu["cores"] >= 1 and cpu["value"] > 0 and cpu["sample"]
     clk = d["clocks"]
-    assert clk["sm_max_mhz"] >= clk["sm_mhz"] > 0 and isinstance(clk["reasons"], list)
+    assert clk["sm_max_mhz"] >= clk["sm_mhz"] > 0 and isinstance(clk["reasons"], list) and clk["samples"] >= 10
+    # three measured passes, the median one is the headline
+    ps = d["passes"]
+    assert ps["measured"] == 3 and sorted(ps["ms_per_step"])[1] == d["ms_per_step"]
+    assert d["roofline_other"]["floor_us"] > 0 and d["roofline_other"]["frac_above_floor"] > d["roofline_other"]["frac"]
+    # the arm-specific descriptions sit beside `config`, which both arms fill identically
+    assert "launch" in d and "arithmetic" in d and "launch" not in d["config"]
+    (tiny,) = d["configs"]
+    assert tiny["name"] == "tiny" and tiny["recall_rate_realised"] == 0.25 and tiny["tokens_per_s"] > 0
+    assert tiny["head"]["us"] > 0 and tiny["local"]["us"] > 0 and tiny["full"]["us"] > 0
