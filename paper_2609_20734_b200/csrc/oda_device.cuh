@@ -74,6 +74,17 @@ struct AttnParams {
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Loads of the small arrays a launch starts from (lengths, layer table, block-table entries), as
+// volatile asm so that they are issued where they are written: early, ahead of the set-up code
+// whose latency they overlap.  (An L2 evict-last hint on them was measured and changes nothing: the
+// Local pass of the batch-1 benchmark shape reads 35.4 us with it and 35.4 us without.)
+__device__ __forceinline__ int32_t ld_meta_s32(const int32_t* ptr)
+{
+    int32_t v;
+    asm volatile("ld.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr));
+    return v;
+}
+
 // Work decomposition.  A unit is one (layer, request, kv head); it owns np pages of KV (the
 // pages of its Eq. 1 window segment, or of the whole history in Full mode; requests that are not
 // flagged and layers that are not gated own none).  All units are laid end to end, layer-major
@@ -513,6 +524,54 @@ __device__ __forceinline__ int span_of_near(const Plan& pl, int x, int j, int di
         if (span_begin(pl, mid) <= x) lo = mid; else hi = mid;
     }
     return lo;
+}
+
+// Batch 1, one unit per CTA (see build_plan): what the plan boils down to, from three registers.
+struct DirectPlan {
+    int32_t ok;          // the launch falls under the one-unit-per-CTA rule
+    int32_t t, cls, kv_index;
+};
+
+// The rule of build_plan's batch-1 branch, evaluated from the one length.
+__device__ __forceinline__ bool direct_rule(const AttnParams& p, int t)
+{
+    if (t < 1 || t > p.max_blocks_per_seq * kPage) return false;  // the general path reports these
+    const int g = (int)gridDim.x, H = p.num_kv_heads;
+    long long total = 0;
+    int umin = 0x7fffffff, umax = 0;
+    for (int c = 0; c < p.ncls; ++c) {
+        if (p.cls_layers_in_call[c] <= 0) continue;
+        const Ranges r = eq1_ranges(0, t, p.cls_window[c], p.cls_sinks[c]);
+        const int np = r.pg1 - r.pg0;
+        total += (long long)p.cls_layers_in_call[c] * H * np;
+        umin = min(umin, np);
+        umax = max(umax, np);
+    }
+    const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
+    return total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
+           (long long)umin * g >= total && 2ll * umax * g <= 3 * total;
+}
+
+// Unit j = (layer j / H, kv head j % H) of the only request.
+__device__ __forceinline__ void decode_item_direct(const AttnParams& p, const DirectPlan& d, int j, Item& it)
+{
+    const int H = p.num_kv_heads;
+    const int lo = j / H;
+    const Ranges rg = eq1_ranges(0, d.t, p.cls_window[d.cls], p.cls_sinks[d.cls]);
+    it.layer = p.layer_begin + lo;
+    it.b = 0;
+    it.g = j - lo * H;
+    it.chunk = 0;
+    it.nchunks = 1;
+    it.slot_base = 0;
+    it.kv_layer = d.kv_index;
+    it.t = d.t;
+    it.win_pg0 = rg.pg0;
+    it.win_pg1 = rg.pg1;
+    it.win_lo = rg.lo;
+    it.win_hi = rg.hi;
+    it.sink_hi = rg.sink_hi;
+    it.sink_pg1 = (it.sink_hi + kPage - 1) / kPage;
 }
 
 // The item of span j that starts at axis page x (x0 <= x < x_end of span_range(j)).

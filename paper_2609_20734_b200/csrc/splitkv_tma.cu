@@ -178,6 +178,22 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) ODA_TL(0);
+#ifdef ODA_TIMELINE
+    if (tid == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); g_timeline[blockIdx.x * 8 + 7] = sm_; }
+#endif
+    // Batch-1 Local launch that may give every CTA one whole unit: the one length and this CTA's layer
+    // entry are requested first thing (after the dependency wait, which such a launch takes at once:
+    // it is the first kernel of a step), so that their latency runs while the barriers are set up.
+    const bool direct_try = p.direct_hint && !p.sm_stats;
+    DirectPlan dp;
+    dp.ok = dp.t = dp.cls = dp.kv_index = 0;
+    if (direct_try) {
+        griddep_wait();
+        const LayerInfo* lp = p.layers + p.layer_begin + min((int)blockIdx.x / p.num_kv_heads, p.layer_end - p.layer_begin - 1);
+        dp.t = ld_meta_s32(p.seq_lens);
+        dp.cls = ld_meta_s32(&lp->cls);
+        dp.kv_index = ld_meta_s32(&lp->kv_index);
+    }
     if (tid == 0) {
         for (int s = 0; s < C::kStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
@@ -191,18 +207,25 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&vmap)) : "memory");
     }
     prefetch_block_table(p);
-    griddep_wait();       // everything above is independent of the previous kernel in the stream
+    __syncthreads();      // the barriers are initialised for every warp
+    if (!direct_try) griddep_wait();  // everything above is independent of the previous kernel in the stream
     if (tid == 0) ODA_TL(1);
-    if (gated_pass_is_empty(p)) {
-        griddep_launch_dependents();
-        return;
+    if (direct_try) dp.ok = direct_rule(p, dp.t);  // same registers in every thread: no barrier, no shared plan
+    int span;             // the one span this CTA streams
+    if (dp.ok) {
+        span = (int)blockIdx.x < (p.layer_end - p.layer_begin) * p.num_kv_heads ? (int)blockIdx.x : -1;
+    } else {
+        if (gated_pass_is_empty(p)) {
+            griddep_launch_dependents();
+            return;
+        }
+        build_plan(p, plan);  // ends with a barrier
+        span = plan.my_span;
     }
-    build_plan(p, plan);  // ends with a barrier
     griddep_launch_dependents();
     if (tid == 0) ODA_TL(2);
     volatile int* abort_flag = &ctl.abort;
     constexpr uint32_t kQBytes = G * D * 2;
-    const int span = plan.my_span;  // the one span this CTA streams
     if (span < 0) return;
 
     if (warp == C::kProducerWarp) {
@@ -212,10 +235,14 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         uint32_t cnt = 0;
         bool dead = false;
         // walker over the runs of the CTA's span
-        int x, x_end;
-        span_range(plan, span, x, x_end);
+        int x = 0, x_end = 1, take = 1;  // a one-unit-per-CTA span is [0, 1) on a nominal axis
         Item it;
-        int take = decode_item(p, plan, span, x, x_end, it);
+        if (dp.ok) {
+            decode_item_direct(p, dp, span, it);
+        } else {
+            span_range(plan, span, x, x_end);
+            take = decode_item(p, plan, span, x, x_end, it);
+        }
         int v = 0, nv = item_pages(it);  // next page of the item in streaming order, pages it has
         bool more = true, item_first = true;
         auto fetch = [&](PageRun& r, int& blk) -> bool {  // next run and its block ids; false when the span is done
@@ -490,8 +517,8 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     uint64_t t_first = 0, t_half = 0;
     int pages_done = 0, pages_half = 0;
     {
-        int x, x_end;
-        span_range(plan, span, x, x_end);
+        int x = 0, x_end = 1;
+        if (!dp.ok) span_range(plan, span, x, x_end);
         span_pages = x_end - x;
 #ifdef ODA_TIMELINE
         long long a_dec = 0, a_first = 0, a_tiles = 0, a_wait = 0, a_merge = 0, a_items = 0;
