@@ -624,10 +624,13 @@ def extra_config(torch, args, name, steps, flush, side, peak):
 
 
 def paper_head_section(torch, args, flush, side):
-    """The paper's 28,325,889-parameter recall head on the headline configuration: the head call
-    alone, and what it adds to an all-Local step (recall rate 0), i.e. the time between the end of
-    the Local pass and the flags being ready."""
-    from paper_2609_20734_b200 import binding, workloads
+    """The paper's 28,325,889-parameter recall head on the headline configuration at recall rate 0:
+    the head call alone, and what it adds to an all-Local step (the time between the end of the Local
+    pass and the flags being ready) in three arrangements -- the whole head after the Local pass; its
+    first part (what needs only h_{t-1} and E(x_t)) run ahead, outside the timed step, as a backbone
+    with other work between two steps can; and that first part forked beside the Local pass inside
+    the step's own graph."""
+    from paper_2609_20734_b200 import workloads
 
     dm, T, F, nb = 2048, 1024, 2048, 2
     wl = workloads.make(args.config, recall_rate=0.0)
@@ -635,27 +638,73 @@ def paper_head_section(torch, args, flush, side):
     params = torch.from_numpy(workloads.full_head_params(wl.seed, dm, T, F, nb)).cuda()
     x = [torch.from_numpy(workloads.full_head_input(wl.seed, i, B, dm)).cuda() for i in range(3)]
     steps = 16
+
+    def med_step_ms(run):
+        return float(np.median([np.mean(run.one_pass()) for _ in range(3)]))
+
     base = Runner(torch, args, wl, flush, side, steps=steps, warmup=3, calibrate=False)
-    t_base = float(np.median([np.mean(base.one_pass()) for _ in range(3)]))
+    t_base = med_step_ms(base)
     scratch = base.ctx.full_head_scratch(B, dm, T, F, nb)
     scores = torch.zeros(B, device="cuda")
     flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
     g_head = capture(torch, side, lambda s_: base.ctx.recall_score_full(
         B, params, T, F, nb, x[0], x[1], x[2], 0.5, None, scores, None, flags, scratch=scratch, stream=s_))
+    g_pre = capture(torch, side, lambda s_: base.ctx.recall_score_full_pre(
+        B, params, T, F, nb, x[0], x[1], scratch, stream=s_))
+    g_post = capture(torch, side, lambda s_: base.ctx.recall_score_full(
+        B, params, T, F, nb, x[0], x[1], x[2], 0.5, None, scores, None, flags, scratch=scratch, stream=s_, variant=3))
     torch.cuda.synchronize()
-    t_head = [timed_replay(torch, g_head, flush, r) for r in range(args.kernel_reps + 2)][2:]
+    reps = args.kernel_reps + 2
+    t_head = [timed_replay(torch, g_head, flush, r) for r in range(reps)][2:]
+    t_pre = [timed_replay(torch, g_pre, flush, r) for r in range(reps)][2:]
+    t_post = [timed_replay(torch, g_post, flush, r) for r in range(reps)][2:]
     base.close()
+    res = {"parameters": int(params.numel()), "weight_bytes": int(params.numel()) * 4, "batch": B,
+           "call_alone_us": float(np.mean(t_head)) * 1e3,
+           "call_alone_gbs": params.numel() * 4 / (float(np.mean(t_head)) * 1e-3) / 1e9,
+           "first_part_alone_us": float(np.mean(t_pre)) * 1e3, "second_part_alone_us": float(np.mean(t_post)) * 1e3,
+           "all_local_step_ms": t_base}
     fh = dict(params=params, d_tower=T, d_ff=F, n_blocks=nb, h_prev=x[0], emb=x[1], h_local=x[2], scratch=scratch)
-    withh = Runner(torch, args, wl, flush, side, steps=steps, warmup=3, calibrate=False, paper_head=fh)
-    t_with = float(np.median([np.mean(withh.one_pass()) for _ in range(3)]))
-    launches = withh.launches_per_step
-    withh.close()
-    return {"parameters": int(params.numel()), "weight_bytes": int(params.numel()) * 4, "batch": B,
-            "call_alone_us": float(np.mean(t_head)) * 1e3,
-            "call_alone_gbs": params.numel() * 4 / (float(np.mean(t_head)) * 1e-3) / 1e9,
-            "all_local_step_ms": t_base, "all_local_step_with_head_ms": t_with,
-            "added_to_step_us": (t_with - t_base) * 1e3, "launches_per_step_with_head": launches,
-            "note": "recall rate 0, forced flags; the step without it publishes the forced flags from the gated pass"}
+    # (1) the whole head after the Local pass
+    r1 = Runner(torch, args, wl, flush, side, steps=steps, warmup=3, calibrate=False, paper_head=fh)
+    t1 = med_step_ms(r1)
+    res["launches_per_step_with_head"] = r1.launches_per_step
+    r1.close()
+    # (2) first part ahead of the step (untimed, like the input copies), second part in the step
+    r2 = Runner(torch, args, wl, flush, side, steps=steps, warmup=3, calibrate=False, paper_head=dict(fh, variant=3))
+    plain_set_inputs = r2.set_inputs
+
+    def set_inputs_and_first_part(s):
+        plain_set_inputs(s)
+        r2.ctx.recall_score_full_pre(B, params, T, F, nb, x[0], x[1], scratch)
+    r2.set_inputs = set_inputs_and_first_part
+    t2 = med_step_ms(r2)
+    # (3) the same two parts inside one graph, the first on a branch forked beside the Local pass
+    ctx, st = r2.ctx, r2.st
+    side2 = torch.cuda.Stream()
+
+    def forked_step(s_):
+        main = torch.cuda.ExternalStream(s_)
+        side2.wait_stream(main)
+        ctx.local_decode(0, wl.L, B, r2.q_s, st.k_cache, st.v_cache, st.block_table, st.seq_lens, r2.out, r2.lse, stream=s_)
+        ctx.recall_score_full_pre(B, params, T, F, nb, x[0], x[1], scratch, stream=side2.cuda_stream)
+        main.wait_stream(side2)
+        ctx.recall_score_full(B, params, T, F, nb, x[0], x[1], x[2], 0.5, r2.ov_s, r2.scores, None, r2.flags,
+                              scratch=scratch, stream=s_, variant=3)
+        ctx.full_decode_gated(0, wl.L, B, r2.q_s, st.k_cache, st.v_cache, st.block_table, st.seq_lens, r2.flags,
+                              r2.out, r2.lse, stream=s_)
+    r2.graph = capture(torch, side, forked_step)
+    r2.set_inputs = plain_set_inputs
+    torch.cuda.synchronize()
+    t3 = float(np.median([np.mean(r2.run_steps(3, steps, True)) for _ in range(3)]))
+    r2.close()
+    res.update({"all_local_step_with_head_ms": t1, "added_to_step_us": (t1 - t_base) * 1e3,
+                "added_to_step_first_part_ahead_us": (t2 - t_base) * 1e3,
+                "added_to_step_first_part_forked_beside_local_us": (t3 - t_base) * 1e3,
+                "note": "recall rate 0, forced flags; the step without a head publishes the forced flags from the gated "
+                        "pass.  first_part_ahead: towers a, b and their four segments of the fusion product computed "
+                        "before the timed step (Eq. 2: h_{t-1} and E(x_t) exist before the Local pass)"})
+    return res
 
 
 def main():

@@ -300,11 +300,23 @@ oda_status_t oda_merge_partials_exchange(oda_ctx_t* ctx, int32_t world, int32_t 
  * barriers (a barrier that times out after ~1 s sets bit 2 of the device status word and the kernel
  * returns).  It is kept as the measured alternative: on a B200 it is slower than the stage launches
  * (80 vs 59 us at batch 1).  Both are deterministic; they differ in summation order only.
+ *
+ * Two of the head's three inputs exist before the step's Local pass (Eq. 2: q_t = R(h_{t-1}, E(x_t),
+ * h_t^L)), so the head can be run in two parts.  oda_recall_score_full_pre computes what needs only
+ * h_prev and emb -- towers a and b and the four segments (a, b, a.b, |a-b|) of W_f u -- and leaves
+ * it in the scratch; oda_recall_score_full with variant 3 on the same scratch then computes tower c,
+ * the remaining five segments, the blocks and the output.  The sum W_f u is then taken in the order
+ * (first part) + (second part): scores may differ from variants 0-2 in the last bits.  The first part
+ * can run whenever the caller has room for it between two steps -- beside the backbone's other work,
+ * on another stream -- and oda_step given a full_head with variant 3 then pays only for the second
+ * part after its Local pass.  (Beside a Local pass that already saturates DRAM there is no room: on
+ * a B200 the batch-1 benchmark step gets slower when the first part is forked next to it.)
  */
 typedef struct {
     int32_t d_model, d_tower, d_ff, n_blocks;
     float eps;      /* RMSNorm epsilon (the paper does not print it; 1e-6 is customary) */
-    int32_t variant; /* 0 = auto (= 1), 1 = one launch per stage, 2 = one persistent kernel (batch <= 4) */
+    int32_t variant; /* 0 = auto (= 1), 1 = one launch per stage, 2 = one persistent kernel (batch <= 4),
+                        3 = second part only, after oda_recall_score_full_pre on the same scratch */
     const float* params;
 } oda_full_head_t;
 int64_t oda_full_head_param_count(int32_t d_model, int32_t d_tower, int32_t d_ff, int32_t n_blocks);
@@ -314,6 +326,11 @@ oda_status_t oda_recall_score_full(oda_ctx_t* ctx, int32_t batch, const oda_full
                                    float threshold, const uint8_t* override_flags, float* scores,
                                    float* logits, uint8_t* flags, int32_t* counters, void* scratch,
                                    size_t scratch_bytes, void* stream);
+/* First part of the paper's head (see above): needs neither the Local hidden state nor a threshold;
+ * writes only into scratch.  Two stage launches after one memset. */
+oda_status_t oda_recall_score_full_pre(oda_ctx_t* ctx, int32_t batch, const oda_full_head_t* head,
+                                       const float* h_prev, const float* emb, void* scratch,
+                                       size_t scratch_bytes, void* stream);
 
 /*
  * Gated Full pass (Eq. 1, S^F; Algorithm 1, line 4): for gated layers in [layer_begin,

@@ -26,7 +26,7 @@ EXPORTS = [
     "oda_local_decode_static_status",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
     "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
-    "oda_recall_score_full", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
+    "oda_recall_score_full", "oda_recall_score_full_pre", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
     "oda_recall_finalize_exchange", "oda_merge_partials_exchange", "oda_set_cache_resident_bytes",
 ]
 
@@ -139,6 +139,7 @@ def load_library():
         lib.oda_full_head_scratch_bytes.restype = ctypes.c_size_t
         lib.oda_recall_score_full.argtypes = [vp, i32, ctypes.POINTER(_FullHead), vp, vp, vp, f32, vp, vp, vp, vp,
                                               vp, vp, ctypes.c_size_t, vp]
+        lib.oda_recall_score_full_pre.argtypes = [vp, i32, ctypes.POINTER(_FullHead), vp, vp, vp, ctypes.c_size_t, vp]
         lib.oda_calibration_begin.argtypes = [vp, vp]
         lib.oda_calibration_end.argtypes = [vp, vp]
         lib.oda_calibration_spread.argtypes = [vp]
@@ -359,6 +360,15 @@ class OdaContext:
             _ptr(override_flags), _ptr(scores), _ptr(logits), _ptr(flags), _ptr(counters), _ptr(scratch),
             scratch.numel(), _stream() if stream is None else stream), "oda_recall_score_full")
         return scratch
+
+    def recall_score_full_pre(self, batch, params, d_tower, d_ff, n_blocks, h_prev, emb, scratch, eps=1e-6,
+                              stream=None):
+        """First part of the paper's head (towers a, b and their share of the fusion product), left in
+        `scratch` for a recall_score_full(..., variant=3) on the same scratch."""
+        head = _FullHead(h_prev.shape[1], d_tower, d_ff, n_blocks, eps, 0, _ptr(params))
+        self._check(self.lib.oda_recall_score_full_pre(
+            self._h, batch, ctypes.byref(head), _ptr(h_prev), _ptr(emb), _ptr(scratch), scratch.numel(),
+            _stream() if stream is None else stream), "oda_recall_score_full_pre")
 
     def full_head_scratch(self, batch, d_model, d_tower, d_ff, n_blocks, device="cuda"):
         """A scratch tensor large enough for the paper's head at this batch."""

@@ -794,7 +794,7 @@ oda_status_t oda_recall_score_full(oda_ctx_t* c, int32_t batch, const oda_full_h
         return fail(c, ODA_ERR_UNSUPPORTED, "d_model and d_ff must be multiples of 4, d_tower of 8");
     if (!h->params || !h_prev || !emb || !h_local || !scores || !flags || !scratch)
         return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
-    if (h->variant < 0 || h->variant > 2) return fail(c, ODA_ERR_INVALID_ARG, "head variant outside 0..2");
+    if (h->variant < 0 || h->variant > 3) return fail(c, ODA_ERR_INVALID_ARG, "head variant outside 0..3");
     if (!aligned16(h->params) || !aligned16(h_prev) || !aligned16(emb) || !aligned16(h_local) ||
         (reinterpret_cast<uintptr_t>(scratch) % 256) != 0)
         return fail(c, ODA_ERR_INVALID_ARG, "parameters and inputs must be 16-byte aligned, scratch 256-byte aligned");
@@ -803,14 +803,40 @@ oda_status_t oda_recall_score_full(oda_ctx_t* c, int32_t batch, const oda_full_h
     int launches = 0;
     cudaError_t e = launch_full_head(batch, h->d_model, h->d_tower, h->d_ff, h->n_blocks, h->eps, h->params, h_prev,
                                      emb, h_local, threshold, override_flags, scores, logits, flags, counters,
-                                     scratch, static_cast<cudaStream_t>(stream), c->use_pdl, &launches, h->variant,
-                                     c->ws ? reinterpret_cast<int32_t*>(c->ws + c->lay.status) : nullptr);
+                                     scratch, static_cast<cudaStream_t>(stream), c->use_pdl, &launches,
+                                     h->variant == 3 ? 0 : h->variant,
+                                     c->ws ? reinterpret_cast<int32_t*>(c->ws + c->lay.status) : nullptr,
+                                     h->variant == 3 ? 2 : 0);
     c->launches += launches;
     if (e == cudaErrorNotSupported) {
         (void)cudaGetLastError();
         return fail(c, ODA_ERR_UNSUPPORTED, "the fused head needs batch <= 4 and a device that can hold one CTA per SM cooperatively");
     }
     if (e != cudaSuccess) return cuda_fail(c, e, "full recall head launch");
+    return ODA_OK;
+}
+
+oda_status_t oda_recall_score_full_pre(oda_ctx_t* c, int32_t batch, const oda_full_head_t* h, const float* h_prev,
+                                       const float* emb, void* scratch, size_t scratch_bytes, void* stream)
+{
+    if (!c || !h) return ODA_ERR_INVALID_ARG;
+    if (batch < 0 || batch > kMaxBatch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, 128]");
+    if (batch == 0) return ODA_OK;
+    if (h->d_model < 4 || h->d_tower < 8 || h->d_ff < 4 || h->n_blocks < 0 || !(h->eps >= 0.f))
+        return fail(c, ODA_ERR_INVALID_ARG, "bad head dimensions");
+    if ((h->d_model % 4) || (h->d_tower % 8) || (h->d_ff % 4))
+        return fail(c, ODA_ERR_UNSUPPORTED, "d_model and d_ff must be multiples of 4, d_tower of 8");
+    if (!h->params || !h_prev || !emb || !scratch) return fail(c, ODA_ERR_INVALID_ARG, "null pointer");
+    if (!aligned16(h->params) || !aligned16(h_prev) || !aligned16(emb) || (reinterpret_cast<uintptr_t>(scratch) % 256) != 0)
+        return fail(c, ODA_ERR_INVALID_ARG, "parameters and inputs must be 16-byte aligned, scratch 256-byte aligned");
+    if (scratch_bytes < full_head_scratch_bytes(h->d_model, h->d_tower, h->d_ff, batch))
+        return fail(c, ODA_ERR_WORKSPACE, "scratch smaller than oda_full_head_scratch_bytes()");
+    int launches = 0;
+    cudaError_t e = launch_full_head(batch, h->d_model, h->d_tower, h->d_ff, h->n_blocks, h->eps, h->params, h_prev,
+                                     emb, nullptr, 0.f, nullptr, nullptr, nullptr, nullptr, nullptr, scratch,
+                                     static_cast<cudaStream_t>(stream), c->use_pdl, &launches, 0, nullptr, 1);
+    c->launches += launches;
+    if (e != cudaSuccess) return cuda_fail(c, e, "full recall head (first part) launch");
     return ODA_OK;
 }
 
@@ -851,6 +877,8 @@ oda_status_t oda_step(oda_ctx_t* c, const oda_step_args_t* a, void* stream)
     const bool fused_decision = !paper_head && f.head_d_hidden == 0 && c->last_gated >= 0;
     const uint8_t* decided = fused_decision ? a->override_flags : a->flags;  // valid once the head (if any) has run
     if (paper_head) {
+        // (variant 3: the caller has run oda_recall_score_full_pre on head_scratch since the last step;
+        // only the part that needs the Local hidden state is left for after the Local pass)
         s = oda_recall_score_full(c, B, a->full_head, a->head_h_prev, a->head_emb, a->head_h_local, a->threshold,
                                   a->override_flags, a->scores, a->logits, a->flags, a->counters, a->head_scratch,
                                   a->head_scratch_bytes, stream);

@@ -27,7 +27,7 @@ cudaError_t launch_full_head(int batch, int d_model, int d_tower, int d_ff, int 
                              const float* params, const float* h_prev, const float* emb, const float* h_local,
                              float threshold, const uint8_t* override_flags, float* scores, float* logits,
                              uint8_t* flags, int32_t* counters, void* scratch, cudaStream_t st, bool pdl,
-                             int* launches, int variant, int32_t* status);
+                             int* launches, int variant, int32_t* status, int phase = 0);
 // the same head as one persistent cooperative kernel (batch <= kFullHeadFusedMaxBatch)
 constexpr int kFullHeadFusedMaxBatch = 4;
 constexpr int kFullHeadFusedSmem = 230400;    // dynamic shared memory of the fused head (stage input + ring + control)

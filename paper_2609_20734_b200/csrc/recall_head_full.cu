@@ -25,7 +25,12 @@ enum { kStageTower = 0, kStageFusion = 1, kStageGateUp = 2, kStageDown = 3, kSta
 
 struct FullStageParams {
     int32_t stage, batch, T, F, d_model;
-    int32_t K;                   // reduction length of this stage
+    int32_t K;                   // reduction length of this stage (fusion: of the segments this launch covers)
+    int32_t w_stride;            // floats between consecutive weight rows (fusion: always 9 T)
+    int32_t tower_base;          // tower stage: blockIdx.z = 0 is this tower
+    int32_t fus_part;            // fusion stage: 0 all nine segments of u; 1 the four that need only a and b
+                                 // (a, b, a.b, |a-b|), raw sums to `out`; 2 the five that need c, added to `fpre`
+    const float* fpre;           // fus_part 2: the sums of part 1, [B][T]
     int32_t row_blocks;
     float eps;
     const float* W;              // towers: W of tower 0 (+ i * tower_stride); gate+up: W_gate, W_up = W + F*T
@@ -49,6 +54,18 @@ struct FullStageParams {
 
 __device__ __forceinline__ float silu_f(float a) { return a / (1.f + expf(-a)); }
 
+// Fusion stage over a subset of the nine segments of u: position k of the launch's own numbering
+// -> position in u (and in a row of W_f).  Segments are T long and T % 4 == 0, so four consecutive
+// positions never straddle two segments.
+__device__ __forceinline__ int fusion_k(const FullStageParams& p, int k)
+{
+    if (p.fus_part == 0) return k;
+    const int s = k / p.T, j = k - s * p.T;
+    // part 1: a, b, a.b, |a-b| = segments 0, 1, 3, 4;  part 2: c, a.c, |a-c|, b.c, |b-c| = 2, 5, 6, 7, 8
+    const int seg = p.fus_part == 1 ? (s < 2 ? s : s + 1) : (s == 0 ? 2 : s + 4);
+    return seg * p.T + j;
+}
+
 // four consecutive elements k..k+3 (k % 4 == 0) of the stage input of request b
 __device__ __forceinline__ float4 stage_x4(const FullStageParams& p, int tower, int b, int k)
 {
@@ -58,6 +75,7 @@ __device__ __forceinline__ float4 stage_x4(const FullStageParams& p, int tower, 
     }
     if (p.stage == kStageFusion) {
         // u = [a; b; c; a.b; |a-b|; a.c; |a-c|; b.c; |b-c|]
+        k = fusion_k(p, k);
         const int seg = k / p.T, j = k - seg * p.T;
         const float* abc = p.in0;
         const size_t row = (size_t)b * p.T + j, plane = (size_t)p.batch * p.T;
@@ -81,7 +99,12 @@ __device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, in
         p.out[((size_t)i * p.batch + b) * p.T + j] = silu_f(acc * rs + __ldg(p.bias + i * p.tower_stride + j));
     } else if (p.stage == kStageFusion) {
         const size_t row = (size_t)b * p.T + r, plane = (size_t)p.batch * p.T;
-        p.out[row] = 0.5f * (p.in0[row] + p.in0[plane + row] + p.in0[2 * plane + row] + silu_f(acc + __ldg(p.bias + r)));
+        if (p.fus_part == 1) {
+            p.out[row] = acc;   // the share of W_f u that needs only a and b
+        } else {
+            if (p.fus_part == 2) acc = p.fpre[row] + acc;   // fixed order: the earlier share first
+            p.out[row] = 0.5f * (p.in0[row] + p.in0[plane + row] + p.in0[2 * plane + row] + silu_f(acc + __ldg(p.bias + r)));
+        }
     } else if (p.stage == kStageGateUp) {
         p.out[(size_t)b * p.F + r] = silu_f(acc * rs) * (acc_up * rs);
     } else if (p.stage == kStageDown) {
@@ -122,7 +145,7 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ks = blockIdx.y, n_ks = gridDim.y;
-    const int tower = p.stage == kStageTower ? (int)blockIdx.z : 0;
+    const int tower = p.stage == kStageTower ? p.tower_base + (int)blockIdx.z : 0;
     const int k0 = ks * kFKT;
     const int n_rows = p.stage == kStageTower ? 3 * p.T : (p.stage == kStageGateUp ? 2 * p.F : (p.stage == kStageOut ? 1 : p.T));
     const int out_rows = p.stage == kStageGateUp ? kFRows / 2 : kFRows;
@@ -147,11 +170,12 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
     auto load_w = [&](float4 (&w)[kWC], int rb) {
         bool ok;
         const int n = row_of(rb, ok);
-        const float* wrow = wbase + (size_t)(n - group_row0) * p.K;
+        const float* wrow = wbase + (size_t)(n - group_row0) * p.w_stride;
 #pragma unroll
         for (int c = 0; c < kWC; ++c) {
             const int k = k0 + c * 128 + lane * 4;
-            w[c] = (ok && k < p.K) ? __ldg(reinterpret_cast<const float4*>(wrow + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const int kw = p.stage == kStageFusion ? fusion_k(p, k) : k;
+            w[c] = (ok && k < p.K) ? __ldg(reinterpret_cast<const float4*>(wrow + kw)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     };
     for (int b0 = 0; b0 < p.batch; b0 += kFBT) {
@@ -307,9 +331,9 @@ long long full_head_param_count(int d_model, int T, int F, int n_blocks)
 static int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 constexpr int kFKT = 512;  // the narrower tile: what the scratch is sized for
 
-// scratch layout (floats unless noted): abc [3][B][T] | z [B][T] | h [B][F] | pre | ssq | tickets (int32)
+// scratch layout (floats unless noted): abc [3][B][T] | z [B][T] | h [B][F] | fpre [B][T] | pre | ssq | tickets (int32)
 struct FullScratch {
-    size_t abc, z, h, pre, ssq, tickets, total;
+    size_t abc, z, h, fpre, pre, ssq, tickets, total;
 };
 
 static FullScratch full_scratch_layout(int d_model, int T, int F, int batch)
@@ -321,6 +345,7 @@ static FullScratch full_scratch_layout(int d_model, int T, int F, int batch)
     s.abc = off; off = al(off + 3 * B * T * 4);
     s.z = off; off = al(off + B * T * 4);
     s.h = off; off = al(off + B * F * 4);
+    s.fpre = off; off = al(off + B * T * 4);
     // pre: max over stages of k slices * rows
     const size_t pre_rows = std::max({(size_t)ceil_div(d_model, kFKT) * 3 * T, (size_t)ceil_div(9ll * T, kFKT) * T,
                                       (size_t)ceil_div(T, kFKT) * 2 * F, (size_t)ceil_div(F, kFKT) * T});
@@ -343,13 +368,18 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
                              const float* h_prev, const float* emb, const float* h_local, float threshold,
                              const uint8_t* override_flags, float* scores, float* logits, uint8_t* flags,
                              int32_t* counters, void* scratch, cudaStream_t st, bool pdl, int* launches, int variant,
-                             int32_t* status)
+                             int32_t* status, int phase)
 {
+    // phase 0: the whole head.  phase 1: what does not need the Local hidden state -- towers a and b
+    // and their four segments of the fusion product -- left in the scratch.  phase 2: the rest, on top
+    // of a phase 1 that ran on the same scratch: tower c, the five segments that need c, the blocks, the
+    // output.  1 + 2 sum the fusion product in a different (fixed) order than 0: last bits may differ.
     char* sc = static_cast<char*>(scratch);
     const FullScratch L = full_scratch_layout(d_model, T, F, batch);
     // variant 2: the whole chain as one persistent kernel (measured slower than the stage launches, so
     // 0 = auto picks the stage launches; see recall_head_fused.cu)
     const long long x_floats = full_head_fused_x_floats(batch, d_model, T, F);
+    if (variant == 2 && phase != 0) return cudaErrorNotSupported;
     const int fused_grid = (variant == 2 && batch <= kFullHeadFusedMaxBatch && x_floats * 4 + 1024 + 8 * 4096 <= kFullHeadFusedSmem)
                                ? full_head_fused_grid() : 0;
     if (variant == 2 && fused_grid == 0) return cudaErrorNotSupported;
@@ -370,23 +400,29 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
     float* abc = reinterpret_cast<float*>(sc + L.abc);
     float* z = reinterpret_cast<float*>(sc + L.z);
     float* h = reinterpret_cast<float*>(sc + L.h);
-    cudaError_t e = cudaMemsetAsync(sc + L.tickets, 0, L.total - L.tickets, st);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (phase != 2) {  // phase 2 finds the tickets as phase 1 left them: every one back at zero
+        e = cudaMemsetAsync(sc + L.tickets, 0, L.total - L.tickets, st);
+        if (e != cudaSuccess) return e;
+    }
     FullStageParams p = {};
     p.batch = batch; p.T = T; p.F = F; p.d_model = d_model; p.eps = eps;
     p.pre = reinterpret_cast<float*>(sc + L.pre);
     p.ssq = reinterpret_cast<float*>(sc + L.ssq);
     p.rb_tickets = reinterpret_cast<int32_t*>(sc + L.tickets);
+    int n_towers = 3;
     auto launch = [&](bool dep) {
         // small batches: a 2048-wide k tile (one CTA per SM) where that divides k (towers, down: no
         // split over k), else a 1024-wide one (gate+up fits it whole; the fusion's k = 9 x 1024 splits
         // evenly): two CTAs per SM.  Measured: 2048 everywhere 61 us, 1024 everywhere 68 us, mixed 59 us.
         const int kt = batch <= 4 ? ((p.K <= 1024 || p.K % 2048 != 0) ? 1024 : 2048) : 512;
         const int n_ks = ceil_div(p.K, kt);
-        const int groups = p.stage == kStageTower ? 3 : 1;
+        const int groups = p.stage == kStageTower ? n_towers : 1;
         const int group_rbs = p.stage == kStageTower ? ceil_div(T, kFRows) : p.row_blocks;
         // about one CTA per SM in total for small batches and two for large ones (narrow tiles, two
         // CTAs fit an SM), each staging its x tile once and walking several row blocks
+        // (half as many CTAs, so that the next stage's CTAs could sit beside them and have their first
+        // weights in flight when this stage ends, was measured: 58 -> 96 us per call at batch 1)
         int gx = (kt >= 2048 ? sms : 2 * sms) / (n_ks * groups);
         gx = std::max(1, std::min(gx, group_rbs));
         const dim3 grid(gx, n_ks, groups);
@@ -398,27 +434,34 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
     };
     const long long tower_stride = (long long)d_model + (long long)T * d_model + T;
     const float* cur = params;
-    // towers (one launch for the three)
-    p.stage = kStageTower; p.K = d_model; p.row_blocks = ceil_div(3ll * T, kFRows);
+    float* fpre = reinterpret_cast<float*>(sc + L.fpre);
+    // towers (one launch for those of this phase)
+    n_towers = phase == 0 ? 3 : (phase == 1 ? 2 : 1);
+    p.stage = kStageTower; p.K = d_model; p.w_stride = d_model; p.row_blocks = ceil_div(3ll * T, kFRows);
+    p.tower_base = phase == 2 ? 2 : 0;
     p.gain = cur; p.W = cur + d_model; p.bias = cur + d_model + (long long)T * d_model; p.tower_stride = tower_stride;
     p.in0 = h_prev; p.in1 = emb; p.in2 = h_local; p.out = abc;
-    if ((e = launch(false)) != cudaSuccess) return e;  // follows a memset: ordinary launch
+    if ((e = launch(false)) != cudaSuccess) return e;  // follows a memset (phases 0, 1) or a join of two streams (phase 2): ordinary launch
     cur += 3 * tower_stride;
     // fusion
-    p.stage = kStageFusion; p.K = 9 * T; p.row_blocks = ceil_div(T, kFRows);
-    p.gain = nullptr; p.W = cur; p.bias = cur + (long long)T * 9 * T; p.in0 = abc; p.in1 = p.in2 = nullptr; p.out = z;
+    p.stage = kStageFusion; p.K = (phase == 0 ? 9 : (phase == 1 ? 4 : 5)) * T; p.w_stride = 9 * T; p.row_blocks = ceil_div(T, kFRows);
+    p.fus_part = phase; p.fpre = fpre;
+    p.gain = nullptr; p.W = cur; p.bias = cur + (long long)T * 9 * T; p.in0 = abc; p.in1 = p.in2 = nullptr;
+    p.out = phase == 1 ? fpre : z;
     if ((e = launch(pdl)) != cudaSuccess) return e;
+    if (phase == 1) return cudaSuccess;
+    p.fus_part = 0;
     cur += (long long)T * 9 * T + T;
     for (int k = 0; k < n_blocks; ++k) {
-        p.stage = kStageGateUp; p.K = T; p.row_blocks = ceil_div(F, kFRows / 2);
+        p.stage = kStageGateUp; p.K = T; p.w_stride = T; p.row_blocks = ceil_div(F, kFRows / 2);
         p.gain = cur; p.W = cur + T; p.bias = nullptr; p.in0 = z; p.out = h;
         if ((e = launch(pdl)) != cudaSuccess) return e;
-        p.stage = kStageDown; p.K = F; p.row_blocks = ceil_div(T, kFRows);
+        p.stage = kStageDown; p.K = F; p.w_stride = F; p.row_blocks = ceil_div(T, kFRows);
         p.gain = nullptr; p.W = cur + T + 2ll * F * T; p.in0 = h; p.out = z;
         if ((e = launch(pdl)) != cudaSuccess) return e;
         cur += (long long)T + 3ll * F * T;
     }
-    p.stage = kStageOut; p.K = T; p.row_blocks = 1;
+    p.stage = kStageOut; p.K = T; p.w_stride = T; p.row_blocks = 1;
     p.gain = cur; p.W = cur + T; p.bias = cur + 2 * T; p.in0 = z; p.out = nullptr;
     p.threshold = threshold; p.override_flags = override_flags; p.scores = scores; p.logits = logits;
     p.flags = flags; p.counters = counters;

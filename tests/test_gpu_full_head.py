@@ -88,6 +88,44 @@ def test_full_head_parity(dm, T, F, nb, B, variant):
     np.testing.assert_allclose(scores.cpu().numpy(), s, rtol=0, atol=2e-5)
 
 
+@pytest.mark.parametrize("dm,T,F,nb,B", [(64, 32, 40, 2, 5), (128, 64, 96, 1, 20), (2048, 1024, 2048, 2, 1),
+                                          (2048, 1024, 2048, 2, 4), (4104, 24, 2052, 1, 2)])
+def test_full_head_in_two_parts(dm, T, F, nb, B):
+    """The part that needs only h_prev and emb first (its own call), then the rest on the same scratch:
+    same scores as the oracle, flags exact outside the band, and the same bits on a second round."""
+    ctx = _ctx()
+    params = _params(3, dm, T, F, nb)
+    x = [synth.gauss_f32_tensor(4, i, (B, dm)) for i in range(3)]
+    q, s = orc.full_head(params, *x, d_tower=T, d_ff=F, n_blocks=nb)
+    srt = np.sort(s)
+    tau = float(0.5 * (srt[B // 2 - 1] + srt[B // 2])) if B > 1 else 0.5
+    scores = torch.zeros(B, device="cuda")
+    logits = torch.zeros(B, device="cuda")
+    flags = torch.zeros(B, dtype=torch.uint8, device="cuda")
+    pd = torch.from_numpy(params).cuda()
+    xd = [torch.from_numpy(v).cuda() for v in x]
+    scratch = ctx.full_head_scratch(B, dm, T, F, nb)
+    scratch.fill_(0xFF)     # NaN patterns: nothing may be read before it is written
+    # the Local hidden state does not exist yet when the first part runs: hand the second part a buffer
+    # that is only filled in between
+    h_local = torch.full_like(xd[2], float("nan"))
+    rounds = []
+    for _ in range(2):
+        h_local.fill_(float("nan"))
+        ctx.recall_score_full_pre(B, pd, T, F, nb, xd[0], xd[1], scratch)
+        h_local.copy_(xd[2])
+        ctx.recall_score_full(B, pd, T, F, nb, xd[0], xd[1], h_local, tau, None, scores, logits, flags,
+                              scratch=scratch, variant=3)
+        torch.cuda.synchronize()
+        rounds.append(logits.clone())
+    assert torch.equal(rounds[0], rounds[1])
+    np.testing.assert_allclose(logits.cpu().numpy(), q, rtol=0, atol=1e-4)
+    np.testing.assert_allclose(scores.cpu().numpy(), s, rtol=0, atol=2e-5)
+    decided = np.abs(s - tau) >= gh.FLAG_BAND
+    np.testing.assert_array_equal(flags.cpu().numpy()[decided], orc.flags(q, s, tau)[decided])
+    assert ctx.read_device_status() == 0
+
+
 def test_full_head_nonfinite_input_selects_full_and_bad_dims_are_refused():
     ctx = _ctx()
     dm, T, F, nb, B = 64, 32, 40, 1, 3
