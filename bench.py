@@ -707,6 +707,63 @@ def paper_head_section(torch, args, flush, side):
     return res
 
 
+def ring_section(torch, args, flush, side):
+    """The Local workspace variant of the paper's runtime (a second view per request holding the sink
+    positions and a ring of recent positions, written by every step's commit) against reading the
+    window in place from the paged history: the Local launch over each view, and the per-step write of
+    the current position into each view, at the configuration's window and at the paper's 2048."""
+    from paper_2609_20734_b200 import binding, ring_view, workloads
+
+    rows = []
+    base = workloads.make(args.config)
+    for w in sorted({max(base.windows), 2048}):
+        wl = replace(base, windows=[w if g else x for g, x in zip(base.gated, base.windows)], steps=8)
+        st = workloads.materialize(wl)
+        B, L = wl.B, wl.L
+        ctx = binding.OdaContext(workloads.oda_config(wl, st.num_blocks, variant=args.variant))
+        geo = ring_view.geometry(B, wl.windows, wl.sinks)
+        n_ring = wl.phys_layers * geo.num_blocks * wl.Hkv * 16 * wl.D
+        ring_k = torch.zeros(n_ring, dtype=torch.bfloat16, device="cuda")
+        ring_v = torch.zeros(n_ring, dtype=torch.bfloat16, device="cuda")
+        ring_tab = torch.from_numpy(ring_view.table(geo, B, wl.max_blocks_per_seq)).cuda()
+        ring_view.fill_from_paged(geo, ring_k, ring_v, st.k_cache, st.v_cache, st.table_host, wl.seq_lens0, wl.windows,
+                                  wl.sinks, phys_layers=wl.phys_layers, paged_blocks=st.num_blocks, kv_heads=wl.Hkv,
+                                  head_dim=wl.D)
+        rcfg = workloads.oda_config(wl, st.num_blocks, variant=args.variant)
+        rcfg.kv_layer_stride = geo.num_blocks * wl.Hkv * 16 * wl.D
+        rctx = binding.OdaContext(rcfg)
+        q = workloads.q_device(wl, 0)
+        out = torch.zeros((L, B, wl.Hq, wl.D), device="cuda")
+        out_r = torch.zeros_like(out)
+        kc = torch.zeros((L, B, wl.Hkv, wl.D), dtype=torch.bfloat16, device="cuda")
+        graphs = {
+            "local_paged": capture(torch, side, lambda s_: ctx.local_decode(
+                0, L, B, q, st.k_cache, st.v_cache, st.block_table, st.seq_lens, out, None, stream=s_)),
+            "local_ring": capture(torch, side, lambda s_: rctx.local_decode(
+                0, L, B, q, ring_k, ring_v, ring_tab, st.seq_lens, out_r, None, stream=s_)),
+            "commit_paged": capture(torch, side, lambda s_: ctx.write_current_kv(
+                B, kc, kc, None, st.k_cache, st.v_cache, st.block_table, st.seq_lens, stream=s_)),
+            "commit_ring": capture(torch, side, lambda s_: rctx.write_current_kv(
+                B, kc, kc, None, ring_k, ring_v, ring_tab, st.seq_lens, stream=s_)),
+        }
+        torch.cuda.synchronize()
+        t = {n: [] for n in graphs}
+        for r in range(args.kernel_reps + 2):
+            for n, g in graphs.items():
+                ms = timed_replay(torch, g, flush, r)
+                if r >= 2:
+                    t[n].append(ms)
+        same = bool(torch.equal(out, out_r))
+        rows.append(dict({n + "_us": float(np.mean(v)) * 1e3 for n, v in t.items()}, window=w,
+                         ring_view_bytes=int(2 * n_ring * 2), same_bits_as_paged=same))
+        del st, ctx, rctx, graphs, ring_k, ring_v
+        torch.cuda.empty_cache()
+    return {"rows": rows,
+            "note": "ring view = sink pages + (window/16 + 1) ring pages per request and layer, a second paged cache "
+                    "with a periodic block table read by the same Local kernel; the variant pays commit_ring_us on "
+                    "top of commit_paged_us every step (both views advance) and buys local_paged_us - local_ring_us"}
+
+
 def main():
     args = parse()
     from paper_2609_20734_b200 import workloads
@@ -968,6 +1025,8 @@ def main():
                 torch.cuda.empty_cache()
         if world == 1 and not args.no_paper_head and wl.B <= 4:
             line["paper_head"] = paper_head_section(torch, args, flush, side)
+        if world == 1 and not args.no_configs and wl.kv_index is None:
+            line["ring_workspace"] = ring_section(torch, args, flush, side)
         line["clocks"] = sampler.stop()
 
         # ---- the oracle on the host cores, bounded sample ----
