@@ -377,9 +377,6 @@ oda_status_t oda_create(const oda_config_t* cfg, oda_ctx_t** out_ctx)
         c->num_sms = 148;  // no device visible: sizes follow a B200 so that host-only checks still work
         c->grid = 148 * 2;
     }
-#ifdef ODA_TIMELINE
-    if (const char* e = std::getenv("ODA_SNAP")) c->snap_span_pages = std::atoi(e);
-#endif
     c->max_items = c->grid + cfg->num_layers * cfg->max_batch * cfg->num_kv_heads;
     c->head_grid = cfg->head_d_hidden > 0 ? recall_head_grid(cfg->head_d_hidden) : 1;
     compute_layout(c);

@@ -60,20 +60,8 @@ struct FusedHeadParams {
     int32_t* counters;
 };
 
-#ifdef ODA_TIMELINE
-__device__ unsigned long long g_fu_timeline[160 * 32];
-#define FU_TL(slot) do { if (threadIdx.x == 0 && (slot) < 32) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_fu_timeline[blockIdx.x * 32 + (slot)] = t_; } } while (0)
-extern "C" int oda_debug_fused_timeline(unsigned long long* host, int n) { return (int)cudaMemcpyFromSymbol(host, g_fu_timeline, sizeof(unsigned long long) * n); }
-#else
-#define FU_TL(slot) do { } while (0)
-#endif
-#ifdef ODA_TIMELINE
-#define FU_CLK(v) const long long v = clock64()
-#define FU_ACC(var, dt) var += (dt)
-#else
 #define FU_CLK(v) do { } while (0)
 #define FU_ACC(slot, dt) do { } while (0)
-#endif
 
 enum { kFuTower = 0, kFuFusion = 1, kFuGateUp = 2, kFuDown = 3 };
 
@@ -415,10 +403,6 @@ __global__ void __launch_bounds__(kFuThreads, 1) full_head_fused_kernel(const __
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    FU_TL(0);
-#ifdef ODA_TIMELINE
-    const long long tl_c0 = clock64();
-#endif
     volatile int* abort_flag = &ctl->abort;
     int* wait_status = p.status ? p.status : p.sync + 1;
     const int n_stages = 4 + 2 * p.n_blocks;
@@ -471,7 +455,6 @@ __global__ void __launch_bounds__(kFuThreads, 1) full_head_fused_kernel(const __
     for (int s = 0; s < n_stages; ++s) {
         const FuStage d = fu_stage(p, s);
         const FuShare sh = fu_share(d, c, G);
-        FU_TL(1 + 3 * s);
         // ---- the stage's whole input -> shared memory, as [B][K] (gain applied where the stage
         //      input is RMS-normalised); gains ride behind the inputs so that every load of the
         //      staging is in flight together
@@ -515,7 +498,6 @@ __global__ void __launch_bounds__(kFuThreads, 1) full_head_fused_kernel(const __
             x = xs + (size_t)s * B * p.d_model;   // staged with tower 0's
         } else {
             aborted |= !fu_grid_barrier(p, ctl, barrier_index++, tid);  // reads what the previous stage wrote
-            FU_TL(2 + 3 * s);
             if (d.type == kFuFusion) {
                 // u = [a; b; c; a.b; |a-b|; a.c; |a-c|; b.c; |b-c|] per request: the towers' outputs go
                 // straight to the first three segments, the other six are formed from them
@@ -554,7 +536,6 @@ __global__ void __launch_bounds__(kFuThreads, 1) full_head_fused_kernel(const __
                 fu_consumer_sync();
             }
         }
-        FU_TL(3 + 3 * s);
         for (int rd = 0; rd < sh.rounds; ++rd) {
             switch (B) {
             case 1: fu_round<1>(p, d, sh, rd, ring, x, ctl, full0, empty0, abort_flag, wait_status, base, aborted, warp, lane); break;
@@ -564,10 +545,6 @@ __global__ void __launch_bounds__(kFuThreads, 1) full_head_fused_kernel(const __
             }
         }
     }
-    FU_TL(1 + 3 * n_stages);
-#ifdef ODA_TIMELINE
-    if (tid == 0) g_fu_timeline[blockIdx.x * 32 + 30] = (unsigned long long)(clock64() - tl_c0);
-#endif
     // ---- final barrier is a ticket: the CTA that arrives last computes q = w . RMSNorm(z) + bias
     fu_consumer_sync();
     if (tid == 0) {

@@ -23,17 +23,6 @@
 namespace oda {
 
 
-#ifdef ODA_TIMELINE
-__device__ unsigned long long g_timeline[1024 * 8];
-#define ODA_TL(slot) do { if ((threadIdx.x & 31) == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); g_timeline[blockIdx.x * 8 + (slot)] = t_; } } while (0)
-extern "C" int oda_debug_timeline(unsigned long long* host, int n) { return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n); }
-__device__ long long g_tl_acc[1024 * 8];
-extern "C" int oda_debug_acc(long long* host, int n) { return (int)cudaMemcpyFromSymbol(host, g_tl_acc, sizeof(long long) * n); }
-#define ODA_CLK(v) const long long v = clock64()
-#else
-#define ODA_CLK(v) do { } while (0)
-#define ODA_TL(slot) do { } while (0)
-#endif
 
 constexpr int kMaxStages = 6;
 // a partial of the TMA variant: the epilogue warp's fragment, 9 rows of one float4 per lane
@@ -177,10 +166,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     const uint32_t efull = smem_u32(&ctl.efull), efree = smem_u32(&ctl.efree);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) ODA_TL(0);
-#ifdef ODA_TIMELINE
-    if (tid == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); g_timeline[blockIdx.x * 8 + 7] = sm_; }
-#endif
     // Batch-1 Local launch that may give every CTA one whole unit: the one length and this CTA's layer
     // entry are requested first thing (after the dependency wait, which such a launch takes at once:
     // it is the first kernel of a step), so that their latency runs while the barriers are set up.
@@ -209,7 +194,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     prefetch_block_table(p);
     __syncthreads();      // the barriers are initialised for every warp
     if (!direct_try) griddep_wait();  // everything above is independent of the previous kernel in the stream
-    if (tid == 0) ODA_TL(1);
     if (direct_try) dp.ok = direct_rule(p, dp.t);  // same registers in every thread: no barrier, no shared plan
     int span;             // the one span this CTA streams
     if (dp.ok) {
@@ -223,7 +207,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         span = plan.my_span;
     }
     griddep_launch_dependents();
-    if (tid == 0) ODA_TL(2);
     volatile int* abort_flag = &ctl.abort;
     constexpr uint32_t kQBytes = G * D * 2;
     if (span < 0) return;
@@ -280,7 +263,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag, p.status)) { dead = true; break; }
                 const bool with_q = cur.first && t0 == 0;
-                if (cnt == 0) ODA_TL(3);
                 if (lane == 0) {
                     if (with_q) {  // visible to the consumers once the stage's barrier completes
                         ctl.items[s] = cur.item;
@@ -490,7 +472,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                     store_final(it, ro, rml);
                 }
             }
-            ODA_TL(6);
         }
         return;
     }
@@ -520,13 +501,8 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         int x = 0, x_end = 1;
         if (!dp.ok) span_range(plan, span, x, x_end);
         span_pages = x_end - x;
-#ifdef ODA_TIMELINE
-        long long a_dec = 0, a_first = 0, a_tiles = 0, a_wait = 0, a_merge = 0, a_items = 0;
-#endif
         while (x < x_end && !aborted) {
             Item it;
-            ODA_CLK(c0);
-            ODA_CLK(c1);
             // the item's descriptor and its Q^T fragments come with the item's first tile; heads >= G stay zero
             uint32_t qa[D / 16][2];
             {
@@ -534,10 +510,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
                 it = ctl.items[s];
                 x += ctl.item_take[s];
-                if (cnt == 0 && warp == 0) ODA_TL(4);
-#ifdef ODA_TIMELINE
-                { const long long c2 = clock64(); a_dec += c1 - c0; a_first += c2 - c1; a_items += 1; }
-#endif
                 if (cnt == 0 && p.sm_stats) t_first = globaltimer_ns();
                 const uint32_t* qs = reinterpret_cast<const uint32_t*>(qring + s * C::kQSlotBytes) + (hrow * D + qc) / 2;
 #pragma unroll
@@ -553,15 +525,10 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
 
             TileWalk tw;
             uint32_t s_last = 0;  // the stage of the item's last tile: kept until the fold below is done with it
-            ODA_CLK(c3);
             for (tw.start(it); !tw.done();) {
                 const uint32_t s = cnt % C::kStages, ph = (cnt / C::kStages) & 1;
                 ++cnt;
-                ODA_CLK(c4);
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status)) { aborted = true; break; }
-#ifdef ODA_TIMELINE
-                a_wait += clock64() - c4;
-#endif
                 if (warp < tw.npages) {
                     const bool sink = tw.v + warp < it.sink_pg1;
                     const int pos0 = item_logical_page(it, tw.v + warp) * kPage;
@@ -649,11 +616,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                     mbar_arrive(empty0 + 8 * s);
             }
             if (aborted || *abort_flag) { aborted = true; break; }
-            if (warp == 0) ODA_TL(5);
-            ODA_CLK(c5);
-#ifdef ODA_TIMELINE
-            a_tiles += c5 - c3;
-#endif
 
             // ---- fold the four warps' states and leave the item to the epilogue warp.  Every warp
             //      parks its fragment in its own page slot of the item's last stage (that data is
@@ -737,16 +699,7 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 if (warp == 0) mbar_arrive(efull);
             }
             ++ecnt;
-#ifdef ODA_TIMELINE
-            a_merge += clock64() - c5;
-#endif
         }
-#ifdef ODA_TIMELINE
-        if (tid == 0) {
-            long long* a = g_tl_acc + blockIdx.x * 8;
-            a[0] = a_dec; a[1] = a_first; a[2] = a_tiles; a[3] = a_wait; a[4] = a_merge; a[5] = a_items;
-        }
-#endif
     }
     // calibration run: how long this SM took to stream how many pages
     if (p.sm_stats && tid == 0 && !aborted && pages_half > 0 && plan.nseg == (int)gridDim.x) {
