@@ -920,6 +920,29 @@ def main():
         t_layers = [timed_replay(torch, g_layers, flush, r) for r in range(reps + 2)][2:]
         lb, fb = wl.algorithmic_bytes(np.asarray(wl.seq_lens0), np.ones(B))
         floor_us = kt["floor"]["us"]
+        # The Local launch without the two events' own cost: one graph of n Local launches, each at a
+        # different length, so that every launch reads a window the others do not touch (n x the window
+        # bytes: far more than L2, no flush needed), one pair of events around all of them.
+        n_win = min(32, int(np.min(wl.seq_lens0)) // (max(wl.windows) + max(wl.sinks))) - 1
+        local_b2b = None
+        if n_win >= 8 and len(set(wl.windows)) == 1:
+            lens = [torch.from_numpy(np.asarray(wl.seq_lens0, np.int32) - i * max(wl.windows)).cuda() for i in range(n_win)]
+            g_b2b = capture(torch, side, lambda s_: [ctx.local_decode(
+                0, L, B, run.qs[0], st.k_cache, st.v_cache, st.block_table, ln, run.out, run.lse, stream=s_) for ln in lens])
+            torch.cuda.synchronize()
+            t_b2b = [timed_replay(torch, g_b2b) for _ in range(reps + 2)][2:]
+            b2b_bytes = float(np.mean([wl.algorithmic_bytes(np.asarray(wl.seq_lens0) - i * max(wl.windows), np.zeros(B))[0]
+                                       for i in range(n_win)]))
+            us_b2b = float(np.mean(t_b2b)) * 1e3 / n_win
+            local_b2b = {"us_per_launch": us_b2b, "launches": n_win, "achieved": b2b_bytes / (us_b2b * 1e-6) / 1e9,
+                         "frac": b2b_bytes / (us_b2b * 1e-6) / 1e9 / peak,
+                         "frac_of_8000_nominal": b2b_bytes / (us_b2b * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+                         "what": f"{n_win} Local launches in one graph between one pair of events, each at a length "
+                                 f"{max(wl.windows)} positions below the last: disjoint windows, {n_win * b2b_bytes / 1e9:.1f} GB "
+                                 "per replay (inputs larger than L2 instead of a flush); the small arrays and the code "
+                                 "stay warm, as in a decode loop; the launches overlap their set-up with the previous "
+                                 "one's tail by programmatic dependent launch"}
+            del g_b2b
         kernels = {}
         for name, nbytes in (("local", lb), ("full", fb)):
             kernels[name] = roofline_entry(nbytes, kt[name]["us"], peak, {
@@ -929,6 +952,8 @@ def main():
         other = "local" if dominant == "full" else "full"
         line["roofline"] = dict(kernels[dominant], kernel=f"splitkv ({dominant} pass)", peak_source=peak_src)
         line["roofline_other"] = dict(kernels[other], kernel=f"splitkv ({other} pass)")
+        if local_b2b:
+            (line["roofline"] if dominant == "local" else line["roofline_other"])["back_to_back_distinct_windows"] = local_b2b
         line["timing_floor"] = {"us": floor_us, "us_l2_warm": kt["floor"]["us_l2_warm"],
                                 "what": "the library's smallest launch (one CTA copying one 16-byte row) timed exactly like "
                                         "the two passes: a one-kernel graph between two events after the same flush; "
