@@ -47,3 +47,19 @@ def test_bench_prints_one_contract_line():
     (tiny,) = d["configs"]
     assert tiny["name"] == "tiny" and tiny["recall_rate_realised"] == 0.25 and tiny["tokens_per_s"] > 0
     assert tiny["head"]["us"] > 0 and tiny["local"]["us"] > 0 and tiny["full"]["us"] > 0
+
+
+@pytest.mark.parametrize("shard", ["heads", "sequence"])
+def test_bench_shard_modes_run_at_world_size_one(shard):
+    """The GPU half of `bench.py --shard ...` with one rank: the library's kernels on either side of an
+    NCCL collective (which a one-rank group performs on itself), one contract line."""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "1", "--shard", shard, "--steps", "4",
+                        "--warmup", "3"], capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["shard"] == shard and d["scaling"] == "strong" and d["n_gpus"] == 1 and d["steps"] == 4
+    assert d["value"] > 0 and abs(d["value"] - 1e3 / d["ms_per_step"]) < 1e-6 * d["value"]
+    assert d["passes"]["measured"] == 3 and d["gpu_launches"] == (4 if shard == "heads" else 2) * 4
+    assert d["config"]["parallelism"].startswith("tp1" if shard == "heads" else "sp1")
