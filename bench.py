@@ -1039,19 +1039,24 @@ def main():
         run.close()
         del run, ctx, st
 
-        # ---- the other benchmark configurations and the recall heads inside a step (one GPU) ----
-        if world == 1 and not args.no_configs:
-            line["configs"] = []
-            for name in [n for n in args.configs.split(",") if n and n != args.config]:
-                try:
-                    line["configs"].append(extra_config(torch, args, name, EXTRA_CONFIGS.get(name, 16), flush, side, peak))
-                except torch.OutOfMemoryError as e:  # a smaller GPU: say so, keep the line
-                    line["configs"].append({"name": name, "skipped": f"out of device memory: {str(e)[:80]}"})
+        # ---- the other benchmark configurations and the recall heads inside a step (one GPU).  Context
+        #      for the headline: a failure in one of them is recorded in its place and the line still goes out ----
+        def guarded(what, fn):
+            try:
+                return fn()
+            except Exception as e:  # noqa: BLE001
                 torch.cuda.empty_cache()
+                return {"name": what, "skipped": f"{type(e).__name__}: {str(e)[:160]}"}
+
+        if world == 1 and not args.no_configs:
+            line["configs"] = [guarded(name, lambda name=name: extra_config(torch, args, name, EXTRA_CONFIGS.get(name, 16),
+                                                                            flush, side, peak))
+                               for name in args.configs.split(",") if name and name != args.config]
+            torch.cuda.empty_cache()
         if world == 1 and not args.no_paper_head and wl.B <= 4:
-            line["paper_head"] = paper_head_section(torch, args, flush, side)
+            line["paper_head"] = guarded("paper_head", lambda: paper_head_section(torch, args, flush, side))
         if world == 1 and not args.no_configs and wl.kv_index is None:
-            line["ring_workspace"] = ring_section(torch, args, flush, side)
+            line["ring_workspace"] = guarded("ring_workspace", lambda: ring_section(torch, args, flush, side))
         line["clocks"] = sampler.stop()
 
         # ---- the oracle on the host cores, bounded sample ----
