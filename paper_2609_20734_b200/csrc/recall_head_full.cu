@@ -422,7 +422,9 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
         // about one CTA per SM in total for small batches and two for large ones (narrow tiles, two
         // CTAs fit an SM), each staging its x tile once and walking several row blocks
         // (half as many CTAs, so that the next stage's CTAs could sit beside them and have their first
-        // weights in flight when this stage ends, was measured: 58 -> 96 us per call at batch 1)
+        // weights in flight when this stage ends, was measured twice -- 1024-wide tiles everywhere, and the
+        // tiles below compiled for two CTAs per SM: 58 -> 96 and 58 -> 92 us per call at batch 1.  A stage is
+        // bound by how many loads an SM has in flight, and half the CTAs are half the loads.)
         int gx = (kt >= 2048 ? sms : 2 * sms) / (n_ks * groups);
         gx = std::max(1, std::min(gx, group_rbs));
         const dim3 grid(gx, n_ks, groups);

@@ -18,7 +18,6 @@ from __future__ import annotations
 
 import json
 import os
-import time
 from dataclasses import replace
 
 import numpy as np
