@@ -355,6 +355,10 @@ oda_status_t oda_full_decode_gated(oda_ctx_t* ctx, int32_t layer_begin, int32_t 
 oda_status_t oda_write_current_kv(oda_ctx_t* ctx, int32_t batch, const void* k_cur, const void* v_cur,
                                   const uint8_t* mask, void* k_cache, void* v_cache,
                                   const int32_t* block_table, const int32_t* seq_lens, void* stream);
+/* Position advance on the device (the appendix on the runtime protocol: a replay updates the
+ * device-side effective length): seq_lens[b] += 1 for b < batch.  oda_step does this by itself
+ * (advance_seq_lens); this call is for steps composed from the separate calls.  One small launch. */
+oda_status_t oda_advance_seq_lens(oda_ctx_t* ctx, int32_t batch, int32_t* seq_lens, void* stream);
 /* Selected-state rule for per-request rows (h_t = h_t^{b_t}): out[b] = flags[b] ? full[b] : local[b];
  * rows of row_bytes bytes (a multiple of 16), 16-byte aligned device pointers. */
 oda_status_t oda_select_rows(oda_ctx_t* ctx, int32_t batch, const void* local, const void* full,

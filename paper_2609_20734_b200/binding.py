@@ -25,7 +25,7 @@ EXPORTS = [
     "oda_status_string", "oda_last_error", "oda_version", "oda_local_decode_static",
     "oda_local_decode_static_status",
     "oda_calibration_begin", "oda_calibration_end", "oda_calibration_spread",
-    "oda_write_current_kv", "oda_select_rows", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
+    "oda_write_current_kv", "oda_select_rows", "oda_advance_seq_lens", "oda_full_head_param_count", "oda_full_head_scratch_bytes",
     "oda_recall_score_full", "oda_recall_score_full_pre", "oda_recall_preact", "oda_recall_finalize", "oda_merge_partials",
     "oda_recall_finalize_exchange", "oda_merge_partials_exchange", "oda_set_cache_resident_bytes",
 ]
@@ -133,6 +133,7 @@ def load_library():
         lib.oda_local_decode_static_status.argtypes = [vp, ctypes.POINTER(i32)]
         lib.oda_write_current_kv.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.oda_select_rows.argtypes = [vp, i32, vp, vp, vp, vp, ctypes.c_int64, vp]
+        lib.oda_advance_seq_lens.argtypes = [vp, i32, vp, vp]
         lib.oda_full_head_param_count.argtypes = [i32, i32, i32, i32]
         lib.oda_full_head_param_count.restype = ctypes.c_int64
         lib.oda_full_head_scratch_bytes.argtypes = [ctypes.POINTER(_FullHead), i32]
@@ -382,6 +383,11 @@ class OdaContext:
         self._check(self.lib.oda_write_current_kv(
             self._h, batch, _ptr(k_cur), _ptr(v_cur), _ptr(mask), _ptr(k_cache), _ptr(v_cache),
             _ptr(block_table), _ptr(seq_lens), _stream() if stream is None else stream), "oda_write_current_kv")
+
+    def advance_seq_lens(self, batch, seq_lens, stream=None):
+        """seq_lens[b] += 1 on the device (steps composed from the separate calls)."""
+        self._check(self.lib.oda_advance_seq_lens(self._h, batch, _ptr(seq_lens),
+                                                  _stream() if stream is None else stream), "oda_advance_seq_lens")
 
     def select_rows(self, batch, local, full, flags, out, stream=None):
         self._check(self.lib.oda_select_rows(

@@ -749,6 +749,18 @@ oda_status_t oda_merge_partials(oda_ctx_t* c, int32_t n_parts, int32_t lb, int32
     return ODA_OK;
 }
 
+oda_status_t oda_advance_seq_lens(oda_ctx_t* c, int32_t batch, int32_t* seq_lens, void* stream)
+{
+    if (!c) return ODA_ERR_INVALID_ARG;
+    if (batch < 0 || batch > c->cfg.max_batch) return fail(c, ODA_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    if (batch == 0) return ODA_OK;
+    if (!seq_lens) return fail(c, ODA_ERR_INVALID_ARG, "seq_lens is null");
+    cudaError_t e = launch_advance_seq_lens(seq_lens, batch, static_cast<cudaStream_t>(stream), c->use_pdl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "seq_lens advance launch");
+    c->launches += 1;
+    return ODA_OK;
+}
+
 oda_status_t oda_select_rows(oda_ctx_t* c, int32_t batch, const void* local, const void* full,
                              const uint8_t* flags, void* out, int64_t row_bytes, void* stream)
 {

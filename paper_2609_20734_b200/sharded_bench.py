@@ -121,7 +121,7 @@ def run(args, wl, bench):
             tp.tp_step(ctx, hs, B, qs[s], st.k_cache, st.v_cache, st.block_table, st.seq_lens, out,
                        W1=head["W1"], b1=head["b1"], w2=head["w2"], b2=head["b2"], threshold=wl.threshold,
                        pre=pre, scores=scores, flags=flags, override_flags=ovs[s])
-            st.seq_lens.add_(1)
+            ctx.advance_seq_lens(B, st.seq_lens)
 
         seq_steps = [np.asarray(wl.seq_lens0) + s for s in range(args.warmup, nsteps)]
         step_bytes = float(np.mean([sum(wl.algorithmic_bytes(sl, f)) for sl, f in zip(seq_steps, flags_h[args.warmup:])]))

@@ -61,5 +61,5 @@ def test_bench_shard_modes_run_at_world_size_one(shard):
     d = json.loads(lines[0])
     assert d["shard"] == shard and d["scaling"] == "strong" and d["n_gpus"] == 1 and d["steps"] == 4
     assert d["value"] > 0 and abs(d["value"] - 1e3 / d["ms_per_step"]) < 1e-6 * d["value"]
-    assert d["passes"]["measured"] == 3 and d["gpu_launches"] == (4 if shard == "heads" else 2) * 4
+    assert d["passes"]["measured"] == 3 and d["gpu_launches"] == (5 if shard == "heads" else 2) * 4
     assert d["config"]["parallelism"].startswith("tp1" if shard == "heads" else "sp1")

@@ -89,3 +89,16 @@ def test_step_with_commit_matches_oracle():
     np.testing.assert_array_equal(synth.torch_to_bf16_bits(dev["v"]), prob["v"])
     np.testing.assert_array_equal(seq_dev.cpu().numpy(), np.asarray(seq) + 1)
     assert ctx.read_device_status() == 0
+
+
+def test_advance_seq_lens_moves_only_the_requests_of_the_call():
+    prob = make_problem(4, 1, 5, 4, 2, 64, [3, 40, 7, 16, 2053])
+    ctx = gh.make_ctx(prob, [16], [0], [1])
+    seq = torch.from_numpy(prob["seq_lens"]).cuda()
+    ctx.advance_seq_lens(3, seq)
+    ctx.advance_seq_lens(5, seq)
+    ctx.advance_seq_lens(0, seq)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(seq.cpu().numpy(), np.array([5, 42, 9, 17, 2054], np.int32))
+    with pytest.raises(binding.OdaError):
+        ctx.advance_seq_lens(6, seq)
