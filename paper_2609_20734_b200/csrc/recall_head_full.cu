@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
     __shared__ __align__(16) float s_x[kFBT][kFKT];   // x * gain
     __shared__ float s_acc[kFRows][kFBT];
     __shared__ float s_ss[kFRows][kFBT];
-    __shared__ int s_last;
+    __shared__ unsigned char s_lastv[kFThreads];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ks = blockIdx.y, n_ks = gridDim.y;
@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                     }
                 }
             }
-            __syncthreads();  // s_acc and s_last are reused by the next row block
+            __syncthreads();  // s_acc is reused by the next row block
 #pragma unroll
             for (int c = 0; c < kWC; ++c) w_cur[c] = w_nxt[c];
         }
@@ -285,16 +285,26 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
             //      row block it worked on; the CTA that completes a row block adds the slices in order
             __threadfence();
             __syncthreads();
-            for (int rb2 = blockIdx.x; rb2 < group_rbs; rb2 += gridDim.x) {
-                const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb2;
-                if (tid == 0) {
+            // the tickets of all the row blocks this CTA worked on are taken at once (one thread each: one
+            // round trip, not one per block), then the blocks it completed are finished one after another
+            const int n_mine = (int)blockIdx.x < group_rbs ? (group_rbs - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+            for (int i0 = 0; i0 < n_mine; i0 += kFThreads) {
+                const int i = i0 + tid;
+                unsigned char last = 0;
+                if (i < n_mine) {
+                    const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + (int)blockIdx.x + i * (int)gridDim.x;
                     const int old = atomicAdd(p.rb_tickets + grb, 1);
-                    s_last = (old == n_ks - 1);
-                    if (s_last) p.rb_tickets[grb] = 0;
+                    last = (old == n_ks - 1);
+                    if (last) p.rb_tickets[grb] = 0;
                 }
+                s_lastv[tid] = last;
+                __threadfence();
                 __syncthreads();
-                if (s_last) {
-                    __threadfence();
+                const int n_here = min(kFThreads, n_mine - i0);
+                for (int j = 0; j < n_here; ++j) {
+                    if (!s_lastv[j]) continue;
+                    const int rb2 = (int)blockIdx.x + (i0 + j) * (int)gridDim.x;
+                    const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb2;
                     for (int e = tid; e < out_rows * p.batch; e += kFThreads) {
                         const int r = e / p.batch, b = e - r * p.batch;
                         float ss = 0.f;
@@ -314,7 +324,7 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                         }
                     }
                 }
-                __syncthreads();
+                __syncthreads();  // s_lastv is reused by the next batch of tickets
             }
         }
     }
