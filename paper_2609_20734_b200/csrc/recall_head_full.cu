@@ -90,27 +90,57 @@ __device__ __forceinline__ float4 stage_x4(const FullStageParams& p, int tower, 
     return *reinterpret_cast<const float4*>(p.in0 + (size_t)b * p.K + k);  // z [B][T] or h [B][F]
 }
 
+// What the epilogue of output element (row r of the stage, request b) reads besides the sums: loaded
+// apart from stage_finish so that a caller can have these loads in flight together with the sums'.
+struct StageEpi {
+    float v[5];
+};
+__device__ __forceinline__ StageEpi stage_epilogue_operands(const FullStageParams& p, int r, int b)
+{
+    StageEpi e;
+    e.v[0] = e.v[1] = e.v[2] = e.v[3] = e.v[4] = 0.f;
+    if (p.stage == kStageTower) {
+        const int i = r / p.T, j = r - i * p.T;
+        e.v[0] = __ldg(p.bias + i * p.tower_stride + j);
+    } else if (p.stage == kStageFusion) {
+        const size_t row = (size_t)b * p.T + r, plane = (size_t)p.batch * p.T;
+        if (p.fus_part != 1) {
+            e.v[0] = p.in0[row];
+            e.v[1] = p.in0[plane + row];
+            e.v[2] = p.in0[2 * plane + row];
+            e.v[3] = __ldg(p.bias + r);
+        }
+        if (p.fus_part == 2) e.v[4] = p.fpre[row];
+    } else if (p.stage == kStageDown) {
+        e.v[0] = p.out[(size_t)b * p.T + r];
+    } else if (p.stage == kStageOut) {
+        e.v[0] = __ldg(p.bias);
+    }
+    return e;
+}
+
 // finishes output element (row r of the stage, request b) from the complete sums
-__device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, int b, float acc, float acc_up, float ss)
+__device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, int b, float acc, float acc_up, float ss,
+                                             const StageEpi& e)
 {
     const float rs = p.gain ? rsqrtf(ss / (float)p.K + p.eps) : 1.f;
     if (p.stage == kStageTower) {
         const int i = r / p.T, j = r - i * p.T;
-        p.out[((size_t)i * p.batch + b) * p.T + j] = silu_f(acc * rs + __ldg(p.bias + i * p.tower_stride + j));
+        p.out[((size_t)i * p.batch + b) * p.T + j] = silu_f(acc * rs + e.v[0]);
     } else if (p.stage == kStageFusion) {
-        const size_t row = (size_t)b * p.T + r, plane = (size_t)p.batch * p.T;
+        const size_t row = (size_t)b * p.T + r;
         if (p.fus_part == 1) {
             p.out[row] = acc;   // the share of W_f u that needs only a and b
         } else {
-            if (p.fus_part == 2) acc = p.fpre[row] + acc;   // fixed order: the earlier share first
-            p.out[row] = 0.5f * (p.in0[row] + p.in0[plane + row] + p.in0[2 * plane + row] + silu_f(acc + __ldg(p.bias + r)));
+            if (p.fus_part == 2) acc = e.v[4] + acc;   // fixed order: the earlier share first
+            p.out[row] = 0.5f * (e.v[0] + e.v[1] + e.v[2] + silu_f(acc + e.v[3]));
         }
     } else if (p.stage == kStageGateUp) {
         p.out[(size_t)b * p.F + r] = silu_f(acc * rs) * (acc_up * rs);
     } else if (p.stage == kStageDown) {
-        p.out[(size_t)b * p.T + r] += acc;
+        p.out[(size_t)b * p.T + r] = e.v[0] + acc;
     } else {
-        const float z = acc * rs + __ldg(p.bias);
+        const float z = acc * rs + e.v[0];
         const float score = 1.f / (1.f + expf(-z));
         uint8_t f;
         if (p.override_flags)
@@ -125,6 +155,10 @@ __device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, in
             p.counters[2 * b + 1] += f;
         }
     }
+}
+__device__ __forceinline__ void stage_finish(const FullStageParams& p, int r, int b, float acc, float acc_up, float ss)
+{
+    stage_finish(p, r, b, acc, acc_up, ss, stage_epilogue_operands(p, r, b));
 }
 
 // Tile shapes (requests x features of x in shared memory, 32 KiB either way): 4 x 2048 for small
@@ -305,23 +339,35 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                     if (!s_lastv[j]) continue;
                     const int rb2 = (int)blockIdx.x + (i0 + j) * (int)gridDim.x;
                     const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb2;
-                    for (int e = tid; e < out_rows * p.batch; e += kFThreads) {
+                    // one warp per output element: the lanes fetch the k slices' partial sums together (one
+                    // round trip, not one per slice) and add them in a fixed shuffle tree
+                    for (int e = warp; e < out_rows * p.batch; e += kFRows) {
                         const int r = e / p.batch, b = e - r * p.batch;
-                        float ss = 0.f;
-                        if (gain)
-                            for (int s2 = 0; s2 < n_ks; ++s2) ss += __ldcg(p.ssq + ((size_t)grb * n_ks + s2) * p.batch + b);
-                        auto acc_of = [&](int row) {
-                            float a = 0.f;
-                            for (int s2 = 0; s2 < n_ks; ++s2) a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
-                            return a;
-                        };
+                        int row = 0, row_up = -1;
+                        bool ok;
                         if (p.stage == kStageGateUp) {
-                            const int m = rb2 * out_rows + r;
-                            if (m < p.F) stage_finish(p, m, b, acc_of(m), acc_of(p.F + m), ss);
+                            row = rb2 * out_rows + r;
+                            row_up = p.F + row;
+                            ok = row < p.F;
                         } else {
                             const int local = rb2 * kFRows + r;
-                            if (local < (p.stage == kStageTower ? p.T : n_rows)) stage_finish(p, group_row0 + local, b, acc_of(group_row0 + local), 0.f, ss);
+                            row = group_row0 + local;
+                            ok = local < (p.stage == kStageTower ? p.T : n_rows);
                         }
+                        if (!ok) continue;  // uniform over the warp
+                        const StageEpi epi = stage_epilogue_operands(p, row, b);  // in flight with the sums below
+                        float a = 0.f, a_up = 0.f, ss = 0.f;
+                        for (int s2 = lane; s2 < n_ks; s2 += 32) {
+                            a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
+                            if (row_up >= 0) a_up += __ldcg(p.pre + ((size_t)s2 * n_rows + row_up) * p.batch + b);
+                            if (gain) ss += __ldcg(p.ssq + ((size_t)grb * n_ks + s2) * p.batch + b);
+                        }
+                        for (int o = 16; o; o >>= 1) {
+                            a += __shfl_xor_sync(0xffffffffu, a, o);
+                            a_up += __shfl_xor_sync(0xffffffffu, a_up, o);
+                            ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                        }
+                        if (lane == 0) stage_finish(p, row, b, a, a_up, ss, epi);
                     }
                 }
                 __syncthreads();  // s_lastv is reused by the next batch of tickets
