@@ -175,7 +175,8 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
     __shared__ __align__(16) float s_x[kFBT][kFKT];   // x * gain
     __shared__ float s_acc[kFRows][kFBT];
     __shared__ float s_ss[kFRows][kFBT];
-    __shared__ unsigned char s_lastv[kFThreads];
+    __shared__ unsigned char s_lastv[kFThreads], s_list[kFThreads];
+    __shared__ int s_nlast;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ks = blockIdx.y, n_ks = gridDim.y;
@@ -335,16 +336,28 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                 __threadfence();
                 __syncthreads();
                 const int n_here = min(kFThreads, n_mine - i0);
-                for (int j = 0; j < n_here; ++j) {
-                    if (!s_lastv[j]) continue;
-                    const int rb2 = (int)blockIdx.x + (i0 + j) * (int)gridDim.x;
-                    const int grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb2;
-                    // one warp per output element: the lanes fetch the k slices' partial sums together (one
-                    // round trip, not one per slice) and add them in a fixed shuffle tree
-                    for (int e = warp; e < out_rows * p.batch; e += kFRows) {
-                        const int r = e / p.batch, b = e - r * p.batch;
-                        int row = 0, row_up = -1;
-                        bool ok;
+                // the row blocks this CTA completed, in a compact list (their order does not matter: every
+                // output element is finished by itself)
+                if (tid == 0) s_nlast = 0;
+                __syncthreads();
+                if (tid < n_here && s_lastv[tid]) s_list[atomicAdd(&s_nlast, 1)] = (unsigned char)tid;
+                __syncthreads();
+                // One group of G lanes per output element (G = the power of two that holds the k slices):
+                // the lanes fetch the slices' partial sums and the epilogue's own operands together (one
+                // round trip) and add them in a fixed shuffle tree; a warp finishes 32 / G elements at a time.
+                const int G = n_ks <= 2 ? 2 : (n_ks <= 4 ? 4 : (n_ks <= 8 ? 8 : (n_ks <= 16 ? 16 : 32)));
+                const int per_warp = 32 / G, sub = lane / G, sl = lane - sub * G;
+                const int per_rb = out_rows * p.batch, total = s_nlast * per_rb;
+                for (int item0 = warp * per_warp; item0 < total; item0 += kFRows * per_warp) {
+                    const int item = item0 + sub;
+                    bool ok = item < total;
+                    int row = 0, row_up = -1, b = 0, grb = 0;
+                    if (ok) {
+                        const int jj = item / per_rb, e = item - jj * per_rb;
+                        const int r = e / p.batch;
+                        b = e - r * p.batch;
+                        const int rb2 = (int)blockIdx.x + (i0 + (int)s_list[jj]) * (int)gridDim.x;
+                        grb = (p.stage == kStageTower ? tower * group_rbs : 0) + rb2;
                         if (p.stage == kStageGateUp) {
                             row = rb2 * out_rows + r;
                             row_up = p.F + row;
@@ -354,21 +367,23 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                             row = group_row0 + local;
                             ok = local < (p.stage == kStageTower ? p.T : n_rows);
                         }
-                        if (!ok) continue;  // uniform over the warp
-                        const StageEpi epi = stage_epilogue_operands(p, row, b);  // in flight with the sums below
-                        float a = 0.f, a_up = 0.f, ss = 0.f;
-                        for (int s2 = lane; s2 < n_ks; s2 += 32) {
+                    }
+                    StageEpi epi;
+                    float a = 0.f, a_up = 0.f, ss = 0.f;
+                    if (ok) {
+                        if (sl == 0) epi = stage_epilogue_operands(p, row, b);  // in flight with the sums below
+                        for (int s2 = sl; s2 < n_ks; s2 += G) {
                             a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
                             if (row_up >= 0) a_up += __ldcg(p.pre + ((size_t)s2 * n_rows + row_up) * p.batch + b);
                             if (gain) ss += __ldcg(p.ssq + ((size_t)grb * n_ks + s2) * p.batch + b);
                         }
-                        for (int o = 16; o; o >>= 1) {
-                            a += __shfl_xor_sync(0xffffffffu, a, o);
-                            a_up += __shfl_xor_sync(0xffffffffu, a_up, o);
-                            ss += __shfl_xor_sync(0xffffffffu, ss, o);
-                        }
-                        if (lane == 0) stage_finish(p, row, b, a, a_up, ss, epi);
                     }
+                    for (int o = G >> 1; o; o >>= 1) {
+                        a += __shfl_xor_sync(0xffffffffu, a, o);
+                        a_up += __shfl_xor_sync(0xffffffffu, a_up, o);
+                        ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    }
+                    if (ok && sl == 0) stage_finish(p, row, b, a, a_up, ss, epi);
                 }
                 __syncthreads();  // s_lastv is reused by the next batch of tickets
             }
