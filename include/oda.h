@@ -299,7 +299,7 @@ oda_status_t oda_merge_partials_exchange(oda_ctx_t* ctx, int32_t world, int32_t 
  * streams all weights through a shared-memory ring and synchronises the stages with bounded grid
  * barriers (a barrier that times out after ~1 s sets bit 2 of the device status word and the kernel
  * returns).  It is kept as the measured alternative: on a B200 it is slower than the stage launches
- * (80 vs 59 us at batch 1).  Both are deterministic; they differ in summation order only.
+ * (80 vs 52 us at batch 1).  Both are deterministic; they differ in summation order only.
  *
  * Two of the head's three inputs exist before the step's Local pass (Eq. 2: q_t = R(h_{t-1}, E(x_t),
  * h_t^L)), so the head can be run in two parts.  oda_recall_score_full_pre computes what needs only

@@ -485,7 +485,8 @@ cudaError_t launch_full_head(int batch, int d_model, int T, int F, int n_blocks,
     auto launch = [&](bool dep) {
         // small batches: a 2048-wide k tile (one CTA per SM) where that divides k (towers, down: no
         // split over k), else a 1024-wide one (gate+up fits it whole; the fusion's k = 9 x 1024 splits
-        // evenly): two CTAs per SM.  Measured: 2048 everywhere 61 us, 1024 everywhere 68 us, mixed 59 us.
+        // evenly): two CTAs per SM.  Measured (before the finishing pass
+        // of the split-k stages was parallelised): 2048 everywhere 61 us, 1024 everywhere 68 us, mixed 59 us.
         const int kt = batch <= 4 ? ((p.K <= 1024 || p.K % 2048 != 0) ? 1024 : 2048) : 512;
         const int n_ks = ceil_div(p.K, kt);
         const int groups = p.stage == kStageTower ? n_towers : 1;
