@@ -44,6 +44,7 @@ struct AttnParams {
     int32_t min_span_pages;  // a CTA is not given fewer pages than this (unless there are fewer)
     int32_t l2_keep_layer_end; // Local pass: pages of layers below this one are loaded with an L2 evict-last hint (0: none)
     int32_t direct_hint;     // batch-1 Local launch whose shape allows one unit per CTA (see build_plan)
+    int32_t uniform_hint;    // batch-1 Local launch over layers of one class: every unit has the same length
     int32_t snap_span_pages; // launches with spans up to this long may be cut at unit boundaries (0: never)
     int32_t max_items;
     float scale_log2e;     // sm_scale * log2(e)
@@ -526,10 +527,15 @@ __device__ __forceinline__ int span_of_near(const Plan& pl, int x, int j, int di
     return lo;
 }
 
-// Batch 1, one unit per CTA (see build_plan): what the plan boils down to, from three registers.
+// Batch 1, Local pass: the whole plan in a few registers, the same in every thread of every CTA.
+//   ok = 1  one unit per CTA (see build_plan): CTA u streams unit u;
+//   ok = 2  layers of one class, so every unit has the same np pages: the equal split of build_plan in
+//           closed form (same cut points, chunks and partial slots: same bits), without its loads,
+//           scans and barriers -- what a launch over one or a few layers spends most of its time on.
 struct DirectPlan {
-    int32_t ok;          // the launch falls under the one-unit-per-CTA rule
-    int32_t t, cls, kv_index;
+    int32_t ok;
+    int32_t t, cls, kv_index;   // ok = 1: of this CTA's layer
+    int32_t np, total, nseg;    // ok = 2: pages per unit, pages on the axis, spans
 };
 
 // The rule of build_plan's batch-1 branch, evaluated from the one length.
@@ -550,6 +556,60 @@ __device__ __forceinline__ bool direct_rule(const AttnParams& p, int t)
     const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
     return total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
            (long long)umin * g >= total && 2ll * umax * g <= 3 * total;
+}
+
+// ok = 2: does the launch qualify, and its three numbers.  Not when the per-SM weighted split would
+// apply (a launch that fills the grid after a calibration), which needs the claims of build_plan.
+__device__ __forceinline__ bool uniform_rule(const AttnParams& p, int t, DirectPlan& d)
+{
+    if (t < 1 || t > p.max_blocks_per_seq * kPage) return false;  // the general path reports these
+    const Ranges r = eq1_ranges(0, t, p.cls_window[0], p.cls_sinks[0]);
+    const int np = r.pg1 - r.pg0;
+    const long long total = (long long)(p.layer_end - p.layer_begin) * p.num_kv_heads * np;
+    if (np < 1 || total > 0x7fffffffll) return false;
+    const int g = (int)gridDim.x;
+    const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
+    long long n = g;
+    if (total < (long long)g * minS) n = (total + minS - 1) / minS;
+    if (p.cum_share != nullptr && n == g && g == 2 * p.num_sms && g <= kMaxGrid) return false;
+    d.np = np;
+    d.total = (int32_t)total;
+    d.nseg = (int)n;
+    d.t = t;
+    return true;
+}
+__device__ __forceinline__ void uniform_span(const DirectPlan& d, int j, int& x0, int& x1)
+{
+    x0 = (int)(((long long)j * d.total) / d.nseg);
+    x1 = j + 1 >= d.nseg ? d.total : (int)(((long long)(j + 1) * d.total) / d.nseg);
+}
+// the item of span j that starts at axis page x; returns the axis pages it covers
+__device__ __forceinline__ int decode_item_uniform(const AttnParams& p, const DirectPlan& d, int j, int x, int x_end, Item& it)
+{
+    const int H = p.num_kv_heads;
+    const int u = x / d.np, off = x - u * d.np;
+    const int unit0 = x - off;
+    const int take = min(d.np - off, x_end - x);
+    // the spans that hold the unit's first and last page (equal split: span_of in closed form)
+    const int j0 = (int)((((long long)unit0 + 1) * d.nseg - 1) / d.total);
+    const int j1 = (int)((((long long)unit0 + d.np) * d.nseg - 1) / d.total);
+    const int lo = u / H;
+    const Ranges rg = eq1_ranges(0, d.t, p.cls_window[0], p.cls_sinks[0]);
+    it.layer = p.layer_begin + lo;
+    it.b = 0;
+    it.g = u - lo * H;
+    it.chunk = j - j0;
+    it.nchunks = j1 - j0 + 1;
+    it.slot_base = j0 + lo * H + it.g;
+    it.kv_layer = __ldg(&p.layers[it.layer].kv_index);
+    it.t = d.t;
+    it.win_pg0 = rg.pg0 + off;
+    it.win_pg1 = it.win_pg0 + take;
+    it.win_lo = rg.lo;
+    it.win_hi = rg.hi;
+    it.sink_hi = (off == 0) ? rg.sink_hi : 0;
+    it.sink_pg1 = (it.sink_hi + kPage - 1) / kPage;
+    return take;
 }
 
 // Unit j = (layer j / H, kv head j % H) of the only request.

@@ -149,7 +149,10 @@ struct PageRun {
     int take;
 };
 
-template <int D, int G>
+// kUniform = true: the instance launched for batch-1 Local calls over layers of one class that do not
+// qualify for one unit per CTA (a call over one or a few layers): it can take its equal split in closed
+// form from the one length.  The other instance does not carry that code.
+template <int D, int G, bool kUniform>
 __global__ void __launch_bounds__(TmaCfg<D>::kThreads, 2)
 splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__ CUtensorMap kmap,
                    const __grid_constant__ CUtensorMap vmap, const int blocks_per_layer)
@@ -166,12 +169,16 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     const uint32_t efull = smem_u32(&ctl.efull), efree = smem_u32(&ctl.efree);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // Batch-1 Local launch that may give every CTA one whole unit: the one length and this CTA's layer
-    // entry are requested first thing (after the dependency wait, which such a launch takes at once:
-    // it is the first kernel of a step), so that their latency runs while the barriers are set up.
+    // Batch-1 Local launch whose plan fits a few registers (one unit per CTA, or identical units cut
+    // into equal spans): the one length -- and for the first kind this CTA's layer entry -- are read
+    // ahead of the plan.  The one-unit-per-CTA launch is the first kernel of a step: its dependency wait
+    // returns at once, and the loads go out before the barriers are set up, whose latency they overlap.
+    // A launch over a few layers is one of a chain: its set-up runs first (it overlaps the previous
+    // launch's tail), then the wait, then the load.
     const bool direct_try = p.direct_hint && !p.sm_stats;
+    const bool early_try = (p.direct_hint || (kUniform && p.uniform_hint)) && !p.sm_stats;
     DirectPlan dp;
-    dp.ok = dp.t = dp.cls = dp.kv_index = 0;
+    dp.ok = dp.t = dp.cls = dp.kv_index = dp.np = dp.total = dp.nseg = 0;
     if (direct_try) {
         griddep_wait();
         const LayerInfo* lp = p.layers + p.layer_begin + min((int)blockIdx.x / p.num_kv_heads, p.layer_end - p.layer_begin - 1);
@@ -192,12 +199,22 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&vmap)) : "memory");
     }
     prefetch_block_table(p);
+    if (kUniform && early_try && !direct_try) {
+        griddep_wait();
+        dp.t = ld_meta_s32(p.seq_lens);
+    }
     __syncthreads();      // the barriers are initialised for every warp
-    if (!direct_try) griddep_wait();  // everything above is independent of the previous kernel in the stream
-    if (direct_try) dp.ok = direct_rule(p, dp.t);  // same registers in every thread: no barrier, no shared plan
+    if (!early_try) griddep_wait();  // everything above is independent of the previous kernel in the stream
+    // same registers in every thread: no barrier, no shared plan
+    if (direct_try && direct_rule(p, dp.t)) dp.ok = 1;
+    if constexpr (kUniform) {
+        if (!dp.ok && early_try && p.uniform_hint && uniform_rule(p, dp.t, dp)) dp.ok = 2;
+    }
     int span;             // the one span this CTA streams
-    if (dp.ok) {
+    if (dp.ok == 1) {
         span = (int)blockIdx.x < (p.layer_end - p.layer_begin) * p.num_kv_heads ? (int)blockIdx.x : -1;
+    } else if (kUniform && dp.ok == 2) {
+        span = (int)blockIdx.x < dp.nseg ? (int)blockIdx.x : -1;
     } else {
         if (gated_pass_is_empty(p)) {
             griddep_launch_dependents();
@@ -220,8 +237,11 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
         // walker over the runs of the CTA's span
         int x = 0, x_end = 1, take = 1;  // a one-unit-per-CTA span is [0, 1) on a nominal axis
         Item it;
-        if (dp.ok) {
+        if (dp.ok == 1) {
             decode_item_direct(p, dp, span, it);
+        } else if (kUniform && dp.ok == 2) {
+            uniform_span(dp, span, x, x_end);
+            take = decode_item_uniform(p, dp, span, x, x_end, it);
         } else {
             span_range(plan, span, x, x_end);
             take = decode_item(p, plan, span, x, x_end, it);
@@ -241,7 +261,8 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             if (v >= nv) {
                 x += take;
                 if (x < x_end) {
-                    take = decode_item(p, plan, span, x, x_end, it);
+                    take = (kUniform && dp.ok == 2) ? decode_item_uniform(p, dp, span, x, x_end, it)
+                                                    : decode_item(p, plan, span, x, x_end, it);
                     v = 0;
                     nv = item_pages(it);
                     item_first = true;
@@ -499,7 +520,8 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
     int pages_done = 0, pages_half = 0;
     {
         int x = 0, x_end = 1;
-        if (!dp.ok) span_range(plan, span, x, x_end);
+        if (kUniform && dp.ok == 2) uniform_span(dp, span, x, x_end);
+        else if (!dp.ok) span_range(plan, span, x, x_end);
         span_pages = x_end - x;
         while (x < x_end && !aborted) {
             Item it;
@@ -778,14 +800,23 @@ static cudaError_t launch_tma_t(const AttnParams& p, const void* kmap, const voi
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(splitkv_tma_kernel<D, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              TmaCfg<D>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(splitkv_tma_kernel<D, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     TmaCfg<D>::kSmemBytes);
         if (e != cudaSuccess) return e;
-        (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                   cudaSharedmemCarveoutMaxShared);
+        (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                    cudaSharedmemCarveoutMaxShared);
         attr_set = true;
     }
-    return launch_ex(splitkv_tma_kernel<D, G>, dim3(grid), dim3(TmaCfg<D>::kThreads), TmaCfg<D>::kSmemBytes, st, pdl,
+    if (p.uniform_hint && !p.direct_hint)
+        return launch_ex(splitkv_tma_kernel<D, G, true>, dim3(grid), dim3(TmaCfg<D>::kThreads), TmaCfg<D>::kSmemBytes, st,
+                         pdl, p, *reinterpret_cast<const CUtensorMap*>(kmap), *reinterpret_cast<const CUtensorMap*>(vmap),
+                         blocks_per_layer);
+    return launch_ex(splitkv_tma_kernel<D, G, false>, dim3(grid), dim3(TmaCfg<D>::kThreads), TmaCfg<D>::kSmemBytes, st, pdl,
                      p, *reinterpret_cast<const CUtensorMap*>(kmap), *reinterpret_cast<const CUtensorMap*>(vmap),
                      blocks_per_layer);
 }
@@ -794,14 +825,14 @@ template <int D, int G>
 static int occupancy_tma_t()
 {
     int n = 0;
-    if (cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(splitkv_tma_kernel<D, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TmaCfg<D>::kSmemBytes) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }
-    (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    (void)cudaFuncSetAttribute(splitkv_tma_kernel<D, G, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, splitkv_tma_kernel<D, G>, TmaCfg<D>::kThreads,
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, splitkv_tma_kernel<D, G, false>, TmaCfg<D>::kThreads,
                                                   TmaCfg<D>::kSmemBytes);
     return n;
 }

@@ -373,3 +373,40 @@ def test_batch_one_unit_per_cta_parity(layout, t):
     np.testing.assert_array_equal(again, out)
     assert ctx.read_device_status() == 0
 
+
+
+@pytest.mark.parametrize("layout,Hq,Hkv,D,w,s", [("hnd", 32, 8, 128, 1024, 4), ("nhd", 8, 2, 128, 256, 0),
+                                                 ("hnd", 8, 1, 64, 100, 17), ("hnd", 16, 2, 128, 2048, 4)])
+def test_batch_one_identical_units_plan_in_registers(layout, Hq, Hkv, D, w, s):
+    """Batch 1 over layers of one class: every unit has the same length and the equal split is taken in
+    closed form from the one length (no shared plan).  Whole stacks and layer ranges (one launch per
+    layer is what a backbone issues), lengths around the page, sink and window edges; the layers alias
+    cache slices so that the per-item layer lookup is exercised; same bits on a second run, and the
+    same bits as the same request inside a batch of two (which takes the general plan)."""
+    L = 5
+    kv_index = [l % 2 for l in range(L)]
+    for t in (1, 16, 17, w + s - 1, w + s, w + s + 1, 3 * w + 9):
+        prob = make_problem(4000 + t, L, 1, Hq, Hkv, D, [t], layout=layout, kv_layers=2)
+        ctx = gh.make_ctx(prob, [w] * L, [s] * L, [1] * L, kv_index=kv_index, variant=binding.VARIANT_TMA_MMA)
+        dev = gh.upload(prob)
+        ref, rlse = oracle_attention(prob, "local", [w] * L, [s] * L, nthreads=8, layer_kv_index=kv_index)
+        whole, whole_lse = gh.gpu_local(ctx, prob, dev)
+        gh.assert_close(whole, ref, gh.ATOL_OUT, f"t={t} whole stack")
+        gh.assert_close(whole_lse, rlse, gh.ATOL_LSE, f"t={t} whole stack lse")
+        for lb, le in ((0, 1), (2, 3), (1, 4), (4, 5)):
+            out, lse = gh.gpu_local(ctx, prob, dev, lb, le)
+            gh.assert_close(out[lb:le], ref[lb:le], gh.ATOL_OUT, f"t={t} layers [{lb},{le})")
+            gh.assert_close(lse[lb:le], rlse[lb:le], gh.ATOL_LSE, f"t={t} layers [{lb},{le}) lse")
+            assert np.isnan(out[:lb]).all() and np.isnan(out[le:]).all()      # other layers untouched
+        again, _ = gh.gpu_local(ctx, prob, dev)
+        np.testing.assert_array_equal(again, whole)
+        # the same request as request 0 of a batch of two: the general plan cuts the same spans
+        prob2 = dict(prob, B=2, q=np.ascontiguousarray(np.repeat(prob["q"], 2, axis=1)),
+                     table=np.ascontiguousarray(np.repeat(prob["table"], 2, axis=0)),
+                     seq_lens=np.array([t, t], np.int32))
+        ctx2 = gh.make_ctx(prob2, [w] * L, [s] * L, [1] * L, kv_index=kv_index, variant=binding.VARIANT_TMA_MMA)
+        dev2 = gh.upload(prob2)
+        both, _ = gh.gpu_local(ctx2, prob2, dev2)
+        gh.assert_close(both[:, 0], ref[:, 0], gh.ATOL_OUT, f"t={t} as request 0 of two")
+        gh.assert_close(both[:, 1], ref[:, 0], gh.ATOL_OUT, f"t={t} as request 1 of two")
+        assert ctx.read_device_status() == 0 and ctx2.read_device_status() == 0
