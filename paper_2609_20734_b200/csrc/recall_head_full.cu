@@ -342,12 +342,16 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                 __syncthreads();
                 if (tid < n_here && s_lastv[tid]) s_list[atomicAdd(&s_nlast, 1)] = (unsigned char)tid;
                 __syncthreads();
-                // One group of G lanes per output element (G = the power of two that holds the k slices):
-                // the lanes fetch the slices' partial sums and the epilogue's own operands together (one
-                // round trip) and add them in a fixed shuffle tree; a warp finishes 32 / G elements at a time.
-                const int G = n_ks <= 2 ? 2 : (n_ks <= 4 ? 4 : (n_ks <= 8 ? 8 : (n_ks <= 16 ? 16 : 32)));
-                const int per_warp = 32 / G, sub = lane / G, sl = lane - sub * G;
+                // One group of G lanes per output element: the lanes fetch the k slices' partial sums (four
+                // in flight per lane) and the epilogue's own operands together and add them in a fixed order
+                // (per lane, then a shuffle tree); a warp finishes 32 / G elements at a time.  G is as large
+                // as the number of elements leaves room for in one pass of the CTA (few elements at batch 1:
+                // a group per element, one round trip; many at batch 16: a thread per element), and no
+                // larger than the power of two that holds the slices.
                 const int per_rb = out_rows * p.batch, total = s_nlast * per_rb;
+                int G = 1;
+                while (G < 32 && G < n_ks && 2 * G * total <= kFThreads) G <<= 1;
+                const int per_warp = 32 / G, sub = lane / G, sl = lane - sub * G;
                 for (int item0 = warp * per_warp; item0 < total; item0 += kFRows * per_warp) {
                     const int item = item0 + sub;
                     bool ok = item < total;
@@ -372,10 +376,19 @@ __global__ void __launch_bounds__(kFThreads, (kFKT >= 2048 ? 1 : 2)) full_head_s
                     float a = 0.f, a_up = 0.f, ss = 0.f;
                     if (ok) {
                         if (sl == 0) epi = stage_epilogue_operands(p, row, b);  // in flight with the sums below
-                        for (int s2 = sl; s2 < n_ks; s2 += G) {
-                            a += __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b);
-                            if (row_up >= 0) a_up += __ldcg(p.pre + ((size_t)s2 * n_rows + row_up) * p.batch + b);
-                            if (gain) ss += __ldcg(p.ssq + ((size_t)grb * n_ks + s2) * p.batch + b);
+                        for (int s0 = sl; s0 < n_ks; s0 += 4 * G) {
+                            float v[4], vu[4], vs[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int s2 = s0 + q * G;
+                                const bool in = s2 < n_ks;
+                                v[q] = in ? __ldcg(p.pre + ((size_t)s2 * n_rows + row) * p.batch + b) : 0.f;
+                                vu[q] = (in && row_up >= 0) ? __ldcg(p.pre + ((size_t)s2 * n_rows + row_up) * p.batch + b) : 0.f;
+                                vs[q] = (in && gain) ? __ldcg(p.ssq + ((size_t)grb * n_ks + s2) * p.batch + b) : 0.f;
+                            }
+                            a += (v[0] + v[1]) + (v[2] + v[3]);
+                            a_up += (vu[0] + vu[1]) + (vu[2] + vu[3]);
+                            ss += (vs[0] + vs[1]) + (vs[2] + vs[3]);
                         }
                     }
                     for (int o = G >> 1; o; o >>= 1) {
