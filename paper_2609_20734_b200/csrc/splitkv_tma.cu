@@ -409,9 +409,13 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
             } else {
                 float4* slots = reinterpret_cast<float4*>(p.partials) + (size_t)it.slot_base * (kFragSlotFloats / 4);
                 float4* mine = slots + (size_t)it.chunk * (kFragSlotFloats / 4);
-                // If every other chunk of the unit has already arrived (the usual case for the last
-                // item of a span: its neighbour finished that unit long ago), this CTA merges, and its own
-                // chunk never has to leave its registers: no partial store, fence and ticket round trips.
+                // The partial goes out first; while it is on its way, a look at the ticket: if every other
+                // chunk of the unit has already arrived (the usual case for the last item of a span: its
+                // neighbour finished that unit long ago) this CTA merges straight from its registers and
+                // needs neither the fence nor its own ticket (the partial it wrote is then never read).
+#pragma unroll
+                for (int n = 0; n < D / 16; ++n) __stcg(mine + n * 32 + lane, make_float4(o[n][0], o[n][1], o[n][2], o[n][3]));
+                __stcg(mine + 8 * 32 + lane, ml);
                 int last = 0;
                 if (lane == 0) {
                     int* tk = p.tickets + ((size_t)it.layer * p.max_batch + it.b) * p.num_kv_heads + it.g;
@@ -424,9 +428,6 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 }
                 last = __shfl_sync(0xffffffffu, last, 0);
                 if (!last) {
-#pragma unroll
-                    for (int n = 0; n < D / 16; ++n) __stcg(mine + n * 32 + lane, make_float4(o[n][0], o[n][1], o[n][2], o[n][3]));
-                    __stcg(mine + 8 * 32 + lane, ml);
                     __threadfence();
                     __syncwarp();
                     if (lane == 0) last = take_ticket(p, it);
