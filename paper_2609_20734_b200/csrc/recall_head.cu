@@ -42,7 +42,10 @@ __device__ __forceinline__ float4 head_x4(const HeadParams& p, int b, int i)
 // publishes the partial pre-activations.  The last CTA of a row block (atomic ticket, no
 // waiting) adds the K slices in order, applies bias, SiLU and w2; the last row block adds the
 // row blocks' sums in a fixed tree and writes score, logit, flag and counters.  Every sum has a
-// fixed order, so the result does not depend on scheduling.
+// fixed order, so the result does not depend on scheduling.  A head whose inputs fit one K slice
+// (d_in <= 512) skips the first level: the row block's sums go from the warps to the CTA's shared
+// memory, with no fence, ticket or reload.
+template <bool kDirect>
 __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_constant__ HeadParams p)
 {
     __shared__ __align__(16) float s_x[kHeadBT][kHeadKT];
@@ -54,6 +57,7 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
     const int j = rb * kHeadRows + warp;
     const int d_in = p.d_ext + p.d_attn;
     const int k0 = ks * kHeadKT;
+    constexpr bool direct = kDirect;   // one K slice: the row block's sums stay in the CTA
     // this lane's 16 weights of row j: features k0 + c*128 + lane*4 + e
     float w[4][4];
 #pragma unroll
@@ -108,41 +112,65 @@ __global__ void __launch_bounds__(kHeadThreads) recall_head_kernel(const __grid_
         for (int u = 0; u < kHeadBT; ++u) {
             float a = acc[u];
             for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-            if (lane == 0 && b0 + u < p.batch && j < p.d_hidden)
-                __stcg(p.pre + ((size_t)ks * p.d_hidden + j) * p.max_batch + b0 + u, a);
+            if (lane == 0 && b0 + u < p.batch && j < p.d_hidden) {
+                if (direct)
+                    s_h[warp][b0 + u] = a;
+                else
+                    __stcg(p.pre + ((size_t)ks * p.d_hidden + j) * p.max_batch + b0 + u, a);
+            }
         }
     }
-    // ---- row block complete?  (last of its n_ks K slices)
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int old = atomicAdd(p.rb_tickets + rb, 1);
-        s_last = (old == n_ks - 1);
-        if (s_last) p.rb_tickets[rb] = 0;
+    if (!direct) {
+        // ---- row block complete?  (last of its n_ks K slices)
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const int old = atomicAdd(p.rb_tickets + rb, 1);
+            s_last = (old == n_ks - 1);
+            if (s_last) p.rb_tickets[rb] = 0;
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+    } else {
+        __syncthreads();
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
     if (p.pre_out) {  // column-split head: this rank's share of W1 x, K slices added in order
         for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
             const int b = e / kHeadRows, jj = rb * kHeadRows + (e - b * kHeadRows);
             if (jj >= p.d_hidden) continue;
             float a = 0.f;
-            for (int s = 0; s < n_ks; ++s) a += __ldcg(p.pre + ((size_t)s * p.d_hidden + jj) * p.max_batch + b);
+            if (direct)
+                a = s_h[e - b * kHeadRows][b];
+            else
+                for (int s = 0; s < n_ks; ++s) a += __ldcg(p.pre + ((size_t)s * p.d_hidden + jj) * p.max_batch + b);
             p.pre_out[(size_t)b * p.d_hidden + jj] = a;
         }
         return;
     }
-    for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
-        const int r = e / p.batch, b = e - r * p.batch;
-        const int jj = rb * kHeadRows + r;
-        float hv = 0.f;
-        if (jj < p.d_hidden) {
-            float a = __ldg(p.b1 + jj);
-            for (int s = 0; s < n_ks; ++s) a += __ldcg(p.pre + ((size_t)s * p.d_hidden + jj) * p.max_batch + b);
-            hv = __ldg(p.w2 + jj) * (a / (1.f + expf(-a)));
+    if (direct) {
+        for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
+            const int r = e / p.batch, b = e - r * p.batch;
+            const int jj = rb * kHeadRows + r;
+            float hv = 0.f;
+            if (jj < p.d_hidden) {
+                const float a = __ldg(p.b1 + jj) + s_h[r][b];
+                hv = __ldg(p.w2 + jj) * (a / (1.f + expf(-a)));
+            }
+            s_h[r][b] = hv;   // each element is read and written by its own thread
         }
-        s_h[r][b] = hv;
+    } else {
+        for (int e = tid; e < kHeadRows * p.batch; e += kHeadThreads) {
+            const int r = e / p.batch, b = e - r * p.batch;
+            const int jj = rb * kHeadRows + r;
+            float hv = 0.f;
+            if (jj < p.d_hidden) {
+                float a = __ldg(p.b1 + jj);
+                for (int s = 0; s < n_ks; ++s) a += __ldcg(p.pre + ((size_t)s * p.d_hidden + jj) * p.max_batch + b);
+                hv = __ldg(p.w2 + jj) * (a / (1.f + expf(-a)));
+            }
+            s_h[r][b] = hv;
+        }
     }
     __syncthreads();
     for (int b = tid; b < p.batch; b += kHeadThreads) {
@@ -254,8 +282,10 @@ cudaError_t launch_recall_head(const HeadParams& p, cudaStream_t st, bool pdl)
     if (p.d_hidden <= 0)
         return launch_ex(copy_flags_kernel, dim3(1), dim3(128), 0, st, pdl, p.override_flags, p.flags, p.scores,
                          p.logits, p.counters, p.batch);
-    return launch_ex(recall_head_kernel, dim3(recall_head_grid(p.d_hidden), recall_head_ksplits(p.d_ext + p.d_attn)),
-                     dim3(kHeadThreads), 0, st, pdl, p);
+    const int n_ks = recall_head_ksplits(p.d_ext + p.d_attn);
+    if (n_ks == 1 && p.batch <= kMaxHeadBatch)
+        return launch_ex(recall_head_kernel<true>, dim3(recall_head_grid(p.d_hidden), 1), dim3(kHeadThreads), 0, st, pdl, p);
+    return launch_ex(recall_head_kernel<false>, dim3(recall_head_grid(p.d_hidden), n_ks), dim3(kHeadThreads), 0, st, pdl, p);
 }
 
 cudaError_t launch_recall_finalize(const HeadParams& p, const float* pre_sum, cudaStream_t st, bool pdl)
