@@ -42,6 +42,9 @@ def test_bench_prints_one_contract_line():
     ps = d["passes"]
     assert ps["measured"] == 3 and sorted(ps["ms_per_step"])[1] == d["ms_per_step"]
     assert d["roofline_other"]["floor_us"] > 0 and d["roofline_other"]["frac_above_floor"] > d["roofline_other"]["frac"]
+    # the Local launch once more with its code warm and its data cold: context beside the flushed figure
+    cw = d["roofline_other"]["code_warm"]
+    assert 0 < cw["us"] < 2 * d["roofline_other"]["us"] and cw["frac"] > 0
     # the arm-specific descriptions sit beside `config`, which both arms fill identically
     assert "launch" in d and "arithmetic" in d and "launch" not in d["config"]
     (tiny,) = d["configs"]
