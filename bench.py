@@ -387,7 +387,7 @@ class Runner:
     """One workload resident on this rank's GPU, its step captured in one CUDA graph, and the timing
     loops over it.  Every replay reads lengths and flags on the device."""
 
-    def __init__(self, torch, args, wl, flush, side, *, steps, warmup, calibrate=True, paper_head=None):
+    def __init__(self, torch, args, wl, flush, side, *, steps, warmup, calibrate=True, paper_head=None, calib_passes=2):
         from paper_2609_20734_b200 import binding, workloads
 
         self.torch, self.args, self.wl, self.flush, self.side = torch, args, wl, flush, side
@@ -422,9 +422,9 @@ class Runner:
             override_flags=None if self.head_decides else self.ov_s, lse=self.lse, counters=self.counters,
             advance_seq_lens=True, full_head=paper_head)
         self.calib = 0.0
-        if calibrate and not args.no_calibrate:  # set-up, once: per-SM streaming rates measured on two all-flagged Full passes
+        if calibrate and not args.no_calibrate:  # set-up, once: per-SM streaming rates measured on all-flagged Full passes
             ctx.calibration_begin()
-            for _ in range(2):
+            for _ in range(calib_passes):
                 ctx.full_decode_gated(0, L, B, self.qs[0], st.k_cache, st.v_cache, st.block_table, st.seq_lens,
                                       self.ones, self.out, self.lse)
             self.calib = ctx.calibration_end()
@@ -610,11 +610,11 @@ def extra_config(torch, args, name, steps, flush, side, peak):
         # layer, with the context cut down to what the windows need (Local's bytes do not depend on it).
         short = int(4 * max(wl.windows))
         wl2 = replace(workloads.make(name), kv_index=None, seq_lens0=np.full(wl.B, short, np.int32))
-        r2 = Runner(torch, args, wl2, flush, side, steps=1, warmup=1, calibrate=False)
+        r2 = Runner(torch, args, wl2, flush, side, steps=1, warmup=1, calib_passes=16)   # short passes: more of them
         kt2 = r2.time_launches(["local"], max(3, args.kernel_reps // 2), warm=False)
         lb2, _ = wl2.algorithmic_bytes(np.asarray(wl2.seq_lens0), np.ones(wl.B))
         entry["local"] = roofline_entry(lb2, kt2["local"]["us"], peak,
-                                        {"measured_on": f"one cache slice per layer, context {short} (no aliasing)"})
+                                        {"measured_on": f"one cache slice per layer, context {short} (no aliasing), per-SM split calibrated on that stack"})
         entry["whole_step_note"] = (f"{wl.L} layers share {wl.phys_layers} physical cache slices (the full-size cache does "
                                     "not fit); inside the step the Local pass therefore sees some L2 hits it would not "
                                     "see on a real stack; its stand-alone figure is taken without aliasing")
