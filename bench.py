@@ -588,6 +588,29 @@ def extra_config(torch, args, name, steps, flush, side, peak):
              "tokens_per_s": wl.B * steps / (med * 1e-3),
              "step_gbs": r.step_bytes(fl) / (med / steps * 1e-3) / 1e9,
              "launches_per_step": r.launches_per_step}
+    if name == "70b" and r.ovs is not None and not args.no_sweep:
+        # this configuration's own recall-rate sweep: per-request draws, so a step reads the history of the
+        # flagged requests only and its time must be affine in the realised rate
+        sweep, n_sw = [], 10
+        for rate in (0.0, 0.1, 0.3, 1.0):
+            wl_r = workloads.make(name, recall_rate=rate, **ov)
+            fl_r = schedule_flags(wl_r, 0, n_sw)
+            r.st.seq_lens.copy_(r.seq0)
+            tms = []
+            for s_ in range(n_sw):
+                r.q_s.copy_(r.qs[s_ % r.nsteps])
+                r.ov_s.copy_(torch.from_numpy(fl_r[s_]).cuda())
+                tms.append(timed_replay(torch, r.graph, flush, s_ & 0xFF))
+            bts = np.mean([sum(wl.algorithmic_bytes(np.asarray(wl.seq_lens0) + s_, fl_r[s_])) for s_ in range(n_sw)])
+            sweep.append({"rate": rate, "realised": float(np.mean([f.mean() for f in fl_r])), "ms_per_step": float(np.mean(tms)),
+                          "tokens_per_s": wl.B / (float(np.mean(tms)) * 1e-3), "gbs": float(bts) / (float(np.mean(tms)) * 1e-3) / 1e9})
+        x, y = np.array([e["realised"] for e in sweep]), np.array([e["ms_per_step"] for e in sweep])
+        A = np.vstack([x, np.ones_like(x)]).T
+        coef = np.linalg.lstsq(A, y, rcond=None)[0]
+        ss_tot = float(((y - y.mean()) ** 2).sum())
+        entry["sweep"] = sweep
+        entry["affine_fit"] = {"slope_ms": float(coef[0]), "intercept_ms": float(coef[1]),
+                               "r2": 1.0 - float(((A @ coef - y) ** 2).sum()) / ss_tot if ss_tot > 0 else 1.0}
     which = ["full"] + (["head"] if wl.head else [])
     aliased = wl.kv_index is not None and len(set(wl.kv_index)) < wl.L
     if not aliased:
