@@ -417,7 +417,9 @@ splitkv_tma_kernel(const __grid_constant__ AttnParams p, const __grid_constant__
                 for (int n = 0; n < D / 16; ++n) __stcg(mine + n * 32 + lane, make_float4(o[n][0], o[n][1], o[n][2], o[n][3]));
                 __stcg(mine + 8 * 32 + lane, ml);
                 int last = 0;
-                if (lane == 0) {
+                // (not in launches whose units are all cut alike: their chunks finish together, the look
+                // would only add a round trip)
+                if (!kUniform && lane == 0) {
                     int* tk = p.tickets + ((size_t)it.layer * p.max_batch + it.b) * p.num_kv_heads + it.g;
                     int seen;
                     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(tk) : "memory");
