@@ -212,7 +212,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     if (advanced) *advanced = advance != nullptr;
     // A Local call over few layers cannot fill the usual grid: the window bounds its pages whatever
     // the lengths are.  Launch only the CTAs the plan can give a span to (it cuts the page axis into
-    // min(grid, pages / min_span_pages) spans either way, so the split and the bits are the same);
+    // min(grid, max(1, pages / min_span_pages)) spans either way, so the split and the bits are the same);
     // the rest would only start, build the plan and leave.
     int grid = c->grid;
     if (mode == 0 && c->min_span_pages > 0) {
@@ -222,7 +222,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
             const long long tokens = (long long)c->cls_window[cls] + c->cls_sinks[cls];  // one range when they touch
             bound += (long long)batch * f.num_kv_heads * (tokens / kPage + 2);
         }
-        const long long need = (bound + c->min_span_pages - 1) / c->min_span_pages;
+        const long long need = bound / c->min_span_pages;   // the plan rounds down too
         if (need < grid) grid = (int)std::max<long long>(need, 1);
     }
     {   // necessary for the batch-1 one-unit-per-CTA plan, whatever the length turns out to be

@@ -314,7 +314,9 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             const int g = (int)gridDim.x;
             const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
             long long n = g;  // the usual case, without the division
-            if (carry < (long long)g * minS) n = (carry + minS - 1) / minS;
+            // (rounded down: a launch of 17 pages is one span, not two of eight and a half with a merge
+            // between them, and units of 65 pages on spans of 16 are cut at their own boundaries)
+            if (carry < (long long)g * minS) n = carry > 0 ? max(1ll, carry / minS) : 0;
             nseg = (int)n;
             pl.nseg = nseg;
             // the weighted split needs every CTA to have real work; small launches stay equal
@@ -570,7 +572,7 @@ __device__ __forceinline__ bool uniform_rule(const AttnParams& p, int t, DirectP
     const int g = (int)gridDim.x;
     const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
     long long n = g;
-    if (total < (long long)g * minS) n = (total + minS - 1) / minS;
+    if (total < (long long)g * minS) n = max(1ll, total / minS);
     if (p.cum_share != nullptr && n == g && g == 2 * p.num_sms && g <= kMaxGrid) return false;
     d.np = np;
     d.total = (int32_t)total;
