@@ -227,7 +227,7 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     }
     {   // necessary for the batch-1 one-unit-per-CTA plan, whatever the length turns out to be
         const long long units = (long long)(le - lb) * f.num_kv_heads;
-        p.direct_hint = (mode == 0 && batch == 1 && c->snap_span_pages > 0 && units <= grid && 2ll * grid <= 3 * units) ? 1 : 0;
+        p.direct_hint = (mode == 0 && batch == 1 && c->snap_span_pages > 0 && units <= grid && grid <= 4 * units) ? 1 : 0;
         // one request and one layer class in the call: every unit has the same length, whatever it turns out to be
         int classes_in_call = 0;
         for (int i = 0; i < c->ncls; ++i) classes_in_call += p.cls_layers_in_call[i] > 0;

@@ -181,7 +181,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
     // same length, so whether the launch falls under the unit-aligned rule (see below) follows from
     // the one length alone, and then CTA u simply takes unit u = (layer u / H, kv head u % H).  No
     // scans, no claims, one barrier: this is the latency-critical launch of batch-1 decoding.
-    if (p.direct_hint && !p.sm_stats) {  // host side of the rule: mode 0, batch 1, units <= CTAs <= 3/2 units
+    if (p.direct_hint && !p.sm_stats) {  // host side of the rule: mode 0, batch 1, units <= CTAs <= 4 units
         const int g = (int)gridDim.x, H = p.num_kv_heads;
         const int t = p.seq_lens[0];
         LayerInfo li;
@@ -201,7 +201,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         }
         const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
         if (total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
-            (long long)umin * g >= total && 2ll * umax * g <= 3 * total) {
+            (long long)umin * g >= total && (long long)umax * g <= 4 * total) {
             if (tid == 0) {
                 pl.snap = 2;
                 pl.weighted = 0;
@@ -346,8 +346,9 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         // merge at the end, where a launch of a few tens of microseconds notices them.  Some CTAs
         // get no unit; such a launch is bound by DRAM, not by the number of streaming CTAs.  Not
         // during calibration (which measures the equal split), and not when units are shorter than
-        // a span (some CTAs would get two: measured 4-6 us slower than the equal split) or much
-        // longer (idle CTAs).
+        // a span (some CTAs would get two: measured 4-6 us slower than the equal split) or more
+        // than four spans long (measured: up to there one CTA per unit is 7-18 % faster than an
+        // equal split whose spans straddle the units, beyond it a lone CTA's own rate sets the time).
         span = __shfl_sync(0xffffffffu, span, 0);
         nseg = __shfl_sync(0xffffffffu, nseg, 0);
         const int total = (int)__shfl_sync(0xffffffffu, (int)carry, 0);
@@ -358,7 +359,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
                 umin = min(umin, pl.umin[c]);
                 umax = max(umax, pl.umax[c]);
             }
-            if (umin * nseg >= total && 2 * umax * nseg <= 3 * total) {  // span <= unit <= 3/2 span
+            if (umin * nseg >= total && (long long)umax * nseg <= 4ll * total) {  // span <= unit <= 4 spans
                 __syncwarp();  // lb[] was written by other lanes of this warp
                 int x = 0;
                 const int j = span + lane;  // lane 0: where the span starts, lane 1: where it ends
@@ -557,7 +558,7 @@ __device__ __forceinline__ bool direct_rule(const AttnParams& p, int t)
     }
     const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
     return total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
-           (long long)umin * g >= total && 2ll * umax * g <= 3 * total;
+           (long long)umin * g >= total && (long long)umax * g <= 4 * total;
 }
 
 // ok = 2: does the launch qualify, and its three numbers.  Not when the per-SM weighted split would
