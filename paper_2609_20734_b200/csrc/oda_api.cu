@@ -42,7 +42,7 @@ struct oda_ctx {
     int grid = 148;
     int min_span_pages = 16;  // four whole tiles; measured against 8 (one-layer launches 14.0 -> 13.4 us) and 12 / 24 (ragged tiles: slower)
     size_t l2_resident_bytes = 0;  // Local working set to keep in L2 between steps (oda_set_cache_resident_bytes)
-    int snap_span_pages = 128;  // launches of up to 1 MiB per CTA may be cut at unit boundaries
+    int snap_span_pages = 256;  // launches of up to 2 MiB per CTA may be cut at unit boundaries (measured against 128 and 512)
     bool calibrated = false;  // the per-SM split table in the workspace is valid
     bool calibrating = false; // attention launches record per-SM streaming rates
     double calib_spread = 0.0; // slowest / fastest SM share seen by oda_calibrate
