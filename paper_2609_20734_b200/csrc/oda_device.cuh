@@ -172,6 +172,16 @@ __device__ __forceinline__ Ranges eq1_ranges(int mode, int t, int w, int s)
 
 // Every CTA builds the same plan from device-resident seq_lens / flags: no host knowledge of
 // lengths or flags is needed, so one captured launch serves every length and every gate.
+// Shape test of the unit-aligned split (one CTA streams a whole unit and writes its rows: no partials, no
+// merge): units between one and four spans long -- shorter ones would double up on some CTAs -- and not so
+// long that a CTA alone on its unit takes longer than the equal split would.  Measured: a CTA streams a page
+// (K and V of 16 positions of one head) in about 0.18 us, a DRAM-bound launch as a whole moves one in 0.0012 us,
+// and the equal split costs about 5 us of partials and merges: 0.18 umax <= 0.0012 total + 5, in integers.
+__device__ __forceinline__ bool unit_aligned_shape(long long total, int umin, int umax, int nseg)
+{
+    return (long long)umin * nseg >= total && (long long)umax * nseg <= 4 * total && 150ll * umax <= total + 4200;
+}
+
 __device__ inline void build_plan(const AttnParams& p, Plan& pl)
 {
     const int tid = threadIdx.x, nth = blockDim.x;
@@ -200,8 +210,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
             }
         }
         const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
-        if (total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
-            (long long)umin * g >= total && (long long)umax * g <= 4 * total) {
+        if (total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g && unit_aligned_shape(total, umin, umax, g)) {
             if (tid == 0) {
                 pl.snap = 2;
                 pl.weighted = 0;
@@ -346,9 +355,9 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
         // merge at the end, where a launch of a few tens of microseconds notices them.  Some CTAs
         // get no unit; such a launch is bound by DRAM, not by the number of streaming CTAs.  Not
         // during calibration (which measures the equal split), and not when units are shorter than
-        // a span (some CTAs would get two: measured 4-6 us slower than the equal split) or more
-        // than four spans long (measured: up to there one CTA per unit is 7-18 % faster than an
-        // equal split whose spans straddle the units, beyond it a lone CTA's own rate sets the time).
+        // a span (some CTAs would get two: measured 4-6 us slower than the equal split), more than
+        // four spans long, or so long that a CTA alone on its unit would be the bottleneck
+        // (unit_aligned_shape).
         span = __shfl_sync(0xffffffffu, span, 0);
         nseg = __shfl_sync(0xffffffffu, nseg, 0);
         const int total = (int)__shfl_sync(0xffffffffu, (int)carry, 0);
@@ -359,7 +368,7 @@ __device__ inline void build_plan(const AttnParams& p, Plan& pl)
                 umin = min(umin, pl.umin[c]);
                 umax = max(umax, pl.umax[c]);
             }
-            if (umin * nseg >= total && (long long)umax * nseg <= 4ll * total) {  // span <= unit <= 4 spans
+            if (unit_aligned_shape(total, umin, umax, nseg)) {
                 __syncwarp();  // lb[] was written by other lanes of this warp
                 int x = 0;
                 const int j = span + lane;  // lane 0: where the span starts, lane 1: where it ends
@@ -557,8 +566,7 @@ __device__ __forceinline__ bool direct_rule(const AttnParams& p, int t)
         umax = max(umax, np);
     }
     const int minS = p.min_span_pages > 0 ? p.min_span_pages : 1;
-    return total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g &&
-           (long long)umin * g >= total && (long long)umax * g <= 4 * total;
+    return total >= (long long)g * minS && total <= (long long)p.snap_span_pages * g && unit_aligned_shape(total, umin, umax, g);
 }
 
 // ok = 2: does the launch qualify, and its three numbers.  Not when the per-SM weighted split would
