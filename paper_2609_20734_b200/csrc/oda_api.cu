@@ -227,7 +227,15 @@ oda_status_t launch_attention(oda_ctx* c, int mode, int lb, int le, int batch, c
     }
     {   // necessary for the batch-1 one-unit-per-CTA plan, whatever the length turns out to be
         const long long units = (long long)(le - lb) * f.num_kv_heads;
-        p.direct_hint = (mode == 0 && batch == 1 && c->snap_span_pages > 0 && units <= grid && grid <= 4 * units) ? 1 : 0;
+        // (the last condition of unit_aligned_shape at the longest unit the windows allow: where it fails, the
+        // launch is better off with the plan in registers than with a hint the device then turns down)
+        long long umax_bound = 0;
+        for (int l = lb; l < le; ++l) {
+            const int cls = c->layers[l].cls;
+            umax_bound = std::max(umax_bound, ((long long)c->cls_window[cls] + c->cls_sinks[cls]) / kPage + 2);
+        }
+        const bool lone_cta_ok = units >= 150 || umax_bound * (150 - units) <= 4200;
+        p.direct_hint = (mode == 0 && batch == 1 && c->snap_span_pages > 0 && units <= grid && grid <= 4 * units && lone_cta_ok) ? 1 : 0;
         // one request and one layer class in the call: every unit has the same length, whatever it turns out to be
         int classes_in_call = 0;
         for (int i = 0; i < c->ncls; ++i) classes_in_call += p.cls_layers_in_call[i] > 0;
